@@ -1,0 +1,98 @@
+"""Seeded synthetic inputs and workload shapes.
+
+This module holds no arithmetic of the method: only the layer lists of the
+benchmark workloads and the seeded generators for initial weights, minibatches
+and labels.  Tests hand the *same arrays* to the CUDA library and to the CPU
+oracle.
+
+Recipe: weights are He-normal, ``std = sqrt(2 / fan_in)`` (conv fan_in =
+R*S*Cin), biases zero, drawn layer after layer from ``default_rng(seed)``;
+minibatch ``n`` is N(0,1) from ``default_rng(1000 + n)``; labels of minibatch
+``n`` are uniform integers from ``default_rng(2000 + n)``.
+"""
+import numpy as np
+
+
+def fc(n_in, n_out, act="relu", bias=True):
+    return dict(kind="fc", n_in=n_in, n_out=n_out, act=act, pool=0, bias=bias)
+
+
+def conv(c_in, c_out, H, W, act="relu", pool=0, bias=True):
+    return dict(kind="conv", n_in=c_in, n_out=c_out, H=H, W=W, R=3, S=3, pad=1,
+                stride=1, act=act, pool=pool, bias=bias)
+
+
+def mlp(widths, act):
+    L = len(widths) - 1
+    return [fc(widths[i], widths[i + 1], act if i < L - 1 else "none") for i in range(L)]
+
+
+def vgg(hw, plan, fcs, act="relu"):
+    """plan: list of channel counts with 'P' marking a 2x2 max-pool after the
+    preceding conv."""
+    layers, c, h = [], 3, hw
+    for i, item in enumerate(plan):
+        if item == "P":
+            continue
+        pool = 2 if i + 1 < len(plan) and plan[i + 1] == "P" else 0
+        layers.append(conv(c, item, h, h, act, pool))
+        c = item
+        if pool:
+            h //= 2
+    n_in = c * h * h
+    for j, w in enumerate(fcs):
+        layers.append(fc(n_in, w, act if j < len(fcs) - 1 else "none"))
+        n_in = w
+    return layers
+
+
+# The five workloads: (layers, batch, stages, delays or None = planner, lr, momentum, parity steps)
+WORKLOADS = {
+    "mlp4_784": dict(layers=mlp([784, 256, 256, 256, 10], "relu"), batch=32, stages=4,
+                     delays=[3, 2, 1, 0], lr=0.01, momentum=0.0, steps=10),
+    "mlp8_4096": dict(layers=mlp([4096] * 8 + [1000], "gelu"), batch=256, stages=8,
+                      delays=[7, 6, 5, 4, 3, 2, 1, 0], lr=0.01, momentum=0.9, steps=50),
+    "vgg_small_32": dict(layers=vgg(32, [64, 64, "P", 128, 128, "P", 256, 256, "P"], [512, 10]),
+                         batch=128, stages=7, delays=None, lr=0.01, momentum=0.0, steps=10),
+    "vgg16_224": dict(layers=vgg(224, [64, 64, "P", 128, 128, "P", 256, 256, 256, "P",
+                                       512, 512, 512, "P", 512, 512, 512, "P"],
+                                 [4096, 4096, 1000]),
+                      batch=64, stages=9, delays=None, lr=0.01, momentum=0.0, steps=10),
+    "mlp16_8192": dict(layers=mlp([8192] * 17, "gelu"), batch=2048, stages=9, delays=None,
+                       lr=0.01, momentum=0.0, steps=10),
+}
+
+
+def weight_shape(layer):
+    if layer["kind"] == "fc":
+        return (layer["n_out"], layer["n_in"])
+    return (layer["n_out"], layer["R"], layer["S"], layer["n_in"])
+
+
+def input_shape(layers, batch):
+    l0 = layers[0]
+    if l0["kind"] == "fc":
+        return (batch, l0["n_in"])
+    return (batch, l0["H"], l0["W"], l0["n_in"])
+
+
+def n_classes(layers):
+    return layers[-1]["n_out"]
+
+
+def initial_weights(layers, seed=0):
+    rng = np.random.default_rng(seed)
+    W0, b0 = [], []
+    for l in layers:
+        shp = weight_shape(l)
+        fan_in = int(np.prod(shp[1:]))
+        W0.append((rng.standard_normal(shp, dtype=np.float32) *
+                   np.float32(np.sqrt(2.0 / fan_in))).astype(np.float32))
+        b0.append(np.zeros(l["n_out"], dtype=np.float32))
+    return W0, b0
+
+
+def minibatch(layers, batch, n):
+    x = np.random.default_rng(1000 + n).standard_normal(input_shape(layers, batch), dtype=np.float32)
+    y = np.random.default_rng(2000 + n).integers(0, n_classes(layers), size=batch).astype(np.int32)
+    return x, y
