@@ -1,0 +1,185 @@
+/*
+ * layerpipe.h -- C ABI of the LayerPipe training hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library trains a chain of layers with the paper's delayed-gradient scheme:
+ * per layer the forward contraction (Eqs. 1-2), then a backward pass split into two
+ * independent tasks, the activation gradient ("delta", Eqs. 3-4) and the weight
+ * gradient ("G", Eq. 5), and the delayed update W(n) = W(n-1) - eta G(n-M) (Eq. 6)
+ * with the weight / activation stashes that retiming leaves on the W->delta and
+ * a->backward edges (Section III-A).  The paper's processors are stages mapped onto
+ * streams of ONE GPU; there is no multi-GPU path.
+ *
+ * Conventions
+ *   - every function returns LP_OK (0) or a negative LP_ERR_* code; nothing throws,
+ *     aborts or prints.  lp_last_error() gives a human-readable reason.
+ *   - "host" / "device" in a parameter comment says where the pointer must live.
+ *   - the caller owns every buffer it passes.  The library allocates no device memory:
+ *     all of its state lives inside the caller's workspace (lp_workspace_size bytes,
+ *     256-byte aligned, must outlive the handle).  Initial weights are copied.
+ *   - layouts at the boundary: FC weights W[out][in] row-major fp32 (the paper's
+ *     out x in matrix of Eq. 1); minibatch [batch][in] row-major.
+ *   - lp_step is asynchronous and never synchronises the device.
+ *   - a handle is not thread-safe; use one host thread per handle.
+ */
+#ifndef LAYERPIPE_H_
+#define LAYERPIPE_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lp_ctx* lp_handle;
+
+enum {
+  LP_OK = 0,
+  LP_ERR_INVALID_ARG = -1,  /* null pointer, bad index, bad shape; no side effects      */
+  LP_ERR_UNSUPPORTED = -2,  /* not an sm_100 device, or a layer kind not built yet       */
+  LP_ERR_WORKSPACE = -3,    /* workspace too small or misaligned                         */
+  LP_ERR_CUDA = -4,         /* a CUDA call failed; the handle is latched into this state */
+  LP_ERR_TIMEOUT = -5,      /* a bounded device-side wait gave up (see lp_device_status) */
+  LP_ERR_NOT_READY = -6     /* the requested step's data is not (or no longer) held      */
+};
+
+enum { LP_FC = 0, LP_CONV = 1 };
+enum { LP_ACT_NONE = 0, LP_ACT_RELU = 1, LP_ACT_GELU = 2 }; /* GELU = exact erf form */
+enum { LP_SCHED_LAYERPIPE = 0, /* delta and G of a layer are separate concurrent tasks;   */
+                               /* delta^{l-1} is released as soon as delta finishes        */
+       LP_SCHED_FUSED_B = 1 }; /* PipeDream-style: delta, G, update = ONE serial task      */
+enum { LP_F32 = 0, LP_BF16 = 1 };
+enum { LP_CAPTURE_GRADS = 1u }; /* keep G of the latest step readable by lp_get_grads */
+
+/* One layer of the chain (Eqs. 1-2: z = W a (+ b), a = f(z)). */
+typedef struct {
+  int kind;                      /* LP_FC | LP_CONV                                        */
+  int in, out;                   /* FC: features in / out.  CONV: channels in / out        */
+  int H, W, R, S, stride, pad;   /* CONV only: input height/width, filter, stride, padding */
+  int act;                       /* LP_ACT_*; the last layer must be LP_ACT_NONE           */
+  int pool;                      /* 0, or 2 = 2x2 stride-2 max pool after the activation   */
+  int has_bias;                  /* 0 = the paper's bias-free Eq. 1                        */
+} lp_layer;
+
+typedef struct {
+  int batch;          /* minibatch size B                                                  */
+  float lr;           /* eta of Eq. 6                                                      */
+  float momentum;     /* mu: m <- mu m + G, W <- W - eta m; 0 = plain Eq. 6                */
+  int schedule;       /* LP_SCHED_*                                                        */
+  int input_dtype;    /* dtype of lp_step's batch: LP_F32 | LP_BF16                        */
+  unsigned flags;     /* LP_CAPTURE_GRADS, ...                                             */
+} lp_config;
+
+/*
+ * Algorithm 1 (partitioning for balanced pipeline generation) on an integer cost model:
+ * T_fix[l] = 2 x MACs of layer l (forward + G), T_flex[l] = MACs (delta; 0 for layer 0).
+ * Layers are walked in reverse, processors filled up to T_p = ceil(T_tot / n_stages);
+ * a delta that does not fit is split into delta'' (stays beside layer l+1) and delta'
+ * (next processor); if more than n_stages processors are needed T_p is relaxed by 1%
+ * and the allocation restarts.  All outputs are host arrays owned by the caller.
+ *   stage_out[n_layers]        stage holding layer l's forward, G and update
+ *   delay_out[n_layers]        d_l = stages_used - 1 - stage(l)
+ *   dgrad_stage_out[2*n_layers], dgrad_amount_out[2*n_layers]
+ *                              the (at most two) pieces of layer l's delta work:
+ *                              [2l] = piece placed first (delta'' or the whole),
+ *                              [2l+1] = delta' (amount 0 and stage -1 if unsplit)
+ *   stages_used, Tp_out, relax_rounds_out   scalars (may be NULL)
+ * Errors: LP_ERR_INVALID_ARG for null arrays, n_layers < 1, n_stages < 1, bad shapes.
+ */
+int lp_plan(const lp_layer* layers, int n_layers, int batch, int n_stages,
+            int* stage_out, int* delay_out, int* dgrad_stage_out,
+            long long* dgrad_amount_out, int* stages_used, long long* Tp_out,
+            int* relax_rounds_out);
+
+/* Same allocation from caller-supplied integer costs (e.g. profiled times); this is the
+ * form in which the paper's worked example (Table II -> Table III) is stated. */
+int lp_plan_costs(const long long* T_fix, const long long* T_flex, int n_layers, int n_stages,
+                  int* stage_out, int* delay_out, int* dgrad_stage_out,
+                  long long* dgrad_amount_out, int* stages_used, long long* Tp_out,
+                  int* relax_rounds_out);
+
+/* Bytes of device workspace lp_create needs for this network.  `delays` host [n_layers]
+ * (NULL = one per stage after the layer, from `stage`); `stage` host [n_layers] (NULL =
+ * lp_plan).  Pure host arithmetic; needs no GPU. */
+int lp_workspace_size(const lp_layer* layers, int n_layers, int n_stages, const int* stage,
+                      const int* delays, const lp_config* cfg, size_t* bytes_out);
+
+/*
+ * Build a trainer.  `stage` / `delays`: host [n_layers] or NULL as above; a delay d_l
+ * means minibatch n reads weight version max(0, n - d_l) of layer l in BOTH its forward
+ * and its delta pass (weight stashing, Section III-A); the ring of layer l holds
+ * d_l + 1 bf16 versions.  W0_host[l] (fp32, [out][in]) and b0_host[l] (fp32 [out], may be
+ * NULL = zeros or has_bias = 0) are copied before the call returns.  workspace_dev:
+ * device, 256-byte aligned, >= lp_workspace_size bytes; zeroed by this call.
+ * Uses the current CUDA device; creates its own streams and events.
+ */
+int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, int n_stages,
+              const int* stage, const int* delays, const lp_config* cfg,
+              const float* const* W0_host, const float* const* b0_host,
+              void* workspace_dev, size_t workspace_bytes);
+
+/*
+ * Enqueue every task of one minibatch: cast+stash of the batch, forward of all layers,
+ * loss, and per layer delta / G / update under the handle's schedule.  batch_dev: device,
+ * [batch][in] of cfg.input_dtype; labels_dev: device int32 [batch], values in [0, classes).
+ * `stream` (a cudaStream_t, may be 0) orders the call after the caller's earlier work;
+ * the batch and labels are consumed by the first kernel, which runs on `stream`, so the
+ * caller may overwrite them after later work on `stream`.  Tasks of consecutive calls
+ * overlap on the device as far as the delays allow.
+ */
+int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev, void* stream);
+
+/* Make `stream` wait for everything enqueued so far (all updates applied: every layer
+ * holds version = number of lp_step calls). Does not block the host. */
+int lp_flush(lp_handle h, void* stream);
+
+/* Copy layer `layer`'s fp32 master weights (host W_out [out][in], b_out [out], either may
+ * be NULL) after waiting for its last enqueued update; *version = updates applied. */
+int lp_get_weights(lp_handle h, int layer, float* W_out, float* b_out, long long* version);
+
+/* G (host dW_out [out][in]) and bias gradient (host db_out [out]) of minibatch `step`;
+ * only the most recently enqueued step is held -> otherwise LP_ERR_NOT_READY. Blocks the
+ * host until that step's G task has finished. */
+int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* db_out);
+
+/* Plan actually in use: host arrays [n_layers] (any may be NULL). ring_slots = d_l + 1. */
+int lp_get_schedule(lp_handle h, int* stage, int* delay, int* ring_slots);
+
+/* For minibatch `step`: per layer the weight version read by forward (v_fwd) and by delta
+ * (v_bwd) and the ring slot it sat in.  Host arrays [n_layers].  Integer bookkeeping of
+ * the last 4096 steps. */
+int lp_get_version_log(lp_handle h, long long step, int* v_fwd, int* v_bwd, int* slot);
+
+/* Mean cross-entropy of minibatch `step` (one of the last 256 steps); blocks the host
+ * until that step's loss kernel has finished. */
+int lp_get_loss(lp_handle h, long long step, float* loss);
+
+/* 0, or the first non-zero status word written by a kernel whose bounded wait expired
+ * (then returns LP_ERR_TIMEOUT and fills *detail). Blocks until the device is idle. */
+int lp_device_status(lp_handle h, int* detail);
+
+/* Number of kernels this handle has launched so far. */
+long long lp_kernel_launches(lp_handle h);
+
+/* Tuning hook for experiments: force the GEMM tile width (64, 128, 256; 0 = automatic) and
+ * the shared-memory pipeline depth (0 = automatic) for handles created afterwards. */
+int lp_set_tuning(int tile_n, int stages);
+
+const char* lp_last_error(lp_handle h); /* valid until the next call on h; h may be NULL */
+int lp_destroy(lp_handle h);
+
+/*
+ * The three contractions of an FC layer in isolation, on caller-owned device buffers
+ * (bf16 operands, fp32 accumulate, fp32 result C[M][ldc]); for kernel-level checks.
+ *   which = 0  forward  (Eq. 1):  C[M][N] = A[M][K] . B[N][K]^T     (A = a, B = W)
+ *   which = 1  delta    (Eq. 4):  C[M][N] = A[M][K] . B[K][N]       (A = delta, B = W)
+ *   which = 2  G        (Eq. 5):  C[M][N] = A[K][M]^T . B[K][N]     (A = delta, B = a)
+ * lda / ldb / ldc are row pitches in elements; lda and ldb must be multiples of 8, ldc of
+ * 4; all base pointers 16-byte aligned.  `stream` is a cudaStream_t.
+ */
+int lp_gemm_bf16(int which, int M, int N, int K, const void* A_dev, int lda,
+                 const void* B_dev, int ldb, float* C_dev, int ldc, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAYERPIPE_H_ */

@@ -1,0 +1,67 @@
+// Internal declarations shared by the host-side translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
+#include <string>
+#include <vector>
+
+#include "../../include/layerpipe.h"
+
+namespace lp {
+
+// ---- gemm.cu ---------------------------------------------------------------
+// Encode a 2-D bf16 tensor map (128-byte swizzle, zero fill out of bounds).
+// inner/outer are the logical extents in elements, pitch_elems the row pitch.
+int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
+                      uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer, std::string* err);
+
+struct GemmArgs;
+// which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
+// Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
+// (see gemm_box_dims).
+int gemm_pick_bn(int which, int M, int N, int K);
+void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]);
+cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const GemmArgs& args, cudaStream_t stream);
+cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process
+void gemm_set_tuning(int bn, int stages);   // 0 = automatic
+
+// ---- planner.cpp ------------------------------------------------------------
+struct PlanResult {
+  std::vector<int> stage, delay;
+  std::vector<int> piece_stage;          // [2*L]
+  std::vector<long long> piece_amount;   // [2*L]
+  int used = 0;
+  long long Tp = 0;
+  int rounds = 0;
+};
+int plan_layers(const lp_layer* layers, int L, int batch, int Np, PlanResult* out);
+
+// ---- elementwise.cu ---------------------------------------------------------
+cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                              int* labels_copy, int B, int n_in, int ld, cudaStream_t stream);
+cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
+                                float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
+                                cudaStream_t stream);
+struct UpdateArgs {
+  const float* dW;      // [out][ldw] fp32 (pad lanes zero)
+  float* W;             // master [out][ldw]
+  float* mW;            // momentum or null
+  __nv_bfloat16* ring;  // bf16 slot that receives RN(W)
+  long long n_elems;    // out * ldw (multiple of 8)
+  const __nv_bfloat16* delta;  // [rows][ldd]: bias gradient = column sums (null: no bias)
+  int rows, ldd, n_out;
+  float* b;             // master bias
+  float* mb;            // bias momentum or null
+  float* db;            // bias gradient out
+  float* bring;         // fp32 bias slot that receives b
+  float lr, mu;
+};
+cudaError_t launch_sgd_update(const UpdateArgs& a, cudaStream_t stream);
+cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long n_elems, cudaStream_t stream);
+
+}  // namespace lp

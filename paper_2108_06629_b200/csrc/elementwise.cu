@@ -1,0 +1,233 @@
+// HBM-bound kernels of the training step: input cast + stash, softmax cross-entropy with
+// delta^L, and the fused SGD update (Eq. 6) that also refreshes the bf16 weight-ring slot.
+#include "common.h"
+
+namespace lp {
+
+// ---------------------------------------------------------------------------
+// a^0 = RN_bf16(batch) into the first layer's activation-stash slot; labels are copied
+// into the library's label ring so that the caller may reuse its buffers.
+__global__ void cast_stash_kernel(const void* __restrict__ batch, int input_is_bf16,
+                                  const int* __restrict__ labels, __nv_bfloat16* __restrict__ x0,
+                                  int* __restrict__ labels_copy, int B, int n_in, int ld) {
+  const long long groups_per_row = ld / 8;
+  const long long total = (long long)B * groups_per_row;
+  for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
+       g += (long long)gridDim.x * blockDim.x) {
+    const int row = int(g / groups_per_row);
+    const int c0 = int(g % groups_per_row) * 8;
+    float v[8];
+    if (input_is_bf16) {
+      const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(batch) + (long long)row * n_in;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = (c0 + j < n_in) ? __bfloat162float(src[c0 + j]) : 0.f;
+    } else {
+      const float* src = reinterpret_cast<const float*>(batch) + (long long)row * n_in;
+      if ((n_in & 3) == 0 && c0 + 8 <= n_in) {
+        const float4 a = *reinterpret_cast<const float4*>(src + c0);
+        const float4 b = *reinterpret_cast<const float4*>(src + c0 + 4);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (c0 + j < n_in) ? src[c0 + j] : 0.f;
+      }
+    }
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]);
+    __nv_bfloat162 p1 = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]);
+    __nv_bfloat162 p3 = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&p0);
+    o.y = *reinterpret_cast<uint32_t*>(&p1);
+    o.z = *reinterpret_cast<uint32_t*>(&p2);
+    o.w = *reinterpret_cast<uint32_t*>(&p3);
+    *reinterpret_cast<uint4*>(x0 + (long long)row * ld + c0) = o;
+  }
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i < B; i += blockDim.x) labels_copy[i] = labels[i];
+  }
+}
+
+cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                              int* labels_copy, int B, int n_in, int ld, cudaStream_t stream) {
+  const long long total = (long long)B * (ld / 8);
+  int blocks = int(std::min<long long>((total + 255) / 256, 148 * 8));
+  if (blocks < 1) blocks = 1;
+  cast_stash_kernel<<<blocks, 256, 0, stream>>>(batch, input_is_bf16, labels, x0, labels_copy, B, n_in, ld);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// One block per row: p = softmax(z^L), delta^L = RN((p - onehot)/B), row loss; the last
+// block to finish adds the row losses in row order (deterministic mean).
+__device__ __forceinline__ float block_reduce(float v, float* sh, bool is_max) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, v, o);
+    v = is_max ? fmaxf(v, other) : v + other;
+  }
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  const int nw = blockDim.x >> 5;
+  float r = sh[0];
+  for (int i = 1; i < nw; ++i) r = is_max ? fmaxf(r, sh[i]) : r + sh[i];
+  return r;
+}
+
+__global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const int* __restrict__ labels,
+                                    __nv_bfloat16* __restrict__ delta, int ldd, float* __restrict__ row_loss,
+                                    unsigned* __restrict__ ticket, float* __restrict__ loss_out, int B, int C) {
+  __shared__ float sh[32];
+  __shared__ bool last;
+  const int row = blockIdx.x;
+  const float* z = zL + (long long)row * ldz;
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) mx = fmaxf(mx, z[c]);
+  mx = block_reduce(mx, sh, true);
+  float s = 0.f;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) s += expf(z[c] - mx);
+  s = block_reduce(s, sh, false);
+  const int y = labels[row];
+  const float invB = 1.0f / float(B);
+  const float inv_s = 1.0f / s;
+  __nv_bfloat16* d = delta + (long long)row * ldd;
+  const int Cpad = (C + 7) & ~7;
+  for (int c = threadIdx.x; c < Cpad; c += blockDim.x) {
+    float v = 0.f;
+    if (c < C) v = (expf(z[c] - mx) * inv_s - (c == y ? 1.f : 0.f)) * invB;
+    d[c] = __float2bfloat16_rn(v);
+  }
+  if (threadIdx.x == 0) {
+    row_loss[row] = -((z[y] - mx) - logf(s));
+    __threadfence();
+    const unsigned t = atomicAdd(ticket, 1u);
+    last = (t == unsigned(B) - 1u);
+  }
+  __syncthreads();
+  if (last && threadIdx.x == 0) {
+    __threadfence();
+    float acc = 0.f;
+    for (int i = 0; i < B; ++i) acc += __ldcg(row_loss + i);
+    *loss_out = acc * invB;
+    *ticket = 0u;     // ready for the next launch on this scratch
+  }
+}
+
+cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
+                                float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
+                                cudaStream_t stream) {
+  softmax_xent_kernel<<<B, 256, 0, stream>>>(zL, ldz, labels, delta, ldd, row_loss, ticket, loss_out, B, C);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Fused update (Eq. 6, optional momentum): m <- mu m + G; W <- W - eta m; ring <- RN(W).
+// 8 elements per thread, 128-bit loads and stores throughout.  Blocks past the weight
+// range own 64 bias columns each: bias gradient = column sums of delta (row order),
+// then the same update for the bias.
+constexpr int UPD_THREADS = 256;
+constexpr int UPD_VEC_PER_THREAD = 2;     // x 8 elements
+constexpr int BIAS_COLS = 64;
+
+__global__ void __launch_bounds__(UPD_THREADS) sgd_update_kernel(const UpdateArgs a, int w_blocks) {
+  if (int(blockIdx.x) < w_blocks) {
+    const long long nvec = a.n_elems >> 3;
+    const long long base = (long long)blockIdx.x * (UPD_THREADS * UPD_VEC_PER_THREAD) + threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < UPD_VEC_PER_THREAD; ++u) {
+      const long long v = base + (long long)u * UPD_THREADS;
+      if (v >= nvec) break;
+      const long long e = v << 3;
+      const float4 g0 = __ldcs(reinterpret_cast<const float4*>(a.dW + e));
+      const float4 g1 = __ldcs(reinterpret_cast<const float4*>(a.dW + e + 4));
+      float4 w0 = *reinterpret_cast<const float4*>(a.W + e);
+      float4 w1 = *reinterpret_cast<const float4*>(a.W + e + 4);
+      float4 m0 = g0, m1 = g1;
+      if (a.mW != nullptr) {
+        const float4 p0 = *reinterpret_cast<const float4*>(a.mW + e);
+        const float4 p1 = *reinterpret_cast<const float4*>(a.mW + e + 4);
+        m0.x = a.mu * p0.x + g0.x; m0.y = a.mu * p0.y + g0.y; m0.z = a.mu * p0.z + g0.z; m0.w = a.mu * p0.w + g0.w;
+        m1.x = a.mu * p1.x + g1.x; m1.y = a.mu * p1.y + g1.y; m1.z = a.mu * p1.z + g1.z; m1.w = a.mu * p1.w + g1.w;
+        *reinterpret_cast<float4*>(a.mW + e) = m0;
+        *reinterpret_cast<float4*>(a.mW + e + 4) = m1;
+      }
+      w0.x -= a.lr * m0.x; w0.y -= a.lr * m0.y; w0.z -= a.lr * m0.z; w0.w -= a.lr * m0.w;
+      w1.x -= a.lr * m1.x; w1.y -= a.lr * m1.y; w1.z -= a.lr * m1.z; w1.w -= a.lr * m1.w;
+      *reinterpret_cast<float4*>(a.W + e) = w0;
+      *reinterpret_cast<float4*>(a.W + e + 4) = w1;
+      __nv_bfloat162 q0 = __floats2bfloat162_rn(w0.x, w0.y);
+      __nv_bfloat162 q1 = __floats2bfloat162_rn(w0.z, w0.w);
+      __nv_bfloat162 q2 = __floats2bfloat162_rn(w1.x, w1.y);
+      __nv_bfloat162 q3 = __floats2bfloat162_rn(w1.z, w1.w);
+      uint4 o;
+      o.x = *reinterpret_cast<uint32_t*>(&q0);
+      o.y = *reinterpret_cast<uint32_t*>(&q1);
+      o.z = *reinterpret_cast<uint32_t*>(&q2);
+      o.w = *reinterpret_cast<uint32_t*>(&q3);
+      *reinterpret_cast<uint4*>(a.ring + e) = o;
+    }
+    return;
+  }
+  // ---- bias part: this block owns BIAS_COLS columns --------------------------
+  __shared__ float part[UPD_THREADS / BIAS_COLS][BIAS_COLS];
+  const int cb = (int(blockIdx.x) - w_blocks) * BIAS_COLS;
+  const int tx = threadIdx.x % BIAS_COLS, ty = threadIdx.x / BIAS_COLS;
+  constexpr int NY = UPD_THREADS / BIAS_COLS;
+  const int col = cb + tx;
+  float acc = 0.f;
+  if (col < a.n_out) {
+    for (int r = ty; r < a.rows; r += NY) acc += __bfloat162float(a.delta[(long long)r * a.ldd + col]);
+  }
+  part[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && col < a.n_out) {
+    float g = 0.f;
+#pragma unroll
+    for (int i = 0; i < NY; ++i) g += part[i][tx];
+    a.db[col] = g;
+    float m = g;
+    if (a.mb != nullptr) {
+      m = a.mu * a.mb[col] + g;
+      a.mb[col] = m;
+    }
+    const float b = a.b[col] - a.lr * m;
+    a.b[col] = b;
+    a.bring[col] = b;
+  }
+}
+
+cudaError_t launch_sgd_update(const UpdateArgs& a, cudaStream_t stream) {
+  const long long nvec = a.n_elems >> 3;
+  const long long per_block = UPD_THREADS * UPD_VEC_PER_THREAD;
+  const int w_blocks = int((nvec + per_block - 1) / per_block);
+  const int b_blocks = a.delta ? (a.n_out + BIAS_COLS - 1) / BIAS_COLS : 0;
+  sgd_update_kernel<<<w_blocks + b_blocks, UPD_THREADS, 0, stream>>>(a, w_blocks);
+  return cudaGetLastError();
+}
+
+}  // namespace lp
+
+namespace lp {
+// dst = RN_bf16(src), n a multiple of 8 (used once per layer to seed ring slot 0).
+__global__ void round_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, long long nvec) {
+  for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nvec; v += (long long)gridDim.x * blockDim.x) {
+    const float4 a = *reinterpret_cast<const float4*>(src + v * 8);
+    const float4 b = *reinterpret_cast<const float4*>(src + v * 8 + 4);
+    __nv_bfloat162 q0 = __floats2bfloat162_rn(a.x, a.y), q1 = __floats2bfloat162_rn(a.z, a.w);
+    __nv_bfloat162 q2 = __floats2bfloat162_rn(b.x, b.y), q3 = __floats2bfloat162_rn(b.z, b.w);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&q0); o.y = *reinterpret_cast<uint32_t*>(&q1);
+    o.z = *reinterpret_cast<uint32_t*>(&q2); o.w = *reinterpret_cast<uint32_t*>(&q3);
+    *reinterpret_cast<uint4*>(dst + v * 8) = o;
+  }
+}
+cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long n_elems, cudaStream_t stream) {
+  const long long nvec = n_elems >> 3;
+  int blocks = int(std::min<long long>((nvec + 255) / 256, 148 * 16));
+  if (blocks < 1) blocks = 1;
+  round_to_bf16_kernel<<<blocks, 256, 0, stream>>>(src, dst, nvec);
+  return cudaGetLastError();
+}
+}  // namespace lp

@@ -1,0 +1,170 @@
+// Host side of the tcgen05 GEMM: tensor-map encoding, tile selection, launch, and the
+// stand-alone lp_gemm_bf16 entry point.
+#include "gemm.cuh"
+
+#include <algorithm>
+#include <mutex>
+
+#include "common.h"
+
+namespace lp {
+
+// ---------------------------------------------------------------------------
+// cuTensorMapEncodeTiled is a driver API; fetch it through the runtime so the library has
+// no link-time dependency on libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn(std::string* err) {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  static std::string first_err;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || p == nullptr) {
+      first_err = std::string("cuTensorMapEncodeTiled unavailable: ") + cudaGetErrorString(e);
+    } else {
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+  });
+  if (!fn && err) *err = first_err;
+  return fn;
+}
+
+int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+                      uint32_t box_inner, uint32_t box_outer, std::string* err) {
+  EncodeTiledFn fn = get_encode_fn(err);
+  if (!fn) return LP_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch_elems & 7) || box_inner != 64 || box_outer > 256) {
+    if (err) *err = "tensor map: base must be 16-byte aligned, pitch a multiple of 8 elements, box <= 256";
+    return LP_ERR_INVALID_ARG;
+  }
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string(int(r));
+    return LP_ERR_CUDA;
+  }
+  return LP_OK;
+}
+
+// ---------------------------------------------------------------------------
+static int g_force_bn = 0;
+static int g_force_stages = 0;
+void gemm_set_tuning(int bn, int stages) {
+  g_force_bn = bn;
+  g_force_stages = stages;
+}
+
+int gemm_pick_bn(int which, int M, int N, int K) {
+  (void)which; (void)M; (void)K;
+  if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
+  if (N <= 64) return 64;
+  return 128;
+}
+
+void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]) {
+  const bool a_mn = (which == 2), b_mn = (which != 0);
+  boxA[0] = 64; boxA[1] = a_mn ? 64 : GEMM_BM;
+  boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(bn);
+}
+
+static int pick_stages(int bn, int K) {
+  const int stage_bytes = GEMM_A_BYTES + bn * GEMM_BK * 2;
+  int s = g_force_stages > 0 ? g_force_stages : (100 * 1024) / stage_bytes;   // two CTAs per SM
+  s = std::min(s, GEMM_MAX_STAGES);
+  const int num_kb = (K + GEMM_BK - 1) / GEMM_BK;
+  s = std::max(2, std::min(s, std::max(num_kb, 2)));
+  while (s > 2 && size_t(s) * stage_bytes + 1280 > 227 * 1024) --s;
+  return s;
+}
+
+template <int BN, bool A_MN, bool B_MN>
+static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
+  a.num_stages = pick_stages(BN, a.K);
+  const size_t smem = GemmSmem<BN>::bytes(a.num_stages);
+  dim3 grid((a.M + GEMM_BM - 1) / GEMM_BM, (a.N + BN - 1) / BN, 1);
+  gemm_tcgen05_kernel<BN, A_MN, B_MN><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a);
+  return cudaGetLastError();
+}
+
+template <int BN, bool A_MN, bool B_MN>
+static cudaError_t configure_one() {
+  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              227 * 1024);
+}
+
+cudaError_t gemm_configure() {
+  cudaError_t e;
+#define LP_CFG(BN)                                                        \
+  if ((e = configure_one<BN, false, false>()) != cudaSuccess) return e;   \
+  if ((e = configure_one<BN, false, true>()) != cudaSuccess) return e;    \
+  if ((e = configure_one<BN, true, true>()) != cudaSuccess) return e;
+  LP_CFG(64) LP_CFG(128) LP_CFG(256)
+#undef LP_CFG
+  return cudaSuccess;
+}
+
+cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
+                        cudaStream_t st) {
+#define LP_DISPATCH(BN)                                                       \
+  case BN:                                                                    \
+    if (which == 0) return launch_one<BN, false, false>(tmA, tmB, args, st);  \
+    if (which == 1) return launch_one<BN, false, true>(tmA, tmB, args, st);   \
+    return launch_one<BN, true, true>(tmA, tmB, args, st);
+  switch (bn) {
+    LP_DISPATCH(64)
+    LP_DISPATCH(128)
+    LP_DISPATCH(256)
+  }
+#undef LP_DISPATCH
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace lp
+
+// status word for the stand-alone entry point (handles keep theirs in the workspace)
+__device__ int g_gemm_status = 0;
+
+// ---------------------------------------------------------------------------
+extern "C" int lp_gemm_bf16(int which, int M, int N, int K, const void* A, int lda, const void* B, int ldb,
+                            float* C, int ldc, void* stream) {
+  using namespace lp;
+  if (which < 0 || which > 2 || M < 1 || N < 1 || K < 1 || !A || !B || !C) return LP_ERR_INVALID_ARG;
+  if ((lda & 7) || (ldb & 7) || (ldc & 3)) return LP_ERR_INVALID_ARG;
+  static int* status_dev = nullptr;   // address of g_gemm_status on the device first used
+  if (!status_dev) {
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status_dev), g_gemm_status) != cudaSuccess) return LP_ERR_CUDA;
+    if (gemm_configure() != cudaSuccess) return LP_ERR_CUDA;
+  }
+  const int bn = gemm_pick_bn(which, M, N, K);
+  uint32_t boxA[2], boxB[2];
+  gemm_box_dims(which, bn, boxA, boxB);
+  CUtensorMap tmA, tmB;
+  std::string err;
+  int rc;
+  // A: forward/delta K-major -> rows = M, inner = K; G: stored [K][M] -> inner = M, rows = K
+  if (which == 2) rc = make_tmap_bf16_2d(&tmA, A, M, K, lda, boxA[0], boxA[1], &err);
+  else            rc = make_tmap_bf16_2d(&tmA, A, K, M, lda, boxA[0], boxA[1], &err);
+  if (rc != LP_OK) return rc;
+  // B: forward stored [N][K]; delta and G stored [K][N]
+  if (which == 0) rc = make_tmap_bf16_2d(&tmB, B, K, N, ldb, boxB[0], boxB[1], &err);
+  else            rc = make_tmap_bf16_2d(&tmB, B, N, K, ldb, boxB[0], boxB[1], &err);
+  if (rc != LP_OK) return rc;
+  GemmArgs a{};
+  a.M = M; a.N = N; a.K = K;
+  a.mode = EPI_STORE_F32;
+  a.out = C; a.ld_out = ldc;
+  a.status = status_dev;
+  cudaError_t e = gemm_launch(which, bn, tmA, tmB, a, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return LP_ERR_CUDA;
+  return LP_OK;
+}

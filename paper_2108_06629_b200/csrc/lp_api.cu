@@ -1,0 +1,711 @@
+// The trainer behind the C ABI: workspace layout, weight-version rings, activation
+// stashes, and the stage scheduler that maps the paper's processors onto CUDA streams.
+//
+// Scheduling model.  Every lp_step enqueues all tasks of one minibatch n:
+//   cast -> F_1..F_L -> loss -> for l = L..1 { delta_l , G_l -> U_l }
+// Each task declares the buffers (ring slots, stash slots, delta buffers) it reads and
+// writes; a small tracker turns read-after-write, write-after-read and write-after-write
+// hazards on those buffers into event waits between streams.  Because F_l(n) only needs
+// weight version max(0, n - d_l), tasks of consecutive minibatches overlap on the device
+// exactly as far as the delays allow -- the pipelining of Section III-A -- while the
+// results stay those of the minibatch-by-minibatch recursion.
+//   LayerPipe schedule: per stage three streams -- delta (highest priority: it carries
+//   the critical loop), forward, and G+update (lowest) -- so delta_l and G_l of one layer
+//   run concurrently and delta^{l-1} is released as soon as delta_l is done.
+//   Fused-B schedule: delta_l, G_l, U_l run back to back as ONE task on the stage's
+//   backward stream and delta^{l-1} is released only when the whole task has finished.
+#include <cstdio>
+#include <cstring>
+#include <memory>
+
+#include "common.h"
+#include "gemm.cuh"
+
+namespace lp {
+
+constexpr int kDeltaSlots = 2;
+constexpr int kLossRing = 256;
+constexpr int kLogRing = 4096;
+constexpr int kEventPool = 2048;
+constexpr int kExtraStashSlots = 1;   // activation stash = d_l + 1 (retiming) + 1 so F may run one ahead
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int pad8(int x) { return (x + 7) & ~7; }
+
+struct Ev {
+  cudaEvent_t e = nullptr;
+  cudaStream_t s = nullptr;
+};
+
+struct Res {                 // one buffer (or ring slot) the tracker protects
+  Ev last_write;
+  std::vector<Ev> readers;
+};
+
+struct Layer {
+  lp_layer d;
+  int stage = 0, delay = 0, slots = 1;
+  int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;
+  int x_slots = 1;
+  // device memory (all inside the workspace)
+  float *W = nullptr, *mW = nullptr, *b = nullptr, *mb = nullptr, *dW = nullptr, *db = nullptr, *bring = nullptr;
+  __nv_bfloat16 *ring = nullptr, *X = nullptr, *Z = nullptr, *delta = nullptr;
+  size_t w_elems = 0, x_elems = 0, z_elems = 0, delta_elems = 0;
+  int z_slots = 0;
+  int bn_f = 128, bn_d = 128, bn_g = 128;
+  std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
+  std::vector<Res> rX, rZ, rDelta, rRing;
+  Res rDW;
+  Ev last_update;
+};
+
+}  // namespace lp
+
+struct lp_ctx {
+  std::vector<lp::Layer> L;
+  lp_config cfg{};
+  int n_stages = 0;
+  int stages_used = 0;
+  int classes = 0, ld_cls = 0;
+  // shared buffers
+  float* zL = nullptr;          // [kDeltaSlots][B][ld_cls] fp32
+  int* labels = nullptr;        // [kDeltaSlots][B]
+  float* row_loss = nullptr;    // [kDeltaSlots][B]
+  unsigned* ticket = nullptr;   // [kDeltaSlots]
+  float* loss = nullptr;        // [kLossRing]
+  int* status = nullptr;        // device status word
+  std::vector<lp::Res> rZL, rLabels;
+  // streams / events
+  std::vector<cudaStream_t> sF, sD, sG;
+  std::vector<cudaEvent_t> pool;
+  size_t pool_next = 0;
+  std::vector<lp::Ev> loss_ev;
+  // bookkeeping
+  long long n_steps = 0;
+  long long launches = 0;
+  std::vector<int> log_v, log_slot;   // [kLogRing][L]
+  std::string err;
+  int latched = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+};
+
+namespace lp {
+
+static thread_local std::string g_err;   // for calls without a handle
+
+static int fail(lp_ctx* h, int code, const std::string& msg) {
+  if (h) {
+    h->err = msg;
+    if (code == LP_ERR_CUDA) h->latched = code;
+  } else {
+    g_err = msg;
+  }
+  return code;
+}
+#define LP_CUDA(h, call)                                                                        \
+  do {                                                                                          \
+    cudaError_t e__ = (call);                                                                   \
+    if (e__ != cudaSuccess)                                                                     \
+      return fail(h, LP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));         \
+  } while (0)
+
+// ---------------------------------------------------------------------------
+static int validate(const lp_layer* layers, int n, const lp_config* cfg, std::string* why) {
+  if (!layers || n < 1 || !cfg) { *why = "null layer list or config"; return LP_ERR_INVALID_ARG; }
+  if (cfg->batch < 1) { *why = "batch must be >= 1"; return LP_ERR_INVALID_ARG; }
+  if (cfg->schedule != LP_SCHED_LAYERPIPE && cfg->schedule != LP_SCHED_FUSED_B) { *why = "unknown schedule"; return LP_ERR_INVALID_ARG; }
+  if (cfg->input_dtype != LP_F32 && cfg->input_dtype != LP_BF16) { *why = "unknown input dtype"; return LP_ERR_INVALID_ARG; }
+  for (int l = 0; l < n; ++l) {
+    const lp_layer& y = layers[l];
+    if (y.kind != LP_FC && y.kind != LP_CONV) { *why = "unknown layer kind"; return LP_ERR_INVALID_ARG; }
+    if (y.in < 1 || y.out < 1) { *why = "layer sizes must be positive"; return LP_ERR_INVALID_ARG; }
+    if (y.act < LP_ACT_NONE || y.act > LP_ACT_GELU) { *why = "unknown activation"; return LP_ERR_INVALID_ARG; }
+    if (l == n - 1 && y.act != LP_ACT_NONE) { *why = "last layer must have no activation"; return LP_ERR_INVALID_ARG; }
+    if (y.kind == LP_CONV) { *why = "convolution layers are not built yet"; return LP_ERR_UNSUPPORTED; }
+    if (y.pool != 0) { *why = "pooling needs a convolution layer"; return LP_ERR_INVALID_ARG; }
+    if (l > 0 && layers[l - 1].out != y.in) { *why = "layer sizes do not chain"; return LP_ERR_INVALID_ARG; }
+  }
+  return LP_OK;
+}
+
+static int resolve_plan(const lp_layer* layers, int n, int n_stages, const int* stage, const int* delays,
+                        const lp_config* cfg, std::vector<int>* st, std::vector<int>* dl, int* used, std::string* why) {
+  if (n_stages < 1) { *why = "n_stages must be >= 1"; return LP_ERR_INVALID_ARG; }
+  st->assign(n, 0);
+  dl->assign(n, 0);
+  if (stage) {
+    int mx = 0;
+    for (int l = 0; l < n; ++l) {
+      if (stage[l] < 0 || stage[l] >= n_stages || (l > 0 && stage[l] < stage[l - 1])) {
+        *why = "stage map must be non-decreasing and within [0, n_stages)";
+        return LP_ERR_INVALID_ARG;
+      }
+      (*st)[l] = stage[l];
+      mx = std::max(mx, stage[l]);
+    }
+    *used = mx + 1;
+  } else {
+    PlanResult r;
+    int rc = plan_layers(layers, n, cfg->batch, n_stages, &r);
+    if (rc != LP_OK) { *why = "planner rejected the layer list"; return rc; }
+    *st = r.stage;
+    *used = r.used;
+    if (delays) {
+      // explicit delays with a planned stage map: keep the planner's stages for stream placement
+    }
+  }
+  for (int l = 0; l < n; ++l) {
+    (*dl)[l] = delays ? delays[l] : (*used - 1 - (*st)[l]);
+    if ((*dl)[l] < 0 || (*dl)[l] > 1024) { *why = "delays must be in [0, 1024]"; return LP_ERR_INVALID_ARG; }
+  }
+  return LP_OK;
+}
+
+// Lays the network out in the workspace.  With base == nullptr only sizes are computed.
+static size_t carve(lp_ctx* c, char* base) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    off = align_up(off, 256);
+    char* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  };
+  const int B = c->cfg.batch;
+  const bool mom = c->cfg.momentum != 0.f;
+  const int nL = int(c->L.size());
+  for (int l = 0; l < nL; ++l) {
+    Layer& y = c->L[l];
+    y.w_elems = size_t(y.n_out) * y.ld_in;
+    y.W = reinterpret_cast<float*>(take(y.w_elems * 4));
+    y.mW = mom ? reinterpret_cast<float*>(take(y.w_elems * 4)) : nullptr;
+    y.dW = reinterpret_cast<float*>(take(y.w_elems * 4));
+    y.ring = reinterpret_cast<__nv_bfloat16*>(take(y.w_elems * 2 * y.slots));
+    y.b = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4));
+    y.mb = mom ? reinterpret_cast<float*>(take(size_t(y.ld_out) * 4)) : nullptr;
+    y.db = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4));
+    y.bring = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4 * y.slots));
+    y.x_elems = size_t(B) * y.ld_in;
+    y.X = reinterpret_cast<__nv_bfloat16*>(take(y.x_elems * 2 * y.x_slots));
+    y.delta_elems = size_t(B) * y.ld_out;
+    y.delta = reinterpret_cast<__nv_bfloat16*>(take(y.delta_elems * 2 * kDeltaSlots));
+    y.z_slots = 0;
+    y.Z = nullptr;
+    if (y.d.act == LP_ACT_GELU && l + 1 < nL) {
+      y.z_slots = c->L[l + 1].x_slots;
+      y.z_elems = size_t(B) * y.ld_out;
+      y.Z = reinterpret_cast<__nv_bfloat16*>(take(y.z_elems * 2 * y.z_slots));
+    }
+  }
+  c->zL = reinterpret_cast<float*>(take(size_t(kDeltaSlots) * B * c->ld_cls * 4));
+  c->labels = reinterpret_cast<int*>(take(size_t(kDeltaSlots) * B * 4));
+  c->row_loss = reinterpret_cast<float*>(take(size_t(kDeltaSlots) * B * 4));
+  c->ticket = reinterpret_cast<unsigned*>(take(size_t(kDeltaSlots) * 4));
+  c->loss = reinterpret_cast<float*>(take(size_t(kLossRing) * 4));
+  c->status = reinterpret_cast<int*>(take(256));
+  return align_up(off, 256);
+}
+
+static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::vector<int>& st,
+                         const std::vector<int>& dl) {
+  c->L.resize(n);
+  for (int l = 0; l < n; ++l) {
+    Layer& y = c->L[l];
+    y.d = layers[l];
+    y.stage = st[l];
+    y.delay = dl[l];
+    y.slots = dl[l] + 1;
+    y.n_in = layers[l].in;
+    y.n_out = layers[l].out;
+    y.ld_in = pad8(y.n_in);
+    y.ld_out = pad8(y.n_out);
+    y.x_slots = y.delay + 1 + kExtraStashSlots;
+  }
+  c->classes = layers[n - 1].out;
+  c->ld_cls = pad8(c->classes);
+}
+
+// ---------------------------------------------------------------------------
+// hazard tracker
+static void wait_on(lp_ctx* c, cudaStream_t s, const Ev& e, std::vector<cudaEvent_t>* seen, cudaError_t* err) {
+  if (!e.e || e.s == s) return;
+  for (cudaEvent_t x : *seen) if (x == e.e) return;
+  seen->push_back(e.e);
+  cudaError_t r = cudaStreamWaitEvent(s, e.e, 0);
+  if (r != cudaSuccess && *err == cudaSuccess) *err = r;
+}
+
+static cudaError_t task_begin(lp_ctx* c, cudaStream_t s, std::initializer_list<Res*> reads,
+                              std::initializer_list<Res*> writes) {
+  std::vector<cudaEvent_t> seen;
+  cudaError_t err = cudaSuccess;
+  for (Res* r : reads) if (r) wait_on(c, s, r->last_write, &seen, &err);
+  for (Res* w : writes) {
+    if (!w) continue;
+    wait_on(c, s, w->last_write, &seen, &err);
+    for (const Ev& e : w->readers) wait_on(c, s, e, &seen, &err);
+  }
+  return err;
+}
+
+static cudaError_t task_end(lp_ctx* c, cudaStream_t s, std::initializer_list<Res*> reads,
+                            std::initializer_list<Res*> writes, Ev* out_ev) {
+  cudaEvent_t e = c->pool[c->pool_next++ % c->pool.size()];
+  cudaError_t r = cudaEventRecord(e, s);
+  Ev ev{e, s};
+  for (Res* x : reads) if (x) x->readers.push_back(ev);
+  for (Res* w : writes) {
+    if (!w) continue;
+    w->last_write = ev;
+    w->readers.clear();
+  }
+  if (out_ev) *out_ev = ev;
+  return r;
+}
+
+// ---------------------------------------------------------------------------
+static int build_tensor_maps(lp_ctx* c) {
+  const int B = c->cfg.batch;
+  const int nL = int(c->L.size());
+  std::string err;
+  for (int l = 0; l < nL; ++l) {
+    Layer& y = c->L[l];
+    y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
+    y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
+    y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
+    uint32_t bA[2], bB[2];
+    int rc;
+    // forward: A = a^{l-1} [B][in] K-major; B = W [out][in] K-major
+    gemm_box_dims(0, y.bn_f, bA, bB);
+    y.tm_f_A.resize(y.x_slots);
+    for (int s = 0; s < y.x_slots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_f_A[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bA[0], bA[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+    y.tm_f_B.resize(y.slots);
+    for (int s = 0; s < y.slots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+    // delta: A = delta^l [B][out] K-major (K = out); B = W [out][in] MN-major (N = in contiguous)
+    gemm_box_dims(1, y.bn_d, bA, bB);
+    y.tm_d_A.resize(kDeltaSlots);
+    for (int s = 0; s < kDeltaSlots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+    y.tm_d_B.resize(y.slots);
+    for (int s = 0; s < y.slots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+    // G: A = delta^l stored [B][out] -> MN-major (M = out contiguous); B = a^{l-1} stored [B][in] -> MN-major
+    gemm_box_dims(2, y.bn_g, bA, bB);
+    y.tm_g_A.resize(kDeltaSlots);
+    for (int s = 0; s < kDeltaSlots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+    y.tm_g_B.resize(y.x_slots);
+    for (int s = 0; s < y.x_slots; ++s)
+      if ((rc = make_tmap_bf16_2d(&y.tm_g_B[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
+        return fail(c, rc, err);
+  }
+  return LP_OK;
+}
+
+static void destroy_ctx(lp_ctx* c) {
+  if (!c) return;
+  auto kill = [](std::vector<cudaStream_t>& v) {
+    for (cudaStream_t s : v) if (s) cudaStreamDestroy(s);
+    v.clear();
+  };
+  cudaDeviceSynchronize();
+  kill(c->sF);
+  kill(c->sD);
+  kill(c->sG);
+  for (cudaEvent_t e : c->pool) if (e) cudaEventDestroy(e);
+  delete c;
+}
+
+// ---------------------------------------------------------------------------
+// the kernels of one minibatch
+static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
+  Layer& y = c->L[l];
+  const int nL = int(c->L.size());
+  const bool last = (l == nL - 1);
+  GemmArgs a{};
+  a.M = c->cfg.batch; a.N = y.n_out; a.K = y.n_in;
+  a.mode = EPI_FPROP;
+  a.act = y.d.act;
+  a.bias = y.d.has_bias ? y.bring + size_t(ring_slot) * y.ld_out : nullptr;
+  a.status = c->status;
+  if (last) {
+    a.out = nullptr;
+    a.out2 = c->zL + size_t(n % kDeltaSlots) * c->cfg.batch * c->ld_cls;
+    a.ld_out2 = c->ld_cls;
+    a.out2_is_f32 = 1;
+  } else {
+    Layer& nx = c->L[l + 1];
+    a.out = nx.X + size_t(n % nx.x_slots) * nx.x_elems;
+    a.ld_out = nx.ld_in;
+    if (y.Z) {
+      a.out2 = y.Z + size_t(n % y.z_slots) * y.z_elems;
+      a.ld_out2 = y.ld_out;
+    }
+  }
+  ++c->launches;
+  return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
+}
+
+static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
+  Layer& y = c->L[l];
+  Layer& pv = c->L[l - 1];
+  GemmArgs a{};
+  a.M = c->cfg.batch; a.N = y.n_in; a.K = y.n_out;
+  a.mode = EPI_DGRAD;
+  a.act = pv.d.act;
+  a.out = pv.delta + size_t(n % kDeltaSlots) * pv.delta_elems;
+  a.ld_out = pv.ld_out;
+  if (pv.d.act == LP_ACT_GELU) {
+    a.aux = pv.Z + size_t(n % pv.z_slots) * pv.z_elems;   // stored z^{l-1}
+    a.ld_aux = pv.ld_out;
+  } else {
+    a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;      // a^{l-1} > 0  <=>  z^{l-1} > 0
+    a.ld_aux = y.ld_in;
+  }
+  a.status = c->status;
+  ++c->launches;
+  return gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
+}
+
+static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
+  Layer& y = c->L[l];
+  GemmArgs a{};
+  a.M = y.n_out; a.N = y.n_in; a.K = c->cfg.batch;
+  a.mode = EPI_STORE_F32;
+  a.out = y.dW;
+  a.ld_out = y.ld_in;
+  a.status = c->status;
+  ++c->launches;
+  return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st);
+}
+
+static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st) {
+  Layer& y = c->L[l];
+  const int dst_slot = int((n + 1) % y.slots);
+  UpdateArgs u{};
+  u.dW = y.dW; u.W = y.W; u.mW = y.mW;
+  u.ring = y.ring + size_t(dst_slot) * y.w_elems;
+  u.n_elems = (long long)y.w_elems;
+  if (y.d.has_bias) {
+    u.delta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
+    u.rows = c->cfg.batch; u.ldd = y.ld_out; u.n_out = y.n_out;
+    u.b = y.b; u.mb = y.mb; u.db = y.db;
+    u.bring = y.bring + size_t(dst_slot) * y.ld_out;
+  }
+  u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
+  ++c->launches;
+  return launch_sgd_update(u, st);
+}
+
+}  // namespace lp
+
+using namespace lp;
+
+// ===========================================================================
+extern "C" int lp_workspace_size(const lp_layer* layers, int n_layers, int n_stages, const int* stage,
+                                 const int* delays, const lp_config* cfg, size_t* bytes_out) {
+  std::string why;
+  if (!bytes_out) return fail(nullptr, LP_ERR_INVALID_ARG, "bytes_out is null");
+  int rc = validate(layers, n_layers, cfg, &why);
+  if (rc != LP_OK) return fail(nullptr, rc, why);
+  std::vector<int> st, dl;
+  int used = 0;
+  rc = resolve_plan(layers, n_layers, n_stages, stage, delays, cfg, &st, &dl, &used, &why);
+  if (rc != LP_OK) return fail(nullptr, rc, why);
+  lp_ctx tmp;
+  tmp.cfg = *cfg;
+  shape_layers(&tmp, layers, n_layers, st, dl);
+  *bytes_out = carve(&tmp, nullptr);
+  return LP_OK;
+}
+
+extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, int n_stages, const int* stage,
+                         const int* delays, const lp_config* cfg, const float* const* W0_host,
+                         const float* const* b0_host, void* workspace_dev, size_t workspace_bytes) {
+  std::string why;
+  if (!out) return fail(nullptr, LP_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  if (!W0_host || !workspace_dev) return fail(nullptr, LP_ERR_INVALID_ARG, "W0_host or workspace is null");
+  int rc = validate(layers, n_layers, cfg, &why);
+  if (rc != LP_OK) return fail(nullptr, rc, why);
+  for (int l = 0; l < n_layers; ++l)
+    if (!W0_host[l]) return fail(nullptr, LP_ERR_INVALID_ARG, "W0_host[l] is null");
+  std::vector<int> st, dl;
+  int used = 0;
+  rc = resolve_plan(layers, n_layers, n_stages, stage, delays, cfg, &st, &dl, &used, &why);
+  if (rc != LP_OK) return fail(nullptr, rc, why);
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
+    return fail(nullptr, LP_ERR_CUDA, "no CUDA device");
+  if (prop.major != 10) return fail(nullptr, LP_ERR_UNSUPPORTED, "this library needs an sm_100 device");
+
+  std::unique_ptr<lp_ctx, void (*)(lp_ctx*)> c(new lp_ctx, destroy_ctx);
+  c->cfg = *cfg;
+  c->n_stages = n_stages;
+  c->stages_used = used;
+  shape_layers(c.get(), layers, n_layers, st, dl);
+  const size_t need = carve(c.get(), nullptr);
+  if ((reinterpret_cast<uintptr_t>(workspace_dev) & 255) != 0 || workspace_bytes < need)
+    return fail(nullptr, LP_ERR_WORKSPACE, "workspace misaligned or smaller than lp_workspace_size");
+  c->ws = static_cast<char*>(workspace_dev);
+  c->ws_bytes = need;
+  carve(c.get(), c->ws);
+
+  lp_ctx* h = c.get();
+  LP_CUDA(nullptr, cudaMemset(c->ws, 0, need));
+  LP_CUDA(nullptr, gemm_configure());
+  // streams: delta highest priority, forward next, G + update lowest
+  int least = 0, greatest = 0;
+  LP_CUDA(nullptr, cudaDeviceGetStreamPriorityRange(&least, &greatest));
+  const int pD = greatest, pF = std::min(least, greatest + 1), pG = least;
+  c->sF.assign(used, nullptr);
+  c->sD.assign(used, nullptr);
+  c->sG.assign(used, nullptr);
+  for (int s = 0; s < used; ++s) {
+    LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sF[s], cudaStreamNonBlocking, pF));
+    LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sD[s], cudaStreamNonBlocking, pD));
+    LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sG[s], cudaStreamNonBlocking, pG));
+  }
+  c->pool.assign(kEventPool, nullptr);
+  for (auto& e : c->pool) LP_CUDA(nullptr, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  c->loss_ev.assign(kLossRing, Ev{});
+  c->rZL.assign(kDeltaSlots, Res{});
+  c->rLabels.assign(kDeltaSlots, Res{});
+  c->log_v.assign(size_t(kLogRing) * n_layers, 0);
+  c->log_slot.assign(size_t(kLogRing) * n_layers, 0);
+
+  // initial weights: fp32 master (padded pitch) and version 0 in ring slot 0
+  for (int l = 0; l < n_layers; ++l) {
+    Layer& y = c->L[l];
+    y.rX.assign(y.x_slots, Res{});
+    y.rZ.assign(std::max(y.z_slots, 1), Res{});
+    y.rDelta.assign(kDeltaSlots, Res{});
+    y.rRing.assign(y.slots, Res{});
+    LP_CUDA(nullptr, cudaMemcpy2D(y.W, size_t(y.ld_in) * 4, W0_host[l], size_t(y.n_in) * 4, size_t(y.n_in) * 4,
+                                  y.n_out, cudaMemcpyHostToDevice));
+    LP_CUDA(nullptr, launch_round_to_bf16(y.W, y.ring, (long long)y.w_elems, 0));
+    if (y.d.has_bias && b0_host && b0_host[l]) {
+      LP_CUDA(nullptr, cudaMemcpy(y.b, b0_host[l], size_t(y.n_out) * 4, cudaMemcpyHostToDevice));
+      LP_CUDA(nullptr, cudaMemcpy(y.bring, b0_host[l], size_t(y.n_out) * 4, cudaMemcpyHostToDevice));
+    }
+  }
+  LP_CUDA(nullptr, cudaDeviceSynchronize());
+  rc = build_tensor_maps(h);
+  if (rc != LP_OK) { g_err = h->err; return rc; }
+  *out = c.release();
+  return LP_OK;
+}
+
+extern "C" int lp_destroy(lp_handle h) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  destroy_ctx(h);
+  return LP_OK;
+}
+
+extern "C" const char* lp_last_error(lp_handle h) { return h ? h->err.c_str() : g_err.c_str(); }
+
+extern "C" int lp_set_tuning(int tile_n, int stages) {
+  if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) || stages < 0 || stages > GEMM_MAX_STAGES)
+    return LP_ERR_INVALID_ARG;
+  gemm_set_tuning(tile_n, stages);
+  return LP_OK;
+}
+
+extern "C" long long lp_kernel_launches(lp_handle h) { return h ? h->launches : 0; }
+
+extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev, void* stream) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (h->latched) return h->latched;
+  if (!batch_dev || !labels_dev) return fail(h, LP_ERR_INVALID_ARG, "batch or labels is null");
+  lp_ctx* c = h;
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  const long long n = c->n_steps;
+  const int nL = int(c->L.size());
+  const int B = c->cfg.batch;
+  const bool fusedB = (c->cfg.schedule == LP_SCHED_FUSED_B);
+  const int ds = int(n % kDeltaSlots);
+
+  // version bookkeeping (the integers the parity tests compare bit-exactly)
+  std::vector<int> slot(nL);
+  for (int l = 0; l < nL; ++l) {
+    const long long v = std::max<long long>(0, n - c->L[l].delay);
+    slot[l] = int(v % c->L[l].slots);
+    c->log_v[size_t(n % kLogRing) * nL + l] = int(v);
+    c->log_slot[size_t(n % kLogRing) * nL + l] = slot[l];
+  }
+
+  // ---- cast + stash on the caller's stream ----------------------------------
+  {
+    Layer& y0 = c->L[0];
+    Res* rx = &y0.rX[n % y0.x_slots];
+    Res* rl = &c->rLabels[ds];
+    LP_CUDA(c, task_begin(c, user, {}, {rx, rl}));
+    ++c->launches;
+    LP_CUDA(c, launch_cast_stash(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
+                                 y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.n_in,
+                                 y0.ld_in, user));
+    LP_CUDA(c, task_end(c, user, {}, {rx, rl}, nullptr));
+  }
+  // ---- forward ---------------------------------------------------------------
+  for (int l = 0; l < nL; ++l) {
+    Layer& y = c->L[l];
+    cudaStream_t st = c->sF[y.stage];
+    Res* rin = &y.rX[n % y.x_slots];
+    Res* rw = &y.rRing[slot[l]];
+    Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[n % c->L[l + 1].x_slots];
+    Res* rz = y.Z ? &y.rZ[n % y.z_slots] : nullptr;
+    LP_CUDA(c, task_begin(c, st, {rin, rw}, {rout, rz}));
+    LP_CUDA(c, launch_forward(c, l, n, slot[l], st));
+    LP_CUDA(c, task_end(c, st, {rin, rw}, {rout, rz}, nullptr));
+  }
+  // ---- loss and delta^L --------------------------------------------------------
+  {
+    Layer& yl = c->L[nL - 1];
+    cudaStream_t st = c->sD[yl.stage];
+    Res* rd = &yl.rDelta[ds];
+    LP_CUDA(c, task_begin(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}));
+    ++c->launches;
+    LP_CUDA(c, launch_softmax_xent(c->zL + size_t(ds) * B * c->ld_cls, c->ld_cls, c->labels + size_t(ds) * B,
+                                   yl.delta + size_t(ds) * yl.delta_elems, yl.ld_out, c->row_loss + size_t(ds) * B,
+                                   c->ticket + ds, c->loss + (n % kLossRing), B, c->classes, st));
+    LP_CUDA(c, task_end(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}, &c->loss_ev[n % kLossRing]));
+  }
+  // ---- backward: delta and G are independent tasks; update follows G -----------
+  for (int l = nL - 1; l >= 0; --l) {
+    Layer& y = c->L[l];
+    Res* rdl = &y.rDelta[ds];
+    Res* rw = &y.rRing[slot[l]];
+    Res* rx = &y.rX[n % y.x_slots];
+    Res* rnew = &y.rRing[(n + 1) % y.slots];
+    Res* rdprev = nullptr;
+    Res* raux = nullptr;
+    if (l > 0) {
+      Layer& pv = c->L[l - 1];
+      rdprev = &pv.rDelta[ds];
+      raux = (pv.d.act == LP_ACT_GELU) ? &pv.rZ[n % pv.z_slots] : rx;
+    }
+    if (fusedB) {
+      cudaStream_t st = c->sD[y.stage];
+      LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux}, {rdprev, &y.rDW, rnew}));
+      if (l > 0) LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+      LP_CUDA(c, launch_G(c, l, n, st));
+      LP_CUDA(c, launch_update(c, l, n, st));
+      LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux}, {rdprev, &y.rDW, rnew}, &y.last_update));
+    } else {
+      if (l > 0) {
+        cudaStream_t st = c->sD[y.stage];
+        LP_CUDA(c, task_begin(c, st, {rdl, rw, raux}, {rdprev}));
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+        LP_CUDA(c, task_end(c, st, {rdl, rw, raux}, {rdprev}, nullptr));
+      }
+      cudaStream_t sg = c->sG[y.stage];
+      LP_CUDA(c, task_begin(c, sg, {rdl, rx}, {&y.rDW}));
+      LP_CUDA(c, launch_G(c, l, n, sg));
+      LP_CUDA(c, task_end(c, sg, {rdl, rx}, {&y.rDW}, nullptr));
+      LP_CUDA(c, task_begin(c, sg, {&y.rDW, rdl}, {rnew}));
+      LP_CUDA(c, launch_update(c, l, n, sg));
+      LP_CUDA(c, task_end(c, sg, {&y.rDW, rdl}, {rnew}, &y.last_update));
+    }
+  }
+  c->n_steps = n + 1;
+  return LP_OK;
+}
+
+extern "C" int lp_flush(lp_handle h, void* stream) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (h->latched) return h->latched;
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  auto join = [&](std::vector<cudaStream_t>& v) -> cudaError_t {
+    for (cudaStream_t s : v) {
+      cudaEvent_t e = h->pool[h->pool_next++ % h->pool.size()];
+      cudaError_t r = cudaEventRecord(e, s);
+      if (r != cudaSuccess) return r;
+      r = cudaStreamWaitEvent(user, e, 0);
+      if (r != cudaSuccess) return r;
+    }
+    return cudaSuccess;
+  };
+  LP_CUDA(h, join(h->sF));
+  LP_CUDA(h, join(h->sD));
+  LP_CUDA(h, join(h->sG));
+  return LP_OK;
+}
+
+extern "C" int lp_get_weights(lp_handle h, int layer, float* W_out, float* b_out, long long* version) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= int(h->L.size())) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
+  Layer& y = h->L[layer];
+  if (y.last_update.e) LP_CUDA(h, cudaEventSynchronize(y.last_update.e));
+  if (W_out)
+    LP_CUDA(h, cudaMemcpy2D(W_out, size_t(y.n_in) * 4, y.W, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
+                            cudaMemcpyDeviceToHost));
+  if (b_out) LP_CUDA(h, cudaMemcpy(b_out, y.b, size_t(y.n_out) * 4, cudaMemcpyDeviceToHost));
+  if (version) *version = h->n_steps;
+  return LP_OK;
+}
+
+extern "C" int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* db_out) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= int(h->L.size())) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
+  if (step != h->n_steps - 1 || step < 0) return fail(h, LP_ERR_NOT_READY, "only the latest step's gradients are held");
+  Layer& y = h->L[layer];
+  if (y.last_update.e) LP_CUDA(h, cudaEventSynchronize(y.last_update.e));
+  if (dW_out)
+    LP_CUDA(h, cudaMemcpy2D(dW_out, size_t(y.n_in) * 4, y.dW, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
+                            cudaMemcpyDeviceToHost));
+  if (db_out) LP_CUDA(h, cudaMemcpy(db_out, y.db, size_t(y.n_out) * 4, cudaMemcpyDeviceToHost));
+  return LP_OK;
+}
+
+extern "C" int lp_get_schedule(lp_handle h, int* stage, int* delay, int* ring_slots) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  for (size_t l = 0; l < h->L.size(); ++l) {
+    if (stage) stage[l] = h->L[l].stage;
+    if (delay) delay[l] = h->L[l].delay;
+    if (ring_slots) ring_slots[l] = h->L[l].slots;
+  }
+  return LP_OK;
+}
+
+extern "C" int lp_get_version_log(lp_handle h, long long step, int* v_fwd, int* v_bwd, int* slot) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (step < 0 || step >= h->n_steps || step < h->n_steps - kLogRing)
+    return fail(h, LP_ERR_NOT_READY, "step outside the version log");
+  const size_t nL = h->L.size();
+  for (size_t l = 0; l < nL; ++l) {
+    const int v = h->log_v[size_t(step % kLogRing) * nL + l];
+    if (v_fwd) v_fwd[l] = v;
+    if (v_bwd) v_bwd[l] = v;      // weight stashing: delta reads the version the forward pass read
+    if (slot) slot[l] = h->log_slot[size_t(step % kLogRing) * nL + l];
+  }
+  return LP_OK;
+}
+
+extern "C" int lp_get_loss(lp_handle h, long long step, float* loss) {
+  if (!h || !loss) return LP_ERR_INVALID_ARG;
+  if (step < 0 || step >= h->n_steps || step < h->n_steps - kLossRing)
+    return fail(h, LP_ERR_NOT_READY, "step outside the loss ring");
+  const Ev& e = h->loss_ev[step % kLossRing];
+  if (e.e) LP_CUDA(h, cudaEventSynchronize(e.e));
+  LP_CUDA(h, cudaMemcpy(loss, h->loss + (step % kLossRing), 4, cudaMemcpyDeviceToHost));
+  return LP_OK;
+}
+
+extern "C" int lp_device_status(lp_handle h, int* detail) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  LP_CUDA(h, cudaDeviceSynchronize());
+  int st = 0;
+  LP_CUDA(h, cudaMemcpy(&st, h->status, 4, cudaMemcpyDeviceToHost));
+  if (detail) *detail = st;
+  if (st != 0) return fail(h, LP_ERR_TIMEOUT, "a bounded device-side wait expired (status " + std::to_string(st) + ")");
+  return LP_OK;
+}
