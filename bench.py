@@ -1,0 +1,437 @@
+#!/usr/bin/env python
+"""Benchmark of the LayerPipe training hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" = one minibatch through the whole path (cast+stash, forward of every layer,
+loss, delta / G / update of every layer under the LayerPipe schedule).  Prints ONE JSON
+line.  The path does not shard (stages are SM partitions of one GPU), so N > 1 runs N
+independent replicas, one process per GPU, and adds their throughput.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2108_06629_b200 import inputs as I  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
+# ncu capture summarised under profiles/ (None until a capture exists for that pair).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ----------------------------------------------------------------------------- work model
+def work_model(layers, batch, momentum):
+    """Algorithmic flops and bytes per launch of each task kind, per layer (true shapes)."""
+    out = {"forward": [], "delta": [], "G": [], "update": []}
+    L = len(layers)
+    for l, y in enumerate(layers):
+        n_in, n_out = y["n_in"], y["n_out"]
+        fl = 2.0 * batch * n_in * n_out
+        gelu = y["act"] == "gelu"
+        last = l == L - 1
+        out["forward"].append(dict(flops=fl, bytes=2.0 * n_in * n_out + 2.0 * batch * n_in +
+                                   (4.0 if last else (4.0 if gelu else 2.0)) * batch * n_out))
+        if l > 0:
+            out["delta"].append(dict(flops=fl, bytes=2.0 * n_in * n_out + 2.0 * batch * n_out + 4.0 * batch * n_in))
+        out["G"].append(dict(flops=fl, bytes=2.0 * batch * (n_in + n_out) + 4.0 * n_in * n_out))
+        per_param = 22.0 if momentum != 0.0 else 14.0   # read G, W (,m); write W (,m) fp32 and the bf16 ring slot
+        out["update"].append(dict(flops=0.0, bytes=per_param * n_in * n_out))
+    return out
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_step_time(orc_factory, layers, batch, rows, n_steps):
+    from oracle import layerpipe_oracle  # noqa: F401  (the oracle is only ever used on this leg)
+    orc = orc_factory()
+    ts = []
+    for n in range(n_steps):
+        x, y = I.minibatch(layers, batch, n)
+        t0 = time.perf_counter()
+        orc.step(x[:rows], y[:rows])
+        ts.append(time.perf_counter() - t0)
+    return ts
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, wl):
+    """The CPU oracle, as it stands, timed on the host cores.  Each step is one oracle
+    minibatch on the first `rows` rows of the synthetic minibatch (full-size layers); rows is
+    chosen so that K + W steps fit a time budget of about three minutes."""
+    from oracle import layerpipe_oracle as O
+    layers, B = wl["layers"], wl["batch"]
+    delays = wl["delays"]
+    if delays is None:
+        from oracle import partition_oracle as P
+        fix, flex = P.mac_costs(layers, B)
+        delays = P.partition(fix, flex, wl["stages"])["delay"]
+    W0, b0 = I.initial_weights(layers, 0)
+
+    def factory():
+        return O.DelayedGradientTrainer(layers, delays, wl["lr"], wl["momentum"], W0, b0, mirror=True,
+                                        dtype=np.float32)
+    total = args.steps + args.warmup
+    budget = 170.0
+    t_small = min(oracle_step_time(factory, layers, B, 8, 2))
+    t_full = min(oracle_step_time(factory, layers, B, B, 1))
+    rows = B
+    while rows > 8:
+        est = t_small + (t_full - t_small) * (rows - 8) / max(B - 8, 1)
+        if est * total <= budget:
+            break
+        rows //= 2
+    rows = max(rows, 8)
+    orc = factory()
+    for n in range(args.warmup):
+        x, y = I.minibatch(layers, B, n)
+        orc.step(x[:rows], y[:rows])
+    t0 = time.perf_counter()
+    for n in range(args.steps):
+        x, y = I.minibatch(layers, B, args.warmup + n)
+        orc.step(x[:rows], y[:rows])
+    dt = time.perf_counter() - t0
+    value = rows * args.steps / dt
+    sample = "first %d of %d rows of each minibatch, full-size layers, %d timed steps" % (rows, B, args.steps)
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": "training samples/sec", "value": value, "unit": "samples/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": B, "delays": delays, "schedule": "sequential CPU oracle"},
+        "cpu_baseline": {"value": value, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- our arm
+def timed_loop(torch, tr, xs, ys, steps, stream):
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    P = len(xs)
+    for k in range(steps):
+        tr.step(xs[k % P], ys[k % P])
+    tr.flush()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def e2e_loop(torch, tr, hx, hy, xd, yd, steps, stream, lag, first_step):
+    """Every step: pinned host -> device copy of that step's minibatch and labels, lp_step,
+    and a device -> host read of one finished step's loss (the step `lag` calls back, so
+    that the read does not drain the pipeline; the last `lag` losses are read at the end)."""
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    P = len(hx)
+    losses = []
+    e0.record(stream)
+    for k in range(steps):
+        xd.copy_(hx[k % P], non_blocking=True)
+        yd.copy_(hy[k % P], non_blocking=True)
+        tr.step(xd, yd)
+        if k >= lag:
+            losses.append(tr.get_loss(first_step + k - lag))
+    for k in range(max(steps - lag, 0), steps):
+        losses.append(tr.get_loss(first_step + k))
+    tr.flush()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    assert len(losses) == steps and all(np.isfinite(losses))
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args, wl):
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lpb.lib()   # fails loudly if the CUDA library is missing
+
+    layers, B = wl["layers"], wl["batch"]
+    W0, b0 = I.initial_weights(layers, 0)
+    sched = lpb.LP_SCHED_FUSED_B if args.schedule == "fused_b" else lpb.LP_SCHED_LAYERPIPE
+    dev = "cuda:%d" % local
+    tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                     schedule=sched, W0=W0, b0=b0, device=dev)
+    stage, delays, slots = tr.get_schedule()
+    P = 8
+    hx, hy = [], []
+    for n in range(P):
+        x, y = I.minibatch(layers, B, n)
+        hx.append(torch.from_numpy(x).pin_memory())
+        hy.append(torch.from_numpy(y).pin_memory())
+    xs = [t.to(dev) for t in hx]
+    ys = [t.to(dev) for t in hy]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # warm-up: fill every ring (max delay + 3 minibatches) plus the requested W
+    prewarm = max(delays) + 3 + max(args.warmup, 3)
+    for k in range(prewarm):
+        tr.step(xs[k % P], ys[k % P])
+    tr.flush()
+    barrier()
+    # ---- device-resident throughput ---------------------------------------------------
+    clocks = ClockSampler(local)
+    time.sleep(0.25)
+    l0 = tr.kernel_launches()
+    ms = timed_loop(torch, tr, xs, ys, args.steps, stream)
+    launches = tr.kernel_launches() - l0
+    barrier()
+    ms = max_over_ranks(ms)
+    # ---- end to end: host buffers, copies inside the timed region --------------------------
+    xd = torch.empty_like(xs[0])
+    yd = torch.empty_like(ys[0])
+    first = prewarm + args.steps
+    lag = max(delays) + 1
+    ms_e2e = e2e_loop(torch, tr, hx, hy, xd, yd, args.steps, stream, lag, first)
+    barrier()
+    ms_e2e = max_over_ranks(ms_e2e)
+    clk = clocks.stop()
+    rc, detail = tr.device_status()
+    if rc != 0:
+        raise SystemExit("device status %d (%d): a bounded wait expired" % (rc, detail))
+    tr.close()
+    del tr
+    torch.cuda.empty_cache()
+
+    # ---- same GPU, same kernels, backward as ONE task per layer (PipeDream-style) -------------
+    other = None
+    if rank == 0:
+        osched = lpb.LP_SCHED_LAYERPIPE if sched == lpb.LP_SCHED_FUSED_B else lpb.LP_SCHED_FUSED_B
+        tro = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                          schedule=osched, W0=W0, b0=b0, device=dev)
+        for k in range(prewarm):
+            tro.step(xs[k % P], ys[k % P])
+        tro.flush()
+        torch.cuda.synchronize()
+        ms_o = timed_loop(torch, tro, xs, ys, args.steps, stream)
+        tro.close()
+        del tro
+        torch.cuda.empty_cache()
+        other = {"schedule": "layerpipe" if osched == lpb.LP_SCHED_LAYERPIPE else "fused_b",
+                 "value": args.steps * B / (ms_o * 1e-3), "unit": "samples/s (1 GPU)", "ms_per_step": ms_o / args.steps}
+
+    line = None
+    if rank == 0:
+        # ---- per-kernel times for the roofline (separate handle with timing events) ----------
+        trp = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                          schedule=sched, flags=lpb.LP_TIME_TASKS, W0=W0, b0=b0, device=dev)
+        for k in range(prewarm):
+            trp.step(xs[k % P], ys[k % P])
+        trp.flush()
+        torch.cuda.synchronize()
+        trp.reset_task_times()
+        nprof = min(args.steps, 32768 // (6 * len(layers)))
+        timed_loop(torch, trp, xs, ys, nprof, stream)
+        kinds = {}
+        for kind in ("forward", "delta", "G", "update", "loss", "cast"):
+            n, tot = trp.task_time(kind)
+            kinds[kind] = dict(launches=n, total_ms=tot, avg_us=1e3 * tot / max(n, 1))
+        trp.close()
+        del trp
+        peaks = load_peaks()
+        wm = work_model(layers, B, wl["momentum"])
+        dom = max(("forward", "delta", "G", "update"), key=lambda k: kinds[k]["total_ms"])
+        per = wm[dom]
+        avg_bytes = sum(p["bytes"] for p in per) / len(per)
+        avg_flops = sum(p["flops"] for p in per) / len(per)
+        avg_s = kinds[dom]["avg_us"] * 1e-6
+        ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        if avg_flops / max(avg_bytes, 1.0) > ridge:
+            roof = {"bound": "tensor", "achieved": avg_flops / avg_s / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s"}
+        else:
+            roof = {"bound": "hbm", "achieved": avg_bytes / avg_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.workload, dom))
+        roof["kernel"] = {"forward": "gemm_tcgen05_kernel<forward>", "delta": "gemm_tcgen05_kernel<delta>",
+                          "G": "gemm_tcgen05_kernel<G>", "update": "sgd_update_kernel"}[dom]
+        roof["peak_source"] = "of " + peaks["_source"]
+        roof["avg_launch_us"] = kinds[dom]["avg_us"]
+        roof["algorithmic_per_launch"] = {"bytes": avg_bytes, "flops": avg_flops}
+        # whole-step figures against both roofs
+        step_flops = sum(p["flops"] for k in ("forward", "delta", "G") for p in wm[k])
+        step_bytes = sum(p["bytes"] for k in wm for p in wm[k])
+        step_s = ms * 1e-3 / args.steps
+        # ---- the oracle on the host cores, bounded sample ---------------------------------------
+        cpu = cpu_baseline(wl)
+        value = world * args.steps * B / (ms * 1e-3)
+        e2e_value = world * args.steps * B / (ms_e2e * 1e-3)
+        in_bytes = xs[0].numel() * xs[0].element_size() + ys[0].numel() * ys[0].element_size()
+        line = {
+            "metric": "training samples/sec", "value": value, "unit": "samples/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": B, "stages_used": max(stage) + 1, "delays": delays,
+                       "ring_slots": slots, "schedule": args.schedule, "parallelism": "replicas only",
+                       "l2": "working set per step exceeds L2 (weights + update streams), no flush",
+                       "prewarm_steps": prewarm},
+            "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": 4,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches),
+            "clocks": clk,
+            "roofline": roof,
+            "step": {"tflops": step_flops / step_s / 1e12, "gbs_algorithmic": step_bytes / step_s / 1e9,
+                     "frac_of_bf16_sustained": step_flops / step_s / 1e12 / peaks["bf16_tflops_sustained"],
+                     "frac_of_hbm": step_bytes / step_s / 1e9 / peaks["hbm_gbs"]},
+            "kernels": kinds,
+            "other_schedule": other,
+            "speedup_vs_fused_b": ((value / world) / other["value"] if other["schedule"] == "fused_b"
+                                   else other["value"] / (value / world)),
+            "cpu_baseline": cpu,
+        }
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+
+
+def cpu_baseline(wl):
+    """The oracle, untouched, on this machine's host cores: whole minibatches until about 10 s of
+    CPU work has been done (at least one)."""
+    from oracle import layerpipe_oracle as O
+    layers, B = wl["layers"], wl["batch"]
+    delays = wl["delays"]
+    if delays is None:
+        from oracle import partition_oracle as P
+        fix, flex = P.mac_costs(layers, B)
+        delays = P.partition(fix, flex, wl["stages"])["delay"]
+    W0, b0 = I.initial_weights(layers, 0)
+    orc = O.DelayedGradientTrainer(layers, delays, wl["lr"], wl["momentum"], W0, b0, mirror=True, dtype=np.float32)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        x, y = I.minibatch(layers, B, n)
+        orc.step(x, y)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= 10.0 or n >= 50:
+            break
+    return {"value": n * B / dt, "unit": "samples/s", "cores": blas_threads(), "kind": "oracle",
+            "sample": "%d whole minibatches of %d, full-size layers, %.1f s" % (n, B, dt)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mlp8_4096", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--schedule", default="layerpipe", choices=["layerpipe", "fused_b"])
+    args = ap.parse_args()
+    wl = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, wl)
+        return
+    run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

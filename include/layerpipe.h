@@ -48,7 +48,8 @@ enum { LP_SCHED_LAYERPIPE = 0, /* delta and G of a layer are separate concurrent
                                /* delta^{l-1} is released as soon as delta finishes        */
        LP_SCHED_FUSED_B = 1 }; /* PipeDream-style: delta, G, update = ONE serial task      */
 enum { LP_F32 = 0, LP_BF16 = 1 };
-enum { LP_CAPTURE_GRADS = 1u }; /* keep G of the latest step readable by lp_get_grads */
+enum { LP_CAPTURE_GRADS = 1u, /* keep G of the latest step readable by lp_get_grads            */
+       LP_TIME_TASKS = 2u };   /* bracket every kernel with timing events (see lp_get_task_time) */
 
 /* One layer of the chain (Eqs. 1-2: z = W a (+ b), a = f(z)). */
 typedef struct {
@@ -141,6 +142,38 @@ int lp_get_weights(lp_handle h, int layer, float* W_out, float* b_out, long long
  * host until that step's G task has finished. */
 int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* db_out);
 
+/*
+ * Verification access.  These three calls exist so that every task of the step can be
+ * checked in isolation against a reference fed with the SAME operands: write operands
+ * into the handle's buffers, run one task, read its outputs.  All three block the host
+ * until the device is idle and must not be mixed with steps still in flight.
+ * Host data is fp32; bf16 buffers are converted (round-to-nearest-even on write).
+ *
+ *   buffer            shape of host array          `index` selects
+ *   LP_BUF_INPUT      [batch][in]   a^{l-1}, stashed input of layer l    minibatch (slot = index mod slots)
+ *   LP_BUF_Z          [batch][out]  stored z^l (GELU layers only)        minibatch
+ *   LP_BUF_DELTA      [batch][out]  delta^l = dE/dz^l                    minibatch
+ *   LP_BUF_LOGITS     [batch][classes] z^L (layer ignored)               minibatch
+ *   LP_BUF_LABELS     [batch] labels as floats (layer ignored)           minibatch
+ *   LP_BUF_LOSS       [1] (layer ignored)                                minibatch
+ *   LP_BUF_RING_W     [out][in]  bf16 weight version                     ring slot
+ *   LP_BUF_RING_B     [out]      fp32 bias version                       ring slot
+ *   LP_BUF_MASTER_W/B, LP_BUF_MOM_W/B, LP_BUF_GRAD_W/B   [out][in] / [out]   (index ignored)
+ */
+enum { LP_BUF_INPUT = 0, LP_BUF_Z = 1, LP_BUF_DELTA = 2, LP_BUF_LOGITS = 3, LP_BUF_LABELS = 4, LP_BUF_LOSS = 5,
+       LP_BUF_RING_W = 6, LP_BUF_RING_B = 7, LP_BUF_MASTER_W = 8, LP_BUF_MASTER_B = 9, LP_BUF_MOM_W = 10,
+       LP_BUF_MOM_B = 11, LP_BUF_GRAD_W = 12, LP_BUF_GRAD_B = 13 };
+int lp_debug_read(lp_handle h, int buffer, int layer, long long index, float* out_host);
+int lp_debug_write(lp_handle h, int buffer, int layer, long long index, const float* in_host);
+
+/* Run ONE task of minibatch `step` on the buffers as they stand (slots and weight version
+ * chosen exactly as lp_step would for that minibatch) and wait for it.  Does not advance
+ * the step counter.  LP_TASK_FORWARD: Eqs. 1-2; LP_TASK_LOSS: loss and delta^L;
+ * LP_TASK_DELTA: Eqs. 3-4 for layer >= 1 (writes delta^{layer-1}); LP_TASK_G: Eq. 5;
+ * LP_TASK_UPDATE: Eq. 6 (writes ring slot (step+1) mod slots). */
+enum { LP_TASK_FORWARD = 0, LP_TASK_LOSS = 1, LP_TASK_DELTA = 2, LP_TASK_G = 3, LP_TASK_UPDATE = 4 };
+int lp_debug_run_task(lp_handle h, int task, int layer, long long step);
+
 /* Plan actually in use: host arrays [n_layers] (any may be NULL). ring_slots = d_l + 1. */
 int lp_get_schedule(lp_handle h, int* stage, int* delay, int* ring_slots);
 
@@ -156,6 +189,14 @@ int lp_get_loss(lp_handle h, long long step, float* loss);
 /* 0, or the first non-zero status word written by a kernel whose bounded wait expired
  * (then returns LP_ERR_TIMEOUT and fills *detail). Blocks until the device is idle. */
 int lp_device_status(lp_handle h, int* detail);
+
+/* Needs LP_TIME_TASKS.  For task kind LP_TASK_* (plus LP_TASK_CAST = 5): number of kernel
+ * launches timed since the last lp_reset_task_times and the sum of their durations in
+ * milliseconds, each measured with CUDA events on the stream the kernel ran on.  Blocks
+ * until the device is idle.  At most 32768 launches are timed between resets. */
+enum { LP_TASK_CAST = 5 };
+int lp_get_task_time(lp_handle h, int task, long long* launches, double* total_ms);
+int lp_reset_task_times(lp_handle h);
 
 /* Number of kernels this handle has launched so far. */
 long long lp_kernel_launches(lp_handle h);

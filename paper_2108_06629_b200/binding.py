@@ -21,6 +21,7 @@ LP_ACT = {"none": 0, "relu": 1, "gelu": 2}
 LP_SCHED_LAYERPIPE, LP_SCHED_FUSED_B = 0, 1
 LP_F32, LP_BF16 = 0, 1
 LP_CAPTURE_GRADS = 1
+LP_TIME_TASKS = 2
 
 
 class lp_layer(C.Structure):
@@ -64,9 +65,14 @@ def lib():
         "lp_get_weights": [vp, C.c_int, fp, fp, llp],
         "lp_get_grads": [vp, C.c_int, C.c_longlong, fp, fp],
         "lp_get_schedule": [vp, ip, ip, ip],
+        "lp_debug_read": [vp, C.c_int, C.c_int, C.c_longlong, fp],
+        "lp_debug_write": [vp, C.c_int, C.c_int, C.c_longlong, fp],
+        "lp_debug_run_task": [vp, C.c_int, C.c_int, C.c_longlong],
         "lp_get_version_log": [vp, C.c_longlong, ip, ip, ip],
         "lp_get_loss": [vp, C.c_longlong, fp],
         "lp_device_status": [vp, ip],
+        "lp_get_task_time": [vp, C.c_int, llp, _P(C.c_double)],
+        "lp_reset_task_times": [vp],
         "lp_set_tuning": [C.c_int, C.c_int],
         "lp_destroy": [vp],
         "lp_gemm_bf16": [C.c_int, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, vp],
@@ -84,8 +90,8 @@ def lib():
 
 
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
-           "lp_get_weights", "lp_get_grads", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
-           "lp_device_status", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
+           "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
+           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
            "lp_gemm_bf16"]
 
 
@@ -221,6 +227,31 @@ class Trainer:
                                   db.ctypes.data_as(_P(C.c_float))), self.h)
         return dW, db
 
+    # ---- verification access (see the header: lp_debug_*) -------------------
+    BUF = {"input": 0, "z": 1, "delta": 2, "logits": 3, "labels": 4, "loss": 5, "ring_w": 6, "ring_b": 7,
+           "master_w": 8, "master_b": 9, "mom_w": 10, "mom_b": 11, "grad_w": 12, "grad_b": 13}
+    TASK = {"forward": 0, "loss": 1, "delta": 2, "G": 3, "update": 4}
+
+    def _buf_shape(self, buf, layer):
+        l = self.layers[layer]
+        classes = self.layers[-1]["n_out"]
+        return {"input": (self.batch, l["n_in"]), "z": (self.batch, l["n_out"]), "delta": (self.batch, l["n_out"]),
+                "logits": (self.batch, classes), "labels": (self.batch,), "loss": (1,),
+                "ring_w": (l["n_out"], l["n_in"]), "master_w": (l["n_out"], l["n_in"]),
+                "mom_w": (l["n_out"], l["n_in"]), "grad_w": (l["n_out"], l["n_in"])}.get(buf, (l["n_out"],))
+
+    def debug_read(self, buf, layer, index):
+        out = np.empty(self._buf_shape(buf, layer), dtype=np.float32)
+        _check(lib().lp_debug_read(self.h, self.BUF[buf], layer, index, out.ctypes.data_as(_P(C.c_float))), self.h)
+        return out
+
+    def debug_write(self, buf, layer, index, value):
+        v = np.ascontiguousarray(np.asarray(value, dtype=np.float32).reshape(self._buf_shape(buf, layer)))
+        _check(lib().lp_debug_write(self.h, self.BUF[buf], layer, index, v.ctypes.data_as(_P(C.c_float))), self.h)
+
+    def debug_run_task(self, task, layer, step):
+        _check(lib().lp_debug_run_task(self.h, self.TASK[task], layer, step), self.h)
+
     def get_schedule(self):
         n = len(self.layers)
         a, b, c = (C.c_int * n)(), (C.c_int * n)(), (C.c_int * n)()
@@ -242,6 +273,16 @@ class Trainer:
         d = C.c_int()
         rc = lib().lp_device_status(self.h, C.byref(d))
         return rc, d.value
+
+    def task_time(self, task):
+        """(launches, total milliseconds) of one task kind; needs flags=LP_TIME_TASKS."""
+        k = dict(self.TASK, cast=5)[task]
+        n, ms = C.c_longlong(), C.c_double()
+        _check(lib().lp_get_task_time(self.h, k, C.byref(n), C.byref(ms)), self.h)
+        return n.value, ms.value
+
+    def reset_task_times(self):
+        _check(lib().lp_reset_task_times(self.h), self.h)
 
     def kernel_launches(self):
         return lib().lp_kernel_launches(self.h)

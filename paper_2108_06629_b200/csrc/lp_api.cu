@@ -84,6 +84,9 @@ struct lp_ctx {
   long long n_steps = 0;
   long long launches = 0;
   std::vector<int> log_v, log_slot;   // [kLogRing][L]
+  std::vector<cudaEvent_t> tpool;              // timing events (LP_TIME_TASKS)
+  size_t tpool_next = 0;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed[6];
   std::string err;
   int latched = 0;
   char* ws = nullptr;
@@ -320,8 +323,28 @@ static void destroy_ctx(lp_ctx* c) {
   kill(c->sD);
   kill(c->sG);
   for (cudaEvent_t e : c->pool) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->tpool) if (e) cudaEventDestroy(e);
   delete c;
 }
+
+// Optional per-kernel timing: a start/stop event pair on the kernel's own stream.
+struct TimedScope {
+  lp_ctx* c;
+  cudaStream_t st;
+  int kind;
+  cudaEvent_t e1 = nullptr;
+  TimedScope(lp_ctx* c_, int kind_, cudaStream_t st_) : c(c_), st(st_), kind(kind_) {
+    if ((c->cfg.flags & LP_TIME_TASKS) && c->tpool_next + 2 <= c->tpool.size()) {
+      cudaEvent_t e0 = c->tpool[c->tpool_next++];
+      e1 = c->tpool[c->tpool_next++];
+      cudaEventRecord(e0, st);
+      c->timed[kind].push_back({e0, e1});
+    }
+  }
+  ~TimedScope() {
+    if (e1) cudaEventRecord(e1, st);
+  }
+};
 
 // ---------------------------------------------------------------------------
 // the kernels of one minibatch
@@ -350,6 +373,7 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
     }
   }
   ++c->launches;
+  TimedScope ts(c, LP_TASK_FORWARD, st);
   return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
 }
 
@@ -371,6 +395,7 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
   }
   a.status = c->status;
   ++c->launches;
+  TimedScope ts(c, LP_TASK_DELTA, st);
   return gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
 }
 
@@ -383,6 +408,7 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   a.ld_out = y.ld_in;
   a.status = c->status;
   ++c->launches;
+  TimedScope ts(c, LP_TASK_G, st);
   return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st);
 }
 
@@ -401,6 +427,7 @@ static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st)
   }
   u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
   ++c->launches;
+  TimedScope ts(c, LP_TASK_UPDATE, st);
   return launch_sgd_update(u, st);
 }
 
@@ -477,6 +504,10 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   }
   c->pool.assign(kEventPool, nullptr);
   for (auto& e : c->pool) LP_CUDA(nullptr, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  if (cfg->flags & LP_TIME_TASKS) {
+    c->tpool.assign(2 * 32768, nullptr);
+    for (auto& e : c->tpool) LP_CUDA(nullptr, cudaEventCreate(&e));
+  }
   c->loss_ev.assign(kLossRing, Ev{});
   c->rZL.assign(kDeltaSlots, Res{});
   c->rLabels.assign(kDeltaSlots, Res{});
@@ -520,6 +551,29 @@ extern "C" int lp_set_tuning(int tile_n, int stages) {
   return LP_OK;
 }
 
+extern "C" int lp_get_task_time(lp_handle h, int task, long long* launches, double* total_ms) {
+  if (!h || task < 0 || task > LP_TASK_CAST) return LP_ERR_INVALID_ARG;
+  if (!(h->cfg.flags & LP_TIME_TASKS)) return fail(h, LP_ERR_NOT_READY, "handle was created without LP_TIME_TASKS");
+  LP_CUDA(h, cudaDeviceSynchronize());
+  double tot = 0.0;
+  for (auto& pr : h->timed[task]) {
+    float ms = 0.f;
+    LP_CUDA(h, cudaEventElapsedTime(&ms, pr.first, pr.second));
+    tot += ms;
+  }
+  if (launches) *launches = (long long)h->timed[task].size();
+  if (total_ms) *total_ms = tot;
+  return LP_OK;
+}
+
+extern "C" int lp_reset_task_times(lp_handle h) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  LP_CUDA(h, cudaDeviceSynchronize());
+  for (auto& v : h->timed) v.clear();
+  h->tpool_next = 0;
+  return LP_OK;
+}
+
 extern "C" long long lp_kernel_launches(lp_handle h) { return h ? h->launches : 0; }
 
 extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev, void* stream) {
@@ -550,6 +604,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     Res* rl = &c->rLabels[ds];
     LP_CUDA(c, task_begin(c, user, {}, {rx, rl}));
     ++c->launches;
+    TimedScope ts(c, LP_TASK_CAST, user);
     LP_CUDA(c, launch_cast_stash(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
                                  y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.n_in,
                                  y0.ld_in, user));
@@ -574,6 +629,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     Res* rd = &yl.rDelta[ds];
     LP_CUDA(c, task_begin(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}));
     ++c->launches;
+    TimedScope ts(c, LP_TASK_LOSS, st);
     LP_CUDA(c, launch_softmax_xent(c->zL + size_t(ds) * B * c->ld_cls, c->ld_cls, c->labels + size_t(ds) * B,
                                    yl.delta + size_t(ds) * yl.delta_elems, yl.ld_out, c->row_loss + size_t(ds) * B,
                                    c->ticket + ds, c->loss + (n % kLossRing), B, c->classes, st));
@@ -663,6 +719,151 @@ extern "C" int lp_get_grads(lp_handle h, int layer, long long step, float* dW_ou
     LP_CUDA(h, cudaMemcpy2D(dW_out, size_t(y.n_in) * 4, y.dW, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
                             cudaMemcpyDeviceToHost));
   if (db_out) LP_CUDA(h, cudaMemcpy(db_out, y.db, size_t(y.n_out) * 4, cudaMemcpyDeviceToHost));
+  return LP_OK;
+}
+
+namespace lp {
+struct BufView {
+  void* ptr = nullptr;
+  int rows = 0, cols = 0, ld = 0;
+  int dtype = 0;   // 0 bf16, 1 f32, 2 i32
+};
+static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v) {
+  const int nL = int(h->L.size());
+  const int B = h->cfg.batch;
+  if (index < 0) return fail(h, LP_ERR_INVALID_ARG, "negative index");
+  if (buffer == LP_BUF_LOGITS) {
+    *v = {h->zL + size_t(index % kDeltaSlots) * B * h->ld_cls, B, h->classes, h->ld_cls, 1};
+    return LP_OK;
+  }
+  if (buffer == LP_BUF_LABELS) { *v = {h->labels + size_t(index % kDeltaSlots) * B, 1, B, B, 2}; return LP_OK; }
+  if (buffer == LP_BUF_LOSS) { *v = {h->loss + (index % kLossRing), 1, 1, 1, 1}; return LP_OK; }
+  if (layer < 0 || layer >= nL) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
+  Layer& y = h->L[layer];
+  switch (buffer) {
+    case LP_BUF_INPUT: *v = {y.X + size_t(index % y.x_slots) * y.x_elems, B, y.n_in, y.ld_in, 0}; return LP_OK;
+    case LP_BUF_Z:
+      if (!y.Z) return fail(h, LP_ERR_NOT_READY, "this layer stores no pre-activation");
+      *v = {y.Z + size_t(index % y.z_slots) * y.z_elems, B, y.n_out, y.ld_out, 0};
+      return LP_OK;
+    case LP_BUF_DELTA: *v = {y.delta + size_t(index % kDeltaSlots) * y.delta_elems, B, y.n_out, y.ld_out, 0}; return LP_OK;
+    case LP_BUF_RING_W:
+      if (index >= y.slots) return fail(h, LP_ERR_INVALID_ARG, "ring slot out of range");
+      *v = {y.ring + size_t(index) * y.w_elems, y.n_out, y.n_in, y.ld_in, 0};
+      return LP_OK;
+    case LP_BUF_RING_B:
+      if (index >= y.slots) return fail(h, LP_ERR_INVALID_ARG, "ring slot out of range");
+      *v = {y.bring + size_t(index) * y.ld_out, 1, y.n_out, y.ld_out, 1};
+      return LP_OK;
+    case LP_BUF_MASTER_W: *v = {y.W, y.n_out, y.n_in, y.ld_in, 1}; return LP_OK;
+    case LP_BUF_MASTER_B: *v = {y.b, 1, y.n_out, y.ld_out, 1}; return LP_OK;
+    case LP_BUF_MOM_W:
+      if (!y.mW) return fail(h, LP_ERR_NOT_READY, "momentum is off");
+      *v = {y.mW, y.n_out, y.n_in, y.ld_in, 1};
+      return LP_OK;
+    case LP_BUF_MOM_B:
+      if (!y.mb) return fail(h, LP_ERR_NOT_READY, "momentum is off");
+      *v = {y.mb, 1, y.n_out, y.ld_out, 1};
+      return LP_OK;
+    case LP_BUF_GRAD_W: *v = {y.dW, y.n_out, y.n_in, y.ld_in, 1}; return LP_OK;
+    case LP_BUF_GRAD_B: *v = {y.db, 1, y.n_out, y.ld_out, 1}; return LP_OK;
+  }
+  return fail(h, LP_ERR_INVALID_ARG, "unknown buffer");
+}
+static inline uint16_t f32_to_bf16_rn(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return uint16_t((u >> 16) | 0x40);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return uint16_t(u >> 16);
+}
+}  // namespace lp
+
+extern "C" int lp_debug_read(lp_handle h, int buffer, int layer, long long index, float* out_host) {
+  if (!h || !out_host) return LP_ERR_INVALID_ARG;
+  BufView v;
+  int rc = locate(h, buffer, layer, index, &v);
+  if (rc != LP_OK) return rc;
+  LP_CUDA(h, cudaDeviceSynchronize());
+  if (v.dtype == 1) {
+    LP_CUDA(h, cudaMemcpy2D(out_host, size_t(v.cols) * 4, v.ptr, size_t(v.ld) * 4, size_t(v.cols) * 4, v.rows,
+                            cudaMemcpyDeviceToHost));
+    return LP_OK;
+  }
+  if (v.dtype == 2) {
+    std::vector<int> tmp(v.cols);
+    LP_CUDA(h, cudaMemcpy(tmp.data(), v.ptr, size_t(v.cols) * 4, cudaMemcpyDeviceToHost));
+    for (int c = 0; c < v.cols; ++c) out_host[c] = float(tmp[c]);
+    return LP_OK;
+  }
+  std::vector<uint16_t> tmp(size_t(v.rows) * v.ld);
+  LP_CUDA(h, cudaMemcpy(tmp.data(), v.ptr, tmp.size() * 2, cudaMemcpyDeviceToHost));
+  for (int r = 0; r < v.rows; ++r)
+    for (int c = 0; c < v.cols; ++c) {
+      const uint32_t bits = uint32_t(tmp[size_t(r) * v.ld + c]) << 16;
+      memcpy(&out_host[size_t(r) * v.cols + c], &bits, 4);
+    }
+  return LP_OK;
+}
+
+extern "C" int lp_debug_write(lp_handle h, int buffer, int layer, long long index, const float* in_host) {
+  if (!h || !in_host) return LP_ERR_INVALID_ARG;
+  BufView v;
+  int rc = locate(h, buffer, layer, index, &v);
+  if (rc != LP_OK) return rc;
+  LP_CUDA(h, cudaDeviceSynchronize());
+  if (v.dtype == 1) {
+    LP_CUDA(h, cudaMemcpy2D(v.ptr, size_t(v.ld) * 4, in_host, size_t(v.cols) * 4, size_t(v.cols) * 4, v.rows,
+                            cudaMemcpyHostToDevice));
+    return LP_OK;
+  }
+  if (v.dtype == 2) {
+    std::vector<int> tmp(v.cols);
+    for (int c = 0; c < v.cols; ++c) tmp[c] = int(in_host[c]);
+    LP_CUDA(h, cudaMemcpy(v.ptr, tmp.data(), size_t(v.cols) * 4, cudaMemcpyHostToDevice));
+    return LP_OK;
+  }
+  std::vector<uint16_t> tmp(size_t(v.rows) * v.ld, 0);
+  for (int r = 0; r < v.rows; ++r)
+    for (int c = 0; c < v.cols; ++c) tmp[size_t(r) * v.ld + c] = f32_to_bf16_rn(in_host[size_t(r) * v.cols + c]);
+  LP_CUDA(h, cudaMemcpy(v.ptr, tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice));
+  return LP_OK;
+}
+
+extern "C" int lp_debug_run_task(lp_handle h, int task, int layer, long long step) {
+  if (!h) return LP_ERR_INVALID_ARG;
+  if (h->latched) return h->latched;
+  const int nL = int(h->L.size());
+  if (step < 0) return fail(h, LP_ERR_INVALID_ARG, "negative step");
+  if (task != LP_TASK_LOSS && (layer < 0 || layer >= nL)) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
+  LP_CUDA(h, cudaDeviceSynchronize());
+  cudaStream_t st = h->sF[0];
+  const int B = h->cfg.batch;
+  const int ds = int(step % kDeltaSlots);
+  int slot = 0;
+  if (task != LP_TASK_LOSS) {
+    Layer& y = h->L[layer];
+    slot = int(std::max<long long>(0, step - y.delay) % y.slots);
+  }
+  switch (task) {
+    case LP_TASK_FORWARD: LP_CUDA(h, launch_forward(h, layer, step, slot, st)); break;
+    case LP_TASK_LOSS: {
+      Layer& yl = h->L[nL - 1];
+      ++h->launches;
+      LP_CUDA(h, launch_softmax_xent(h->zL + size_t(ds) * B * h->ld_cls, h->ld_cls, h->labels + size_t(ds) * B,
+                                     yl.delta + size_t(ds) * yl.delta_elems, yl.ld_out, h->row_loss + size_t(ds) * B,
+                                     h->ticket + ds, h->loss + (step % kLossRing), B, h->classes, st));
+      break;
+    }
+    case LP_TASK_DELTA:
+      if (layer < 1) return fail(h, LP_ERR_INVALID_ARG, "the first layer has no delta task");
+      LP_CUDA(h, launch_delta(h, layer, step, slot, st));
+      break;
+    case LP_TASK_G: LP_CUDA(h, launch_G(h, layer, step, st)); break;
+    case LP_TASK_UPDATE: LP_CUDA(h, launch_update(h, layer, step, st)); break;
+    default: return fail(h, LP_ERR_INVALID_ARG, "unknown task");
+  }
+  LP_CUDA(h, cudaStreamSynchronize(st));
   return LP_OK;
 }
 

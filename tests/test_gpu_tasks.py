@@ -1,0 +1,143 @@
+"""Per-task parity with the SAME operands on both sides.
+
+The oracle walks the delayed-gradient recursion on seeded inputs and records every
+operand and result of every task.  For each task the operands it recorded are written
+into the library's buffers (lp_debug_write), the one CUDA task is run
+(lp_debug_run_task) and its outputs are read back and compared.  Nothing the oracle
+consumes comes from the GPU.  With identical operands the only freedom left is the
+summation order inside a contraction, so bf16 results may differ by one bf16 spacing on
+the rare elements that sat next to a rounding boundary and fp32 results by fp32
+round-off; the stated tolerance (relative L2 <= 2e-3 per tensor) holds with a wide
+margin and much sharper bounds are asserted."""
+import numpy as np
+import pytest
+
+from gpu_common import assert_bf16_close, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None):
+    from oracle import layerpipe_oracle as O
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    W0, b0 = I.initial_weights(layers, 0)
+    rng = np.random.default_rng(5)
+    b0 = [rng.standard_normal(b.shape).astype(np.float32) * 0.1 for b in b0]   # exercise the bias path
+    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, W0=W0, b0=b0)
+    delays = tr.get_schedule()[1]
+    orc = O.DelayedGradientTrainer(layers, delays, lr, mu, W0, b0, mirror=True, dtype=np.float32)
+    L = len(layers)
+    worst = {}
+
+    def note(k, v):
+        worst[k] = max(worst.get(k, 0.0), v)
+
+    for n in range(steps):
+        x, y = I.minibatch(layers, batch, n)
+        pre_W = [w.copy() for w in orc.W]
+        pre_b = [b.copy() for b in orc.b]
+        pre_mW = [m.copy() for m in orc.mW]
+        pre_mb = [m.copy() for m in orc.mb]
+        stash = [dict(s) for s in orc.stash]
+        rec = orc.step(x, y, capture=True)
+        if check_steps is not None and n not in check_steps:
+            continue
+        slot = rec["slot"]
+        # weight versions this minibatch reads
+        for l in range(L):
+            Wv, bv = stash[l][rec["v"][l]]
+            tr.debug_write("ring_w", l, slot[l], Wv)
+            tr.debug_write("ring_b", l, slot[l], bv)
+        tr.debug_write("labels", 0, n, y.astype(np.float32))
+        # forward tasks
+        for l in range(L):
+            tr.debug_write("input", l, n, rec["a"][l])
+            tr.debug_run_task("forward", l, n)
+            if l < L - 1:
+                note("a", assert_bf16_close(tr.debug_read("input", l + 1, n), rec["a"][l + 1], "a^%d step %d" % (l + 1, n)))
+                if layers[l]["act"] == "gelu":
+                    note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n)))
+            else:
+                r = rel_l2(tr.debug_read("logits", 0, n), rec["zL"])
+                assert r < 1e-5, ("logits", n, r)
+                note("logits", r)
+        # loss task
+        tr.debug_write("logits", 0, n, rec["zL"])
+        tr.debug_run_task("loss", 0, n)
+        note("deltaL", assert_bf16_close(tr.debug_read("delta", L - 1, n), rec["delta"][L - 1], "delta^L step %d" % n))
+        loss = float(tr.debug_read("loss", 0, n)[0])
+        assert abs(loss - rec["loss"]) <= 2e-6 * max(1.0, abs(rec["loss"])), (loss, rec["loss"])
+        # backward tasks
+        for l in range(L - 1, -1, -1):
+            tr.debug_write("delta", l, n, rec["delta"][l])
+            tr.debug_write("input", l, n, rec["a"][l])
+            if l > 0:
+                if layers[l - 1]["act"] == "gelu":
+                    tr.debug_write("z", l - 1, n, rec["zs"][l - 1])
+                tr.debug_run_task("delta", l, n)
+                note("delta", assert_bf16_close(tr.debug_read("delta", l - 1, n), rec["delta"][l - 1],
+                                                "delta^%d step %d" % (l - 1, n)))
+            tr.debug_run_task("G", l, n)
+            r = rel_l2(tr.debug_read("grad_w", l, 0), rec["dW"][l])
+            assert r < 2e-5, ("G", l, n, r)
+            note("G", r)
+            # update task from the oracle's pre-update state and the oracle's gradient
+            tr.debug_write("master_w", l, 0, pre_W[l])
+            tr.debug_write("master_b", l, 0, pre_b[l])
+            if mu != 0.0:
+                tr.debug_write("mom_w", l, 0, pre_mW[l])
+                tr.debug_write("mom_b", l, 0, pre_mb[l])
+            tr.debug_write("grad_w", l, 0, rec["dW"][l])
+            tr.debug_run_task("update", l, n)
+            r = rel_l2(tr.debug_read("grad_b", l, 0), rec["db"][l])
+            assert r < 2e-5, ("db", l, n, r)
+            note("db", r)
+            dWn = np.linalg.norm(rec["dW"][l])
+            step_err = np.linalg.norm(tr.debug_read("master_w", l, 0) - orc.W[l]) / max(lr * dWn, 1e-30)
+            assert step_err < 1e-3, ("update of W relative to the step taken", l, n, step_err)
+            assert rel_l2(tr.debug_read("master_b", l, 0), orc.b[l]) < 1e-5
+            if mu != 0.0:
+                assert rel_l2(tr.debug_read("mom_w", l, 0), orc.mW[l]) < 1e-6
+            new_slot = (n + 1) % (delays[l] + 1)
+            Wq, bq = orc.stash[l][n + 1]
+            note("ring", assert_bf16_close(tr.debug_read("ring_w", l, new_slot), Wq, "ring W^%d step %d" % (l, n),
+                                           min_equal=0.995))
+            assert rel_l2(tr.debug_read("ring_b", l, new_slot), bq) < 1e-5
+    rc, detail = tr.device_status()
+    assert rc == 0, detail
+    tr.close()
+    return worst
+
+
+def test_tasks_mlp4_784_full_config():
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp4_784"]
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], wl["steps"])
+    print("worst per-task errors", w)
+
+
+def test_tasks_gelu_momentum_ragged_sizes():
+    """GELU + momentum, feature sizes that are not multiples of the 128 x 128 tile nor of 8
+    (padded pitches), batch 72 (ragged M)."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([200, 328, 130, 257, 75], "gelu")
+    w = run_teacher_forced(layers, 72, 4, [3, 2, 1, 0], 0.05, 0.9, 6)
+    print("worst per-task errors", w)
+
+
+def test_tasks_papers_double_delay_convention():
+    """Delays = 2 x (stages after the layer), the count Section III-A gives for the retimed graph."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([96, 160, 64, 24], "relu")
+    run_teacher_forced(layers, 40, 3, [4, 2, 0], 0.05, 0.0, 7)
+
+
+def test_tasks_mlp8_4096_full_size():
+    """The benchmark configuration at full size; three minibatches (first, one inside the
+    warm-up, one after every ring has wrapped) are checked task by task."""
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp8_4096"]
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 10,
+                           check_steps={0, 4, 9})
+    print("worst per-task errors", w)
