@@ -139,8 +139,8 @@ def test_step_rejects_bad_arguments_without_side_effects():
     with pytest.raises(lpb.LayerPipeError) as e:
         tr.get_grads(0, 0)
     assert e.value.code == lpb.LP_ERR_NOT_READY
-    with pytest.raises(lpb.LayerPipeError):
-        tr.get_weights(5)
+    assert lib.lp_get_weights(tr.h, 5, None, None, None) == lpb.LP_ERR_INVALID_ARG
+    assert lib.lp_get_weights(tr.h, -1, None, None, None) == lpb.LP_ERR_INVALID_ARG
     x, y = I.minibatch(layers, 8, 0)
     tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
     assert tr.get_version_log(0)[0] == [0, 0]
