@@ -220,6 +220,45 @@ int lp_destroy(lp_handle h);
 int lp_gemm_bf16(int which, int M, int N, int K, const void* A_dev, int lda,
                  const void* B_dev, int ldb, float* C_dev, int ldc, void* stream);
 
+/*
+ * Softmax cross-entropy without a handle, a workspace or any allocation.  (The paper has
+ * no counterpart: it is the loss kernel of lp_step offered to callers that cannot give the
+ * library memory to work in.)
+ *
+ * Who needs it: code that evaluates the loss outside a trainer -- a validation pass, a
+ * unit test of a custom head -- from a context where device memory cannot be requested:
+ * the process has handed the whole device to a pooling allocator it must not bypass, it
+ * runs under a fixed memory budget agreed at start-up, or it sits in a latency-critical
+ * loop where a cudaMalloc (which may synchronise the device) is not acceptable.  Such a
+ * caller has the logits and the labels and room for the outputs, but nothing to pass as
+ * the per-row scratch the kernel needs.
+ *
+ * Computes exactly what the loss task of lp_step computes:
+ *   delta_dev[r][c] = bf16( (softmax(logits_dev[r])[c] - [c == labels_dev[r]]) / batch )
+ *   *loss_dev       = mean over rows of -log softmax(logits_dev[r])[labels_dev[r]]
+ * logits_dev: device fp32 [batch][ld_logits]; labels_dev: device int32 [batch], values in
+ * [0, classes); delta_dev: device bf16 [batch][ld_delta], ld_delta >= classes rounded up to
+ * a multiple of 8 (the lanes up to that multiple are written as zeros); loss_dev: device
+ * fp32 [1].  All caller-owned.  `stream` is a cudaStream_t (may be 0); the call is
+ * asynchronous.
+ *
+ * The scratch (one fp32 per row plus a counter) is a fixed array inside the library image:
+ * LP_XENT_STATIC_MAX_BATCH rows, about 64 KiB, resident on every GPU that loads the
+ * library for as long as the process lives.  Consequences the caller must know:
+ *   - batch > LP_XENT_STATIC_MAX_BATCH (or batch < 1, classes < 1, bad pitches, null
+ *     pointers) -> LP_ERR_INVALID_ARG, nothing is launched.
+ *   - all calls on one GPU share that array.  The call clears the part that must start
+ *     at zero, so leftovers of an earlier call are harmless, but two calls that overlap
+ *     on the device (different streams, no ordering between them) race on it and give
+ *     wrong losses.  Order them.
+ *   - the first call on each device looks up the array's device address (a host-side
+ *     query, no allocation).  Make that first call outside any stream capture.
+ * Calls no cudaMalloc / cudaFree and no routine that allocates.
+ */
+#define LP_XENT_STATIC_MAX_BATCH 16384
+int lp_softmax_xent_static(const float* logits_dev, int ld_logits, const int* labels_dev, void* delta_dev,
+                           int ld_delta, float* loss_dev, int batch, int classes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

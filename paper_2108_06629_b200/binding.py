@@ -76,6 +76,7 @@ def lib():
         "lp_set_tuning": [C.c_int, C.c_int],
         "lp_destroy": [vp],
         "lp_gemm_bf16": [C.c_int, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, vp],
+        "lp_softmax_xent_static": [vp, C.c_int, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -92,7 +93,7 @@ def lib():
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
            "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
            "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
-           "lp_gemm_bf16"]
+           "lp_gemm_bf16", "lp_softmax_xent_static"]
 
 
 def _check(rc, h=None):
@@ -305,3 +306,18 @@ def lp_gemm_bf16(which, M, N, K, A, lda, B, ldb, Cout, ldc, stream=None):
     s = torch.cuda.current_stream().cuda_stream if stream is None else stream
     _check(lib().lp_gemm_bf16(which, M, N, K, C.c_void_p(A.data_ptr()), lda, C.c_void_p(B.data_ptr()), ldb,
                               C.c_void_p(Cout.data_ptr()), ldc, C.c_void_p(s)))
+
+
+LP_XENT_STATIC_MAX_BATCH = 16384
+
+
+def lp_softmax_xent_static(logits, labels, delta, loss, classes, stream=None):
+    """Loss kernel on caller-owned torch tensors, no handle and no allocation inside the
+    library: logits fp32 [batch][ld], labels int32 [batch], delta bf16 [batch][ld_delta]
+    (output), loss fp32 [1] (output).  Returns the library's status code."""
+    import torch
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    return lib().lp_softmax_xent_static(C.c_void_p(logits.data_ptr()), logits.stride(0),
+                                        C.c_void_p(labels.data_ptr()), C.c_void_p(delta.data_ptr()),
+                                        delta.stride(0), C.c_void_p(loss.data_ptr()), logits.shape[0], classes,
+                                        C.c_void_p(s))

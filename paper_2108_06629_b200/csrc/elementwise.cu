@@ -1,5 +1,7 @@
 // HBM-bound kernels of the training step: input cast + stash, softmax cross-entropy with
 // delta^L, and the fused SGD update (Eq. 6) that also refreshes the bf16 weight-ring slot.
+#include <cstdio>
+
 #include "common.h"
 
 namespace lp {
@@ -231,3 +233,49 @@ cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long
   return cudaGetLastError();
 }
 }  // namespace lp
+
+// ---------------------------------------------------------------------------
+// lp_softmax_xent_static: the loss kernel for callers that cannot supply scratch memory.
+// The per-row losses and the completion counter live in this fixed device array instead
+// of a workspace.  Host code must not pass `g_xent_scratch` itself to a kernel: in host
+// code that name is only a handle for the runtime.  The device address is looked up once
+// per device with cudaGetSymbolAddress and that pointer is what the kernel receives.
+struct XentScratch {
+  float row_loss[LP_XENT_STATIC_MAX_BATCH];
+  unsigned ticket;
+};
+static __device__ __align__(256) unsigned char g_xent_scratch[sizeof(XentScratch)];
+
+namespace {
+constexpr int kMaxDevices = 64;
+XentScratch* g_xent_scratch_addr[kMaxDevices] = {};   // device address of the array, per device
+thread_local char g_xent_err[160];
+}  // namespace
+
+extern "C" int lp_softmax_xent_static(const float* logits_dev, int ld_logits, const int* labels_dev,
+                                      void* delta_dev, int ld_delta, float* loss_dev, int batch, int classes,
+                                      void* stream) {
+  if (!logits_dev || !labels_dev || !delta_dev || !loss_dev) return LP_ERR_INVALID_ARG;
+  if (batch < 1 || classes < 1) return LP_ERR_INVALID_ARG;
+  if (batch > LP_XENT_STATIC_MAX_BATCH) return LP_ERR_INVALID_ARG;   // the fixed scratch holds no more rows
+  if (ld_logits < classes || ld_delta < ((classes + 7) & ~7)) return LP_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LP_ERR_CUDA;
+  if (g_xent_scratch_addr[dev] == nullptr) {
+    // set-up, once per device, with that device current: ask the runtime where the array lives
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_xent_scratch);
+    if (e != cudaSuccess || p == nullptr) {
+      snprintf(g_xent_err, sizeof(g_xent_err), "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+      return LP_ERR_CUDA;
+    }
+    g_xent_scratch_addr[dev] = static_cast<XentScratch*>(p);
+  }
+  XentScratch* s = g_xent_scratch_addr[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the counter must start at zero whatever an earlier (possibly failed) call left behind
+  if (cudaMemsetAsync(&s->ticket, 0, sizeof(unsigned), st) != cudaSuccess) return LP_ERR_CUDA;
+  cudaError_t e = lp::launch_softmax_xent(logits_dev, ld_logits, labels_dev, static_cast<__nv_bfloat16*>(delta_dev),
+                                          ld_delta, s->row_loss, &s->ticket, loss_dev, batch, classes, st);
+  return e == cudaSuccess ? LP_OK : LP_ERR_CUDA;
+}
