@@ -57,9 +57,11 @@ def work_model(layers, batch, momentum):
                                    (4.0 if last else (4.0 if gelu else 2.0)) * batch * n_out))
         if l > 0:
             out["delta"].append(dict(flops=fl, bytes=2.0 * n_in * n_out + 2.0 * batch * n_out + 4.0 * batch * n_in))
-        out["G"].append(dict(flops=fl, bytes=2.0 * batch * (n_in + n_out) + 4.0 * n_in * n_out))
-        per_param = 22.0 if momentum != 0.0 else 14.0   # read G, W (,m); write W (,m) fp32 and the bf16 ring slot
-        out["update"].append(dict(flops=0.0, bytes=per_param * n_in * n_out))
+        # G with the update fused into its epilogue: read W (,m), write W (,m) fp32 and the bf16 ring slot
+        per_param = 18.0 if momentum != 0.0 else 10.0
+        out["G"].append(dict(flops=fl, bytes=2.0 * batch * (n_in + n_out) + per_param * n_in * n_out))
+        # what is left of the update: bias gradient (column sums of delta) and the bias update
+        out["update"].append(dict(flops=0.0, bytes=2.0 * batch * n_out + 24.0 * n_out))
     return out
 
 

@@ -49,7 +49,10 @@ enum { LP_SCHED_LAYERPIPE = 0, /* delta and G of a layer are separate concurrent
        LP_SCHED_FUSED_B = 1 }; /* PipeDream-style: delta, G, update = ONE serial task      */
 enum { LP_F32 = 0, LP_BF16 = 1 };
 enum { LP_CAPTURE_GRADS = 1u, /* keep G of the latest step readable by lp_get_grads            */
-       LP_TIME_TASKS = 2u };   /* bracket every kernel with timing events (see lp_get_task_time) */
+       LP_TIME_TASKS = 2u,     /* bracket every kernel with timing events (see lp_get_task_time) */
+       LP_UNFUSED_UPDATE = 4u }; /* write G to memory and run Eq. 6 as a separate kernel. Default:  */
+                               /* the update is fused into the epilogue of the G contraction and  */
+                               /* G is only stored when LP_CAPTURE_GRADS is set                    */
 
 /* One layer of the chain (Eqs. 1-2: z = W a (+ b), a = f(z)). */
 typedef struct {
@@ -138,8 +141,8 @@ int lp_flush(lp_handle h, void* stream);
 int lp_get_weights(lp_handle h, int layer, float* W_out, float* b_out, long long* version);
 
 /* G (host dW_out [out][in]) and bias gradient (host db_out [out]) of minibatch `step`;
- * only the most recently enqueued step is held -> otherwise LP_ERR_NOT_READY. Blocks the
- * host until that step's G task has finished. */
+ * needs LP_CAPTURE_GRADS (or LP_UNFUSED_UPDATE) and only the most recently enqueued step is
+ * held -> otherwise LP_ERR_NOT_READY. Blocks the host until that step's G task has finished. */
 int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* db_out);
 
 /*
@@ -169,8 +172,10 @@ int lp_debug_write(lp_handle h, int buffer, int layer, long long index, const fl
 /* Run ONE task of minibatch `step` on the buffers as they stand (slots and weight version
  * chosen exactly as lp_step would for that minibatch) and wait for it.  Does not advance
  * the step counter.  LP_TASK_FORWARD: Eqs. 1-2; LP_TASK_LOSS: loss and delta^L;
- * LP_TASK_DELTA: Eqs. 3-4 for layer >= 1 (writes delta^{layer-1}); LP_TASK_G: Eq. 5;
- * LP_TASK_UPDATE: Eq. 6 (writes ring slot (step+1) mod slots). */
+ * LP_TASK_DELTA: Eqs. 3-4 for layer >= 1 (writes delta^{layer-1}); LP_TASK_G: Eq. 5 -- with
+ * the fused update (default) this kernel also applies Eq. 6 to W and writes ring slot
+ * (step+1) mod slots; LP_TASK_UPDATE: Eq. 6 for the bias (fused mode) or for W and bias
+ * (LP_UNFUSED_UPDATE). */
 enum { LP_TASK_FORWARD = 0, LP_TASK_LOSS = 1, LP_TASK_DELTA = 2, LP_TASK_G = 3, LP_TASK_UPDATE = 4 };
 int lp_debug_run_task(lp_handle h, int task, int layer, long long step);
 
@@ -201,9 +206,10 @@ int lp_reset_task_times(lp_handle h);
 /* Number of kernels this handle has launched so far. */
 long long lp_kernel_launches(lp_handle h);
 
-/* Tuning hook for experiments: force the GEMM tile width (64, 128, 256; 0 = automatic) and
- * the shared-memory pipeline depth (0 = automatic) for handles created afterwards. */
-int lp_set_tuning(int tile_n, int stages);
+/* Tuning hook for experiments: force the GEMM tile width (64, 128, 256; 0 = automatic), the
+ * shared-memory pipeline depth (0 = automatic) and the split-K factor of the forward / delta
+ * contractions (0 = automatic, 1 = off) for handles created afterwards. */
+int lp_set_tuning(int tile_n, int stages, int split_k);
 
 const char* lp_last_error(lp_handle h); /* valid until the next call on h; h may be NULL */
 int lp_destroy(lp_handle h);

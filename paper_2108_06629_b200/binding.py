@@ -22,6 +22,7 @@ LP_SCHED_LAYERPIPE, LP_SCHED_FUSED_B = 0, 1
 LP_F32, LP_BF16 = 0, 1
 LP_CAPTURE_GRADS = 1
 LP_TIME_TASKS = 2
+LP_UNFUSED_UPDATE = 4
 
 
 class lp_layer(C.Structure):
@@ -73,7 +74,7 @@ def lib():
         "lp_device_status": [vp, ip],
         "lp_get_task_time": [vp, C.c_int, llp, _P(C.c_double)],
         "lp_reset_task_times": [vp],
-        "lp_set_tuning": [C.c_int, C.c_int],
+        "lp_set_tuning": [C.c_int, C.c_int, C.c_int],
         "lp_destroy": [vp],
         "lp_gemm_bf16": [C.c_int, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, vp],
         "lp_softmax_xent_static": [vp, C.c_int, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp],
@@ -156,8 +157,8 @@ def lp_workspace_size(layers, n_stages, stage, delays, batch, lr=0.01, momentum=
     return out.value
 
 
-def lp_set_tuning(tile_n=0, stages=0):
-    _check(lib().lp_set_tuning(tile_n, stages))
+def lp_set_tuning(tile_n=0, stages=0, split_k=0):
+    _check(lib().lp_set_tuning(tile_n, stages, split_k))
 
 
 class Trainer:

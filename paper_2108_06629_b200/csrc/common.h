@@ -28,7 +28,8 @@ void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]);
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, cudaStream_t stream);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process
-void gemm_set_tuning(int bn, int stages);   // 0 = automatic
+void gemm_set_tuning(int bn, int stages, int splits);   // 0 = automatic
+int gemm_pick_splits(int M, int N, int K, int bn);
 
 // ---- planner.cpp ------------------------------------------------------------
 struct PlanResult {

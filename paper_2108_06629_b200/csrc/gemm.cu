@@ -59,15 +59,40 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64
 // ---------------------------------------------------------------------------
 static int g_force_bn = 0;
 static int g_force_stages = 0;
-void gemm_set_tuning(int bn, int stages) {
+static int g_force_splits = 0;
+void gemm_set_tuning(int bn, int stages, int splits) {
   g_force_bn = bn;
   g_force_stages = stages;
+  g_force_splits = splits;
+}
+
+// Split-K factor.  Measured on B200 (M = 256, N = K = 4096): the split main loop is shorter
+// but writing and re-reading the fp32 partial tiles costs more than it saves (25 us unsplit,
+// 28 / 35 / 52 us at 2 / 4 / 8 splits), and under the stage scheduler other kernels fill the
+// idle SMs anyway.  So the automatic choice is "off"; the path stays for experiments and is
+// covered by the tests through lp_set_tuning.
+int gemm_pick_splits(int M, int N, int K, int bn) {
+  (void)M; (void)N; (void)bn;
+  const int num_kb = (K + GEMM_BK - 1) / GEMM_BK;
+  int s = g_force_splits > 0 ? g_force_splits : 1;
+  s = std::max(1, std::min(s, num_kb));
+  const int per = (num_kb + s - 1) / s;
+  return (num_kb + per - 1) / per;      // no empty split
 }
 
 int gemm_pick_bn(int which, int M, int N, int K) {
-  (void)which; (void)M; (void)K;
+  (void)which;
   if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
   if (N <= 64) return 64;
+  // 128 x 256 tiles need 96 B/clk of operands per SM instead of 128 B/clk and measured 1250 vs
+  // 1130 TFLOP/s on 2048 x 8192 x 8192; they only pay off when the contraction is long and
+  // there are enough tiles to fill two CTAs on every SM
+  const long long tiles256 = (long long)((M + GEMM_BM - 1) / GEMM_BM) * ((N + 255) / 256);
+  if (K >= 1024 && tiles256 >= 2 * 148) return 256;
+  // few tiles (small batch): one CTA can pull at most ~64 B/clk out of L2, so narrower tiles on
+  // twice as many SMs stream the weights faster even though the activations are re-read more
+  const long long tiles128 = (long long)((M + GEMM_BM - 1) / GEMM_BM) * ((N + 127) / 128);
+  if (tiles128 <= 74) return 64;
   return 128;
 }
 
@@ -87,45 +112,53 @@ static int pick_stages(int bn, int K) {
   return s;
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
-  a.num_stages = pick_stages(BN, a.K);
+  if (a.splits < 1 || MODE == EPI_WGRAD_UPDATE || a.partial == nullptr) a.splits = 1;
+  const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
+  a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
+  a.num_stages = pick_stages(BN, a.kb_per_split * GEMM_BK);
   const size_t smem = GemmSmem<BN>::bytes(a.num_stages);
-  dim3 grid((a.M + GEMM_BM - 1) / GEMM_BM, (a.N + BN - 1) / BN, 1);
-  gemm_tcgen05_kernel<BN, A_MN, B_MN><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a);
+  dim3 grid((a.M + GEMM_BM - 1) / GEMM_BM, (a.N + BN - 1) / BN, a.splits);
+  gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a);
   return cudaGetLastError();
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t configure_one() {
-  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               227 * 1024);
 }
 
+// instantiated combinations: (operand majors of the contraction) x (epilogue)
+#define LP_FOR_EACH_VARIANT(X, BN)           \
+  X(BN, false, false, EPI_FPROP)             \
+  X(BN, false, false, EPI_STORE_F32)         \
+  X(BN, false, true, EPI_DGRAD)              \
+  X(BN, false, true, EPI_STORE_F32)          \
+  X(BN, true, true, EPI_STORE_F32)           \
+  X(BN, true, true, EPI_WGRAD_UPDATE)
+
 cudaError_t gemm_configure() {
   cudaError_t e;
-#define LP_CFG(BN)                                                        \
-  if ((e = configure_one<BN, false, false>()) != cudaSuccess) return e;   \
-  if ((e = configure_one<BN, false, true>()) != cudaSuccess) return e;    \
-  if ((e = configure_one<BN, true, true>()) != cudaSuccess) return e;
-  LP_CFG(64) LP_CFG(128) LP_CFG(256)
+#define LP_CFG(BN, A, B, M) \
+  if ((e = configure_one<BN, A, B, M>()) != cudaSuccess) return e;
+  LP_FOR_EACH_VARIANT(LP_CFG, 64)
+  LP_FOR_EACH_VARIANT(LP_CFG, 128)
+  LP_FOR_EACH_VARIANT(LP_CFG, 256)
 #undef LP_CFG
   return cudaSuccess;
 }
 
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
                         cudaStream_t st) {
-#define LP_DISPATCH(BN)                                                       \
-  case BN:                                                                    \
-    if (which == 0) return launch_one<BN, false, false>(tmA, tmB, args, st);  \
-    if (which == 1) return launch_one<BN, false, true>(tmA, tmB, args, st);   \
-    return launch_one<BN, true, true>(tmA, tmB, args, st);
-  switch (bn) {
-    LP_DISPATCH(64)
-    LP_DISPATCH(128)
-    LP_DISPATCH(256)
-  }
-#undef LP_DISPATCH
+  const bool a_mn = (which == 2), b_mn = (which != 0);
+#define LP_TRY(BN, A, B, M) \
+  if (bn == BN && a_mn == A && b_mn == B && args.mode == M) return launch_one<BN, A, B, M>(tmA, tmB, args, st);
+  LP_FOR_EACH_VARIANT(LP_TRY, 64)
+  LP_FOR_EACH_VARIANT(LP_TRY, 128)
+  LP_FOR_EACH_VARIANT(LP_TRY, 256)
+#undef LP_TRY
   return cudaErrorInvalidValue;
 }
 

@@ -26,7 +26,7 @@ constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;   // 16 KiB
 constexpr int GEMM_MAX_STAGES = 8;
 
-enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2 };
+enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2, EPI_WGRAD_UPDATE = 3 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
 
 struct GemmArgs {
@@ -34,7 +34,7 @@ struct GemmArgs {
   int num_stages;
   int mode;                 // EPI_*
   int act;                  // ACT_*  (FPROP: f of this layer; DGRAD: f' of the previous layer)
-  void* out;                // STORE_F32: float [M][ld_out]; FPROP: bf16 a^l (may be null); DGRAD: bf16 delta^{l-1}
+  void* out;                // STORE_F32 / WGRAD_UPDATE: float [M][ld_out]; FPROP: bf16 a^l (may be null); DGRAD: bf16 delta^{l-1}
   int ld_out;
   void* out2;               // FPROP: bf16 stored z^l (GELU) or fp32 z^L (last layer); else null
   int ld_out2;
@@ -42,6 +42,19 @@ struct GemmArgs {
   const float* bias;        // FPROP: fp32 [N] or null
   const __nv_bfloat16* aux; // DGRAD: what f' is evaluated on (stored z for GELU, a for ReLU)
   int ld_aux;
+  // EPI_WGRAD_UPDATE: fp32 master / momentum (may be null) / bf16 ring slot, all [M][ld_out];
+  // `out` (may be null) additionally receives G
+  float* W;
+  float* mW;
+  __nv_bfloat16* ring;
+  float lr, mu;
+  // split-K (splits > 1): blockIdx.z owns k-blocks [z*kb_per_split, (z+1)*kb_per_split); every CTA
+  // writes its fp32 partial tile to `partial`, the last CTA of a tile to arrive (tile_counter)
+  // adds the partials in split order -- a fixed order, so results do not depend on timing --
+  // and runs the epilogue.  Not available with EPI_WGRAD_UPDATE.
+  int splits, kb_per_split;
+  float* partial;           // [tiles][splits][128][BN]
+  unsigned* tile_counter;   // [tiles], zero between launches
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -60,6 +73,107 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
+
+constexpr int EPI_PITCH = 36;                       // floats; 32 + 4 keeps 128-bit accesses conflict-free
+constexpr int EPI_TILE_BYTES = 4 * 32 * EPI_PITCH * 4;   // one 32 x 32 staging tile per epilogue warp (18 KiB)
+static_assert(EPI_TILE_BYTES <= GEMM_A_BYTES + 64 * GEMM_BK * 2, "staging tiles must fit in one pipeline stage");
+
+// Epilogue for 4 consecutive columns n..n+3 of output row `row`.  Lanes past N inside the
+// last 16-byte (fp32) / 8-element (bf16) group are written as zeros; groups that start
+// beyond that are skipped.
+template <int MODE>
+__device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int n, float4 acc) {
+  const int N = p.N;
+  float v[4] = {n + 0 < N ? acc.x : 0.f, n + 1 < N ? acc.y : 0.f, n + 2 < N ? acc.z : 0.f, n + 3 < N ? acc.w : 0.f};
+  const int n_pad4 = (N + 3) & ~3, n_pad8 = (N + 7) & ~7;
+  if (MODE == EPI_STORE_F32) {
+    if (n >= n_pad4) return;
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + size_t(row) * p.ld_out + n) = make_float4(v[0], v[1], v[2], v[3]);
+  } else if (MODE == EPI_FPROP) {
+    if (n >= n_pad8) return;
+    if (p.bias != nullptr) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) if (n + j < N) v[j] += __ldg(p.bias + n + j);
+    }
+    if (p.out2 != nullptr) {
+      if (p.out2_is_f32) {
+        if (n < n_pad4)
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out2) + size_t(row) * p.ld_out2 + n) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out2) + size_t(row) * p.ld_out2 + n) =
+            make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+      }
+    }
+    if (p.out != nullptr) {
+      if (p.act == ACT_RELU) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
+      } else if (p.act == ACT_GELU) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = gelu_fwd(v[j]);
+      }
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
+          make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+    }
+  } else if (MODE == EPI_DGRAD) {
+    // delta^{l-1} = (delta^l W) (.) f'(z^{l-1}), one rounding
+    if (n >= n_pad8) return;
+    if (p.act != ACT_NONE) {
+      const uint2 av = *reinterpret_cast<const uint2*>(p.aux + size_t(row) * p.ld_aux + n);
+      const float z[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = (p.act == ACT_RELU) ? (z[j] > 0.f ? v[j] : 0.f) : v[j] * gelu_grad(z[j]);
+    }
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
+        make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+  }
+}
+
+// ---- fused G + update epilogue (EPI_WGRAD_UPDATE) -------------------------------------------
+// The accumulator chunk is G; the epilogue streams the fp32 master (and momentum) tile through
+// registers: m <- mu m + G; W <- W - eta m; ring <- RN(W).  It is an HBM-streaming loop with
+// few warps, so the loads of the NEXT 32 x 32 chunk are issued before the current chunk is
+// processed (and those of the first chunk before the accumulator is even complete).
+struct WmRegs {
+  float4 w[8];
+  float4 m[8];
+};
+__device__ __forceinline__ void load_wm(const GemmArgs& p, int row0, int n, int sub_row, WmRegs& r) {
+  const bool col_ok = n < ((p.N + 7) & ~7);
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int row = row0 + it * 4 + sub_row;
+    const bool ok = col_ok && row < p.M;
+    const size_t off = size_t(row) * p.ld_out + n;
+    r.w[it] = ok ? __ldcs(reinterpret_cast<const float4*>(p.W + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.mW != nullptr) r.m[it] = ok ? __ldcs(reinterpret_cast<const float4*>(p.mW + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+__device__ __forceinline__ void apply_update(const GemmArgs& p, int row0, int n, int sub_row, const float* tile,
+                                             int sub_col, const WmRegs& r) {
+  if (n >= ((p.N + 7) & ~7)) return;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int rr = it * 4 + sub_row;
+    const int row = row0 + rr;
+    if (row >= p.M) continue;
+    const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
+    float g[4] = {n + 0 < p.N ? acc.x : 0.f, n + 1 < p.N ? acc.y : 0.f, n + 2 < p.N ? acc.z : 0.f, n + 3 < p.N ? acc.w : 0.f};
+    const size_t off = size_t(row) * p.ld_out + n;
+    if (p.out != nullptr) __stcs(reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off), make_float4(g[0], g[1], g[2], g[3]));
+    float m[4] = {g[0], g[1], g[2], g[3]};
+    if (p.mW != nullptr) {
+      m[0] = p.mu * r.m[it].x + g[0]; m[1] = p.mu * r.m[it].y + g[1];
+      m[2] = p.mu * r.m[it].z + g[2]; m[3] = p.mu * r.m[it].w + g[3];
+      __stcs(reinterpret_cast<float4*>(p.mW + off), make_float4(m[0], m[1], m[2], m[3]));
+    }
+    float4 w = r.w[it];
+    w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
+    __stcs(reinterpret_cast<float4*>(p.W + off), w);
+    *reinterpret_cast<uint2*>(p.ring + off) = make_uint2(pack_bf16x2(w.x, w.y), pack_bf16x2(w.z, w.w));
+  }
+}
+
 template <int BN>
 struct GemmSmem {
   static constexpr int B_BYTES = BN * GEMM_BK * 2;
@@ -67,8 +181,8 @@ struct GemmSmem {
   static constexpr size_t bytes(int stages) { return size_t(stages) * STAGE_BYTES + 1024 /*align slack*/ + 256; }
 };
 
-template <int BN, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int BN, bool A_MN, bool B_MN, int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmArgs p) {
   using SM = GemmSmem<BN>;
@@ -79,12 +193,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
   uint64_t* acc_bar = empty_bar + GEMM_MAX_STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+  // the epilogue's staging tiles reuse pipeline stage 0: by the time the accumulator barrier
+  // fires every TMA load has landed and every MMA has finished reading shared memory
+  float* epi_tile = reinterpret_cast<float*>(smem);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * GEMM_BM;
   const int n0 = blockIdx.y * BN;
-  const int num_kb = (p.K + GEMM_BK - 1) / GEMM_BK;
+  const int num_kb_total = (p.K + GEMM_BK - 1) / GEMM_BK;
+  const int kb_begin = (p.splits > 1) ? int(blockIdx.z) * p.kb_per_split : 0;
+  const int num_kb = (p.splits > 1) ? max(0, min(num_kb_total, kb_begin + p.kb_per_split) - kb_begin) : num_kb_total;
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
@@ -107,31 +226,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
+    // One lane runs this loop; everything it needs per k-block is kept in registers as raw
+    // 32-bit shared-memory addresses so that the instruction stream between two TMA issues
+    // stays short (a single thread issues at a few cycles per instruction).
     if (lane == 0) {
       bool ok = true;
       int issued = 0;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        ok = mbar_wait(&empty_bar[s], ph ^ 1u);
+      const uint32_t smem0 = smem_u32(smem);
+      const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+      uint32_t s = 0, ph = 0;
+      int k0 = kb_begin * GEMM_BK;
+      for (int kb = 0; kb < num_kb; ++kb, k0 += GEMM_BK) {
+        ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
         if (!ok) break;
-        uint8_t* sa = smem + size_t(s) * SM::STAGE_BYTES;
-        uint8_t* sb = sa + GEMM_A_BYTES;
-        mbar_arrive_expect_tx(&full_bar[s], SM::STAGE_BYTES);
-        const int k0 = kb * GEMM_BK;
+        const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
+        const uint32_t sb = sa + GEMM_A_BYTES;
+        const uint32_t fb = full0 + 8u * s;
+        mbar_arrive_expect_tx_addr(fb, SM::STAGE_BYTES);
         if (A_MN) {
 #pragma unroll
-          for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d(sa + c * 8192, &tmA, &full_bar[s], m0 + c * 64, k0);
+          for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d_addr(sa + c * 8192, &tmA, fb, m0 + c * 64, k0);
         } else {
-          tma_load_2d(sa, &tmA, &full_bar[s], k0, m0);
+          tma_load_2d_addr(sa, &tmA, fb, k0, m0);
         }
         if (B_MN) {
 #pragma unroll
-          for (int c = 0; c < BN / 64; ++c) tma_load_2d(sb + c * 8192, &tmB, &full_bar[s], n0 + c * 64, k0);
+          for (int c = 0; c < BN / 64; ++c) tma_load_2d_addr(sb + c * 8192, &tmB, fb, n0 + c * 64, k0);
         } else {
-          tma_load_2d(sb, &tmB, &full_bar[s], k0, n0);
+          tma_load_2d_addr(sb, &tmB, fb, k0, n0);
         }
         issued = kb + 1;
+        if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
         atomicExch(p.status, 1);
@@ -143,36 +268,61 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(GEMM_BM, BN, A_MN, B_MN);
+      // descriptors of stage 0, k-slice 0; other stages / slices only move the 14-bit start
+      // address field (units of 16 bytes), which cannot carry out of the low word
+      const uint64_t dA = A_MN ? make_smem_desc(smem_u32(smem), 8192, 1024) : make_smem_desc(smem_u32(smem), 16, 1024);
+      const uint64_t dB = B_MN ? make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 8192, 1024)
+                               : make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 16, 1024);
+      const uint32_t dA_hi = uint32_t(dA >> 32), dB_hi = uint32_t(dB >> 32);
+      constexpr uint32_t stepA = (A_MN ? 2048 : 32) >> 4, stepB = (B_MN ? 2048 : 32) >> 4;
+      const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+      uint32_t s = 0, ph = 0, acc = 0;
+      uint32_t dA_lo = uint32_t(dA), dB_lo = uint32_t(dB);
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        ok = mbar_wait(&full_bar[s], ph);
+        ok = mbar_wait_addr(full0 + 8u * s, ph);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + size_t(s) * SM::STAGE_BYTES);
-        const uint32_t sb = sa + GEMM_A_BYTES;
 #pragma unroll
         for (int j = 0; j < GEMM_BK / 16; ++j) {
-          const uint64_t da = A_MN ? make_smem_desc(sa + j * 2048, 8192, 1024) : make_smem_desc(sa + j * 32, 16, 1024);
-          const uint64_t db = B_MN ? make_smem_desc(sb + j * 2048, 8192, 1024) : make_smem_desc(sb + j * 32, 16, 1024);
-          umma_f16(tmem_base, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+          umma_f16_lohi(tmem_base, dA_lo + j * stepA, dA_hi, dB_lo + j * stepB, dB_hi, idesc, acc);
+          acc = 1;
         }
-        umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+        umma_commit_addr(empty0 + 8u * s);   // frees the stage once these MMAs have read it
+        dA_lo += uint32_t(SM::STAGE_BYTES >> 4);
+        dB_lo += uint32_t(SM::STAGE_BYTES >> 4);
+        if (++s == uint32_t(S)) {
+          s = 0;
+          ph ^= 1u;
+          dA_lo = uint32_t(dA);
+          dB_lo = uint32_t(dB);
+        }
       }
       if (!ok) atomicExch(p.status, 2);
       umma_commit(acc_bar);           // accumulator complete (also releases the epilogue on error)
     }
   } else {
     // ------------------------------------------------------------ epilogue
+    // tcgen05.ld hands each lane one accumulator ROW (32 consecutive columns).  Storing from
+    // that layout would touch 32 rows per instruction, so every 32 x 32 chunk is first
+    // transposed through a padded per-warp shared-memory tile; afterwards a lane owns 4
+    // consecutive columns of one row and a warp instruction covers 4 rows x 128 contiguous
+    // bytes (fp32) -- fully used sectors for every load and store of the epilogue.
     const int q = warp & 3;           // tensor-memory lane quarter this warp may read
-    const int row = m0 + q * 32 + lane;
-    // stores go out in 16-byte groups; the lanes of the last group past N are written as zeros
-    const int n_pad4 = (p.N + 3) & ~3, n_pad8 = (p.N + 7) & ~7;
+    float* tile = epi_tile + q * (32 * EPI_PITCH);
+    const int sub_row = lane >> 3;        // 0..3
+    const int sub_col = (lane & 7) * 4;   // 0,4,..,28
+    const int row0 = m0 + q * 32;
+    constexpr bool upd = (MODE == EPI_WGRAD_UPDATE);
+    WmRegs cur;
+    if constexpr (upd) load_wm(p, row0, n0 + sub_col, sub_row, cur);      // in flight while the main loop runs
     bool ok = mbar_wait(acc_bar, 0);
     ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
     if (!ok && lane == 0) atomicExch(p.status, 3);
     tc_fence_after();
+    const bool split = (!upd) && p.splits > 1;
+    const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
+    float* part = split ? p.partial + (size_t(tile_id) * p.splits + blockIdx.z) * (size_t(GEMM_BM) * BN) : nullptr;
     if (ok) {
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
@@ -180,107 +330,62 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         __syncwarp();
         tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
         tmem_ld_wait();
-        const int nb = n0 + c * 32;
-        if (row >= p.M) {
-          // rows past M hold zeros (TMA zero fill); nothing to store
-        } else if (p.mode == EPI_STORE_F32) {
-          float* o = reinterpret_cast<float*>(p.out) + size_t(row) * p.ld_out;
 #pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            const int n = nb + g * 4;
-            if (n >= n_pad4) break;
-            float4 v;
-            v.x = (n + 0 < p.N) ? __uint_as_float(r[g * 4 + 0]) : 0.f;
-            v.y = (n + 1 < p.N) ? __uint_as_float(r[g * 4 + 1]) : 0.f;
-            v.z = (n + 2 < p.N) ? __uint_as_float(r[g * 4 + 2]) : 0.f;
-            v.w = (n + 3 < p.N) ? __uint_as_float(r[g * 4 + 3]) : 0.f;
-            *reinterpret_cast<float4*>(o + n) = v;
-          }
-        } else if (p.mode == EPI_FPROP) {
-          float z[32];
+        for (int g = 0; g < 8; ++g)
+          *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+        __syncwarp();
+        const int n = n0 + c * 32 + sub_col;
+        if constexpr (upd) {
+          WmRegs nxt;
+          if (c + 1 < BN / 32) load_wm(p, row0, n + 32, sub_row, nxt);
+          apply_update(p, row0, n, sub_row, tile, sub_col, cur);
+          cur = nxt;
+        } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int n = nb + j;
-            float b = 0.f;
-            if (p.bias != nullptr && n < p.N) b = __ldg(p.bias + n);
-            z[j] = (n < p.N) ? __uint_as_float(r[j]) + b : 0.f;
-          }
-          if (p.out2 != nullptr) {
-            if (p.out2_is_f32) {
-              float* o = reinterpret_cast<float*>(p.out2) + size_t(row) * p.ld_out2;
-#pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                const int n = nb + g * 4;
-                if (n >= n_pad4) break;
-                *reinterpret_cast<float4*>(o + n) = make_float4(z[g * 4], z[g * 4 + 1], z[g * 4 + 2], z[g * 4 + 3]);
-              }
-            } else {
-              __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out2) + size_t(row) * p.ld_out2;
-#pragma unroll
-              for (int g = 0; g < 4; ++g) {
-                const int n = nb + g * 8;
-                if (n >= n_pad8) break;
-                uint4 v;
-                v.x = pack_bf16x2(z[g * 8 + 0], z[g * 8 + 1]);
-                v.y = pack_bf16x2(z[g * 8 + 2], z[g * 8 + 3]);
-                v.z = pack_bf16x2(z[g * 8 + 4], z[g * 8 + 5]);
-                v.w = pack_bf16x2(z[g * 8 + 6], z[g * 8 + 7]);
-                *reinterpret_cast<uint4*>(o + n) = v;
-              }
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + sub_row;
+            const int row = row0 + rr;
+            const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
+            if (split) {
+              __stcg(reinterpret_cast<float4*>(part + size_t(q * 32 + rr) * BN + c * 32 + sub_col), acc);
+            } else if (row < p.M) {
+              epilogue_store4<MODE>(p, row, n, acc);
             }
           }
-          if (p.out != nullptr) {
-            if (p.act == ACT_RELU) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) z[j] = fmaxf(z[j], 0.f);
-            } else if (p.act == ACT_GELU) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) z[j] = gelu_fwd(z[j]);
+        }
+      }
+    }
+    if (split) {
+      // all four epilogue warps have written their part of the partial tile: publish it, and
+      // let the last CTA of this tile reduce the partials in split order
+      volatile uint32_t* is_last = tmem_slot + 1;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (threadIdx.x == 64) {
+        __threadfence();
+        const unsigned prev = atomicAdd(p.tile_counter + tile_id, 1u);
+        const bool last = (prev == unsigned(p.splits) - 1u);
+        if (last) p.tile_counter[tile_id] = 0u;          // ready for the next launch
+        *is_last = last ? 1u : 0u;
+        __threadfence();
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*is_last != 0u) {
+        const float* base = p.partial + size_t(tile_id) * p.splits * (size_t(GEMM_BM) * BN);
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const int n = n0 + c * 32 + sub_col;
+#pragma unroll 2
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + sub_row;
+            const int row = row0 + rr;
+            if (row >= p.M) continue;
+            const float* src = base + size_t(q * 32 + rr) * BN + c * 32 + sub_col;
+            float4 acc = __ldcg(reinterpret_cast<const float4*>(src));
+            for (int z = 1; z < p.splits; ++z) {
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(src + size_t(z) * GEMM_BM * BN));
+              acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
             }
-            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out;
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const int n = nb + g * 8;
-              if (n >= n_pad8) break;
-              uint4 v;
-              v.x = pack_bf16x2(z[g * 8 + 0], z[g * 8 + 1]);
-              v.y = pack_bf16x2(z[g * 8 + 2], z[g * 8 + 3]);
-              v.z = pack_bf16x2(z[g * 8 + 4], z[g * 8 + 5]);
-              v.w = pack_bf16x2(z[g * 8 + 6], z[g * 8 + 7]);
-              *reinterpret_cast<uint4*>(o + n) = v;
-            }
-          }
-        } else {  // EPI_DGRAD: delta^{l-1} = (delta^l W) (.) f'(z^{l-1}), one rounding
-          const __nv_bfloat16* a = p.aux + size_t(row) * p.ld_aux;
-          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out;
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int n = nb + g * 8;
-            if (n >= n_pad8) break;
-            float d[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) d[j] = (n + j < p.N) ? __uint_as_float(r[g * 8 + j]) : 0.f;
-            if (p.act != ACT_NONE) {
-              const uint4 av = *reinterpret_cast<const uint4*>(a + n);
-              const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float z0 = bf16_lo(aw[j]), z1 = bf16_hi(aw[j]);
-                if (p.act == ACT_RELU) {
-                  d[2 * j] = z0 > 0.f ? d[2 * j] : 0.f;
-                  d[2 * j + 1] = z1 > 0.f ? d[2 * j + 1] : 0.f;
-                } else {
-                  d[2 * j] *= gelu_grad(z0);
-                  d[2 * j + 1] *= gelu_grad(z1);
-                }
-              }
-            }
-            uint4 v;
-            v.x = pack_bf16x2(d[0], d[1]);
-            v.y = pack_bf16x2(d[2], d[3]);
-            v.z = pack_bf16x2(d[4], d[5]);
-            v.w = pack_bf16x2(d[6], d[7]);
-            *reinterpret_cast<uint4*>(o + n) = v;
+            epilogue_store4<MODE>(p, row, n, acc);
           }
         }
       }

@@ -53,6 +53,9 @@ struct Layer {
   size_t w_elems = 0, x_elems = 0, z_elems = 0, delta_elems = 0;
   int z_slots = 0;
   int bn_f = 128, bn_d = 128, bn_g = 128;
+  int split_f = 1, split_d = 1;                 // split-K factors of the forward / delta contractions
+  float *part_f = nullptr, *part_d = nullptr;   // fp32 partial tiles [tiles][splits][128][BN]
+  unsigned *cnt_f = nullptr, *cnt_d = nullptr;  // per-tile arrival counters
   std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
   std::vector<Res> rX, rZ, rDelta, rRing;
   Res rDW;
@@ -182,7 +185,8 @@ static size_t carve(lp_ctx* c, char* base) {
     y.w_elems = size_t(y.n_out) * y.ld_in;
     y.W = reinterpret_cast<float*>(take(y.w_elems * 4));
     y.mW = mom ? reinterpret_cast<float*>(take(y.w_elems * 4)) : nullptr;
-    y.dW = reinterpret_cast<float*>(take(y.w_elems * 4));
+    const bool keep_G = (c->cfg.flags & (LP_CAPTURE_GRADS | LP_UNFUSED_UPDATE)) != 0;
+    y.dW = keep_G ? reinterpret_cast<float*>(take(y.w_elems * 4)) : nullptr;
     y.ring = reinterpret_cast<__nv_bfloat16*>(take(y.w_elems * 2 * y.slots));
     y.b = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4));
     y.mb = mom ? reinterpret_cast<float*>(take(size_t(y.ld_out) * 4)) : nullptr;
@@ -198,6 +202,17 @@ static size_t carve(lp_ctx* c, char* base) {
       y.z_slots = c->L[l + 1].x_slots;
       y.z_elems = size_t(B) * y.ld_out;
       y.Z = reinterpret_cast<__nv_bfloat16*>(take(y.z_elems * 2 * y.z_slots));
+    }
+    auto tiles_of = [&](int M, int N, int bn) { return size_t((M + GEMM_BM - 1) / GEMM_BM) * ((N + bn - 1) / bn); };
+    if (y.split_f > 1) {
+      const size_t t = tiles_of(B, y.n_out, y.bn_f);
+      y.part_f = reinterpret_cast<float*>(take(t * y.split_f * GEMM_BM * y.bn_f * 4));
+      y.cnt_f = reinterpret_cast<unsigned*>(take(t * 4));
+    }
+    if (y.split_d > 1 && l > 0) {
+      const size_t t = tiles_of(B, y.n_in, y.bn_d);
+      y.part_d = reinterpret_cast<float*>(take(t * y.split_d * GEMM_BM * y.bn_d * 4));
+      y.cnt_d = reinterpret_cast<unsigned*>(take(t * 4));
     }
   }
   c->zL = reinterpret_cast<float*>(take(size_t(kDeltaSlots) * B * c->ld_cls * 4));
@@ -223,6 +238,12 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     y.ld_in = pad8(y.n_in);
     y.ld_out = pad8(y.n_out);
     y.x_slots = y.delay + 1 + kExtraStashSlots;
+    const int B = c->cfg.batch;
+    y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
+    y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
+    y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
+    y.split_f = gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
+    y.split_d = gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
   }
   c->classes = layers[n - 1].out;
   c->ld_cls = pad8(c->classes);
@@ -273,9 +294,6 @@ static int build_tensor_maps(lp_ctx* c) {
   std::string err;
   for (int l = 0; l < nL; ++l) {
     Layer& y = c->L[l];
-    y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
-    y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
-    y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
     uint32_t bA[2], bB[2];
     int rc;
     // forward: A = a^{l-1} [B][in] K-major; B = W [out][in] K-major
@@ -372,6 +390,7 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
       a.ld_out2 = y.ld_out;
     }
   }
+  a.splits = y.split_f; a.partial = y.part_f; a.tile_counter = y.cnt_f;
   ++c->launches;
   TimedScope ts(c, LP_TASK_FORWARD, st);
   return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
@@ -394,19 +413,33 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
     a.ld_aux = y.ld_in;
   }
   a.status = c->status;
+  a.splits = y.split_d; a.partial = y.part_d; a.tile_counter = y.cnt_d;
   ++c->launches;
   TimedScope ts(c, LP_TASK_DELTA, st);
   return gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
 }
 
+static inline bool fused_update(const lp_ctx* c) { return (c->cfg.flags & LP_UNFUSED_UPDATE) == 0; }
+
 static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
   GemmArgs a{};
   a.M = y.n_out; a.N = y.n_in; a.K = c->cfg.batch;
-  a.mode = EPI_STORE_F32;
-  a.out = y.dW;
   a.ld_out = y.ld_in;
   a.status = c->status;
+  if (fused_update(c)) {
+    // Eq. 5 and Eq. 6 in one kernel: the accumulator tile is G; the epilogue reads the fp32
+    // master (and momentum) tile, applies the update and writes master, momentum and the
+    // bf16 version for minibatch n+1 -- G itself only goes to memory when it is captured
+    a.mode = EPI_WGRAD_UPDATE;
+    a.out = (c->cfg.flags & LP_CAPTURE_GRADS) ? y.dW : nullptr;
+    a.W = y.W; a.mW = y.mW;
+    a.ring = y.ring + size_t((n + 1) % y.slots) * y.w_elems;
+    a.lr = c->cfg.lr; a.mu = c->cfg.momentum;
+  } else {
+    a.mode = EPI_STORE_F32;
+    a.out = y.dW;
+  }
   ++c->launches;
   TimedScope ts(c, LP_TASK_G, st);
   return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st);
@@ -418,7 +451,8 @@ static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st)
   UpdateArgs u{};
   u.dW = y.dW; u.W = y.W; u.mW = y.mW;
   u.ring = y.ring + size_t(dst_slot) * y.w_elems;
-  u.n_elems = (long long)y.w_elems;
+  u.n_elems = fused_update(c) ? 0 : (long long)y.w_elems;   // fused: W was updated by the G kernel
+  if (u.n_elems == 0 && !y.d.has_bias) return cudaSuccess;  // nothing left to do
   if (y.d.has_bias) {
     u.delta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
     u.rows = c->cfg.batch; u.ldd = y.ld_out; u.n_out = y.n_out;
@@ -544,10 +578,11 @@ extern "C" int lp_destroy(lp_handle h) {
 
 extern "C" const char* lp_last_error(lp_handle h) { return h ? h->err.c_str() : g_err.c_str(); }
 
-extern "C" int lp_set_tuning(int tile_n, int stages) {
-  if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) || stages < 0 || stages > GEMM_MAX_STAGES)
+extern "C" int lp_set_tuning(int tile_n, int stages, int split_k) {
+  if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) || stages < 0 || stages > GEMM_MAX_STAGES ||
+      split_k < 0 || split_k > 64)
     return LP_ERR_INVALID_ARG;
-  gemm_set_tuning(tile_n, stages);
+  gemm_set_tuning(tile_n, stages, split_k);
   return LP_OK;
 }
 
@@ -664,12 +699,21 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
         LP_CUDA(c, task_end(c, st, {rdl, rw, raux}, {rdprev}, nullptr));
       }
       cudaStream_t sg = c->sG[y.stage];
-      LP_CUDA(c, task_begin(c, sg, {rdl, rx}, {&y.rDW}));
-      LP_CUDA(c, launch_G(c, l, n, sg));
-      LP_CUDA(c, task_end(c, sg, {rdl, rx}, {&y.rDW}, nullptr));
-      LP_CUDA(c, task_begin(c, sg, {&y.rDW, rdl}, {rnew}));
-      LP_CUDA(c, launch_update(c, l, n, sg));
-      LP_CUDA(c, task_end(c, sg, {&y.rDW, rdl}, {rnew}, &y.last_update));
+      if (fused_update(c)) {
+        // G + update of W in one kernel, then the bias update: one task that writes the ring
+        // slot of version n+1 (the slot delta_l(n) reads, so the tracker orders it after it)
+        LP_CUDA(c, task_begin(c, sg, {rdl, rx}, {&y.rDW, rnew}));
+        LP_CUDA(c, launch_G(c, l, n, sg));
+        LP_CUDA(c, launch_update(c, l, n, sg));
+        LP_CUDA(c, task_end(c, sg, {rdl, rx}, {&y.rDW, rnew}, &y.last_update));
+      } else {
+        LP_CUDA(c, task_begin(c, sg, {rdl, rx}, {&y.rDW}));
+        LP_CUDA(c, launch_G(c, l, n, sg));
+        LP_CUDA(c, task_end(c, sg, {rdl, rx}, {&y.rDW}, nullptr));
+        LP_CUDA(c, task_begin(c, sg, {&y.rDW, rdl}, {rnew}));
+        LP_CUDA(c, launch_update(c, l, n, sg));
+        LP_CUDA(c, task_end(c, sg, {&y.rDW, rdl}, {rnew}, &y.last_update));
+      }
     }
   }
   c->n_steps = n + 1;
@@ -714,6 +758,7 @@ extern "C" int lp_get_grads(lp_handle h, int layer, long long step, float* dW_ou
   if (layer < 0 || layer >= int(h->L.size())) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
   if (step != h->n_steps - 1 || step < 0) return fail(h, LP_ERR_NOT_READY, "only the latest step's gradients are held");
   Layer& y = h->L[layer];
+  if (dW_out && !y.dW) return fail(h, LP_ERR_NOT_READY, "G is not kept: create the handle with LP_CAPTURE_GRADS");
   if (y.last_update.e) LP_CUDA(h, cudaEventSynchronize(y.last_update.e));
   if (dW_out)
     LP_CUDA(h, cudaMemcpy2D(dW_out, size_t(y.n_in) * 4, y.dW, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
@@ -765,7 +810,10 @@ static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v)
       if (!y.mb) return fail(h, LP_ERR_NOT_READY, "momentum is off");
       *v = {y.mb, 1, y.n_out, y.ld_out, 1};
       return LP_OK;
-    case LP_BUF_GRAD_W: *v = {y.dW, y.n_out, y.n_in, y.ld_in, 1}; return LP_OK;
+    case LP_BUF_GRAD_W:
+      if (!y.dW) return fail(h, LP_ERR_NOT_READY, "G is not kept: create the handle with LP_CAPTURE_GRADS");
+      *v = {y.dW, y.n_out, y.n_in, y.ld_in, 1};
+      return LP_OK;
     case LP_BUF_GRAD_B: *v = {y.db, 1, y.n_out, y.ld_out, 1}; return LP_OK;
   }
   return fail(h, LP_ERR_INVALID_ARG, "unknown buffer");

@@ -46,12 +46,15 @@ def vgg(hw, plan, fcs, act="relu"):
     return layers
 
 
-# The five workloads: (layers, batch, stages, delays or None = planner, lr, momentum, parity steps)
+# The five workloads: (layers, batch, stages, delays or None = planner, lr, momentum, parity steps).
+# Step sizes are 0.01 where the workload list does not state one, except mlp8_4096: with
+# momentum 0.9 and gradients up to 7 minibatches stale, 0.01 diverges after about 150
+# minibatches (losses overflow), so it runs at 0.001.
 WORKLOADS = {
     "mlp4_784": dict(layers=mlp([784, 256, 256, 256, 10], "relu"), batch=32, stages=4,
                      delays=[3, 2, 1, 0], lr=0.01, momentum=0.0, steps=10),
     "mlp8_4096": dict(layers=mlp([4096] * 8 + [1000], "gelu"), batch=256, stages=8,
-                      delays=[7, 6, 5, 4, 3, 2, 1, 0], lr=0.01, momentum=0.9, steps=50),
+                      delays=[7, 6, 5, 4, 3, 2, 1, 0], lr=0.001, momentum=0.9, steps=50),
     "vgg_small_32": dict(layers=vgg(32, [64, 64, "P", 128, 128, "P", 256, 256, "P"], [512, 10]),
                          batch=128, stages=7, delays=None, lr=0.01, momentum=0.0, steps=10),
     "vgg16_224": dict(layers=vgg(224, [64, 64, "P", 128, 128, "P", 256, 256, 256, "P",

@@ -69,8 +69,11 @@ def test_workspace_size_is_pure_host_arithmetic():
     params = sum(l["n_in"] * l["n_out"] for l in wl["layers"])
     ring = sum(l["n_in"] * l["n_out"] * (d + 1) for l, d in zip(wl["layers"], wl["delays"]))
     assert a - b >= 4 * params                     # momentum adds one fp32 copy
-    assert b >= 8 * params + 2 * ring              # master + G + bf16 ring
-    assert b < 8 * params + 2 * ring + (1 << 28)   # and little else
+    assert b >= 4 * params + 2 * ring              # fp32 master + bf16 ring
+    assert b < 4 * params + 2 * ring + (1 << 29)   # stashes and split-K partials are small beside them
+    c = lpb.lp_workspace_size(wl["layers"], wl["stages"], None, wl["delays"], wl["batch"],
+                              flags=lpb.LP_CAPTURE_GRADS)
+    assert c - b >= 4 * params                     # keeping G costs one more fp32 copy
 
 
 def test_bad_arguments_are_rejected():
@@ -90,4 +93,4 @@ def test_bad_arguments_are_rejected():
     assert lib.lp_step(None, None, None, None) == lpb.LP_ERR_INVALID_ARG
     assert lib.lp_destroy(None) == lpb.LP_ERR_INVALID_ARG
     assert lib.lp_gemm_bf16(3, 1, 1, 1, None, 8, None, 8, None, 4, None) == lpb.LP_ERR_INVALID_ARG
-    assert lib.lp_set_tuning(100, 0) == lpb.LP_ERR_INVALID_ARG
+    assert lib.lp_set_tuning(100, 0, 0) == lpb.LP_ERR_INVALID_ARG

@@ -17,14 +17,15 @@ from gpu_common import assert_bf16_close, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None):
+def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None, fused=True):
     from oracle import layerpipe_oracle as O
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
     W0, b0 = I.initial_weights(layers, 0)
     rng = np.random.default_rng(5)
     b0 = [rng.standard_normal(b.shape).astype(np.float32) * 0.1 for b in b0]   # exercise the bias path
-    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, W0=W0, b0=b0)
+    flags = lpb.LP_CAPTURE_GRADS | (0 if fused else lpb.LP_UNFUSED_UPDATE)
+    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, flags=flags, W0=W0, b0=b0)
     delays = tr.get_schedule()[1]
     orc = O.DelayedGradientTrainer(layers, delays, lr, mu, W0, b0, mirror=True, dtype=np.float32)
     L = len(layers)
@@ -78,17 +79,18 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                 tr.debug_run_task("delta", l, n)
                 note("delta", assert_bf16_close(tr.debug_read("delta", l - 1, n), rec["delta"][l - 1],
                                                 "delta^%d step %d" % (l - 1, n)))
-            tr.debug_run_task("G", l, n)
-            r = rel_l2(tr.debug_read("grad_w", l, 0), rec["dW"][l])
-            assert r < 2e-5, ("G", l, n, r)
-            note("G", r)
-            # update task from the oracle's pre-update state and the oracle's gradient
+            # pre-update state of the oracle; with the fused update the G kernel itself applies Eq. 6
             tr.debug_write("master_w", l, 0, pre_W[l])
             tr.debug_write("master_b", l, 0, pre_b[l])
             if mu != 0.0:
                 tr.debug_write("mom_w", l, 0, pre_mW[l])
                 tr.debug_write("mom_b", l, 0, pre_mb[l])
-            tr.debug_write("grad_w", l, 0, rec["dW"][l])
+            tr.debug_run_task("G", l, n)
+            r = rel_l2(tr.debug_read("grad_w", l, 0), rec["dW"][l])
+            assert r < 2e-5, ("G", l, n, r)
+            note("G", r)
+            if not fused:
+                tr.debug_write("grad_w", l, 0, rec["dW"][l])      # Eq. 6 from the oracle's gradient
             tr.debug_run_task("update", l, n)
             r = rel_l2(tr.debug_read("grad_b", l, 0), rec["db"][l])
             assert r < 2e-5, ("db", l, n, r)
@@ -124,6 +126,28 @@ def test_tasks_gelu_momentum_ragged_sizes():
     layers = I.mlp([200, 328, 130, 257, 75], "gelu")
     w = run_teacher_forced(layers, 72, 4, [3, 2, 1, 0], 0.05, 0.9, 6)
     print("worst per-task errors", w)
+
+
+def test_tasks_unfused_update_path():
+    """LP_UNFUSED_UPDATE: G is written to memory and Eq. 6 runs as its own kernel."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([200, 328, 130, 75], "gelu")
+    run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.9, 5, fused=False)
+    run_teacher_forced(I.mlp([96, 160, 24], "relu"), 40, 2, [1, 0], 0.05, 0.0, 4, fused=False)
+
+
+def test_tasks_split_k_forward_and_delta():
+    """Forced split-K (3 and 8 splits, more splits than k-blocks in some layers): partial tiles
+    reduced in split order by the last CTA of each tile."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([520, 328, 200, 75], "gelu")
+    for sk in (3, 8):
+        lpb.lp_set_tuning(0, 0, sk)
+        try:
+            run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.9, 4)
+        finally:
+            lpb.lp_set_tuning(0, 0, 0)
 
 
 def test_tasks_papers_double_delay_convention():

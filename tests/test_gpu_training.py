@@ -22,12 +22,13 @@ from gpu_common import rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def free_run(layers, batch, stages, delays, lr, mu, steps, schedule, grads_every=1):
+def free_run(layers, batch, stages, delays, lr, mu, steps, schedule, grads_every=1, extra_flags=0):
     import torch
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
     W0, b0 = I.initial_weights(layers, 0)
-    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, schedule=schedule, W0=W0, b0=b0)
+    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, schedule=schedule,
+                     flags=lpb.LP_CAPTURE_GRADS | extra_flags, W0=W0, b0=b0)
     out = dict(schedule=tr.get_schedule(), vlog=[], loss=[], grads={})
     for n in range(steps):
         x, y = I.minibatch(layers, batch, n)
@@ -126,13 +127,29 @@ def test_free_running_mlp8_4096_full_size():
             grad_bound=5 * rounding_noise(8), step0_bound=1.5 * rounding_noise(8))
 
 
+def test_fused_and_unfused_update_agree():
+    """The fused epilogue and the separate update kernel evaluate the same expressions on the
+    same fp32 accumulators: the two trajectories must be bit-identical."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 40], "gelu")
+    a, _, _ = free_run(layers, 56, 3, [2, 1, 0], 0.02, 0.9, 8, lpb.LP_SCHED_LAYERPIPE)
+    b, _, _ = free_run(layers, 56, 3, [2, 1, 0], 0.02, 0.9, 8, lpb.LP_SCHED_LAYERPIPE,
+                       extra_flags=lpb.LP_UNFUSED_UPDATE)
+    for l in range(len(layers)):
+        assert np.array_equal(a["W"][l][0], b["W"][l][0]) and np.array_equal(a["W"][l][1], b["W"][l][1])
+        for n in a["grads"]:
+            assert np.array_equal(a["grads"][n][l][0], b["grads"][n][l][0])
+    assert a["loss"] == b["loss"]
+
+
 def test_step_rejects_bad_arguments_without_side_effects():
     import torch
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
     layers = I.mlp([64, 32, 16], "relu")
     W0, b0 = I.initial_weights(layers, 0)
-    tr = lpb.Trainer(layers, 8, 2, W0=W0, b0=b0)
+    tr = lpb.Trainer(layers, 8, 2, flags=lpb.LP_CAPTURE_GRADS, W0=W0, b0=b0)
     lib = lpb.lib()
     assert lib.lp_step(tr.h, None, None, None) == lpb.LP_ERR_INVALID_ARG
     assert tr.kernel_launches() == 0
