@@ -162,10 +162,13 @@ int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* d
  *   LP_BUF_RING_W     [out][in]  bf16 weight version                     ring slot
  *   LP_BUF_RING_B     [out]      fp32 bias version                       ring slot
  *   LP_BUF_MASTER_W/B, LP_BUF_MOM_W/B, LP_BUF_GRAD_W/B   [out][in] / [out]   (index ignored)
+ *   LP_BUF_POOL_IDX   [pooled pixels][channels]  position 0..3 of the maximum in its 2x2 window   minibatch
+ * For convolution layers "batch" rows become batch*H*W pixel rows (NHWC) and [out][in] becomes
+ * [Cout][R][S][Cin].
  */
 enum { LP_BUF_INPUT = 0, LP_BUF_Z = 1, LP_BUF_DELTA = 2, LP_BUF_LOGITS = 3, LP_BUF_LABELS = 4, LP_BUF_LOSS = 5,
        LP_BUF_RING_W = 6, LP_BUF_RING_B = 7, LP_BUF_MASTER_W = 8, LP_BUF_MASTER_B = 9, LP_BUF_MOM_W = 10,
-       LP_BUF_MOM_B = 11, LP_BUF_GRAD_W = 12, LP_BUF_GRAD_B = 13 };
+       LP_BUF_MOM_B = 11, LP_BUF_GRAD_W = 12, LP_BUF_GRAD_B = 13, LP_BUF_POOL_IDX = 14 };
 int lp_debug_read(lp_handle h, int buffer, int layer, long long index, float* out_host);
 int lp_debug_write(lp_handle h, int buffer, int layer, long long index, const float* in_host);
 

@@ -308,7 +308,7 @@ class DelayedGradientTrainer:
         self.n = n + 1
         rec["dW"], rec["db"] = dW, db
         if capture:
-            rec["a"], rec["zs"], rec["delta"], rec["zL"] = a, zs, deltas, zL
+            rec["a"], rec["zs"], rec["delta"], rec["zL"], rec["amax"] = a, zs, deltas, zL, amax
         return rec
 
     def weights(self):

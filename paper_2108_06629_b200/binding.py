@@ -231,16 +231,25 @@ class Trainer:
 
     # ---- verification access (see the header: lp_debug_*) -------------------
     BUF = {"input": 0, "z": 1, "delta": 2, "logits": 3, "labels": 4, "loss": 5, "ring_w": 6, "ring_b": 7,
-           "master_w": 8, "master_b": 9, "mom_w": 10, "mom_b": 11, "grad_w": 12, "grad_b": 13}
+           "master_w": 8, "master_b": 9, "mom_w": 10, "mom_b": 11, "grad_w": 12, "grad_b": 13, "pool_idx": 14}
     TASK = {"forward": 0, "loss": 1, "delta": 2, "G": 3, "update": 4}
 
     def _buf_shape(self, buf, layer):
         l = self.layers[layer]
         classes = self.layers[-1]["n_out"]
-        return {"input": (self.batch, l["n_in"]), "z": (self.batch, l["n_out"]), "delta": (self.batch, l["n_out"]),
-                "logits": (self.batch, classes), "labels": (self.batch,), "loss": (1,),
-                "ring_w": (l["n_out"], l["n_in"]), "master_w": (l["n_out"], l["n_in"]),
-                "mom_w": (l["n_out"], l["n_in"]), "grad_w": (l["n_out"], l["n_in"])}.get(buf, (l["n_out"],))
+        B = self.batch
+        if l["kind"] == "conv":
+            H, W = l["H"], l["W"]
+            Hp, Wp = (H // 2, W // 2) if l.get("pool", 0) else (H, W)
+            wshape = (l["n_out"], l["R"], l["S"], l["n_in"])
+            shapes = {"input": (B, H, W, l["n_in"]), "delta": (B, H, W, l["n_out"]),
+                      "pool_idx": (B, Hp, Wp, l["n_out"])}
+        else:
+            wshape = (l["n_out"], l["n_in"])
+            shapes = {"input": (B, l["n_in"]), "z": (B, l["n_out"]), "delta": (B, l["n_out"])}
+        shapes.update({"logits": (B, classes), "labels": (B,), "loss": (1,), "ring_w": wshape, "master_w": wshape,
+                       "mom_w": wshape, "grad_w": wshape})
+        return shapes.get(buf, (l["n_out"],))
 
     def debug_read(self, buf, layer, index):
         out = np.empty(self._buf_shape(buf, layer), dtype=np.float32)

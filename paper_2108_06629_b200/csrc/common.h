@@ -19,6 +19,9 @@ namespace lp {
 int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                       uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer, std::string* err);
 
+int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
+                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err);
+
 struct GemmArgs;
 // which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
 // Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
@@ -44,7 +47,7 @@ int plan_layers(const lp_layer* layers, int L, int batch, int Np, PlanResult* ou
 
 // ---- elementwise.cu ---------------------------------------------------------
 cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
-                              int* labels_copy, int B, int n_in, int ld, cudaStream_t stream);
+                              int* labels_copy, int rows, int B, int n_in, int ld, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
                                 cudaStream_t stream);
@@ -56,6 +59,8 @@ struct UpdateArgs {
   long long n_elems;    // out * ldw (multiple of 8)
   const __nv_bfloat16* delta;  // [rows][ldd]: bias gradient = column sums (null: no bias)
   int rows, ldd, n_out;
+  const float* col_partial;    // if set: [chunks][n_out] partial column sums to add instead of delta
+  int n_chunks;
   float* b;             // master bias
   float* mb;            // bias momentum or null
   float* db;            // bias gradient out
@@ -63,6 +68,15 @@ struct UpdateArgs {
   float lr, mu;
 };
 cudaError_t launch_sgd_update(const UpdateArgs& a, cudaStream_t stream);
+// 2x2 stride-2 max pool of an NHWC bf16 tensor (C a multiple of 8); idx = position of the first
+// maximum in (dh, dw) row-major order.
+cudaError_t launch_maxpool2(const __nv_bfloat16* a, __nv_bfloat16* pooled, unsigned char* idx, int B, int H, int W,
+                            int C, cudaStream_t stream);
+// Column sums of a [rows][ld] bf16 matrix in two deterministic passes: partial[chunk][col] over
+// chunks of kColsumChunk rows, then (inside launch_sgd_update) the chunks in order.
+constexpr int kColsumChunk = 2048;
+cudaError_t launch_colsum_partial(const __nv_bfloat16* x, int rows, int ld, int n_cols, float* partial,
+                                  cudaStream_t stream);
 cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long n_elems, cudaStream_t stream);
 
 }  // namespace lp

@@ -11,9 +11,9 @@ namespace lp {
 // into the library's label ring so that the caller may reuse its buffers.
 __global__ void cast_stash_kernel(const void* __restrict__ batch, int input_is_bf16,
                                   const int* __restrict__ labels, __nv_bfloat16* __restrict__ x0,
-                                  int* __restrict__ labels_copy, int B, int n_in, int ld) {
+                                  int* __restrict__ labels_copy, int rows, int B, int n_in, int ld) {
   const long long groups_per_row = ld / 8;
-  const long long total = (long long)B * groups_per_row;
+  const long long total = (long long)rows * groups_per_row;
   for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < total;
        g += (long long)gridDim.x * blockDim.x) {
     const int row = int(g / groups_per_row);
@@ -51,11 +51,11 @@ __global__ void cast_stash_kernel(const void* __restrict__ batch, int input_is_b
 }
 
 cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
-                              int* labels_copy, int B, int n_in, int ld, cudaStream_t stream) {
-  const long long total = (long long)B * (ld / 8);
+                              int* labels_copy, int rows, int B, int n_in, int ld, cudaStream_t stream) {
+  const long long total = (long long)rows * (ld / 8);
   int blocks = int(std::min<long long>((total + 255) / 256, 148 * 8));
   if (blocks < 1) blocks = 1;
-  cast_stash_kernel<<<blocks, 256, 0, stream>>>(batch, input_is_bf16, labels, x0, labels_copy, B, n_in, ld);
+  cast_stash_kernel<<<blocks, 256, 0, stream>>>(batch, input_is_bf16, labels, x0, labels_copy, rows, B, n_in, ld);
   return cudaGetLastError();
 }
 
@@ -180,7 +180,12 @@ __global__ void __launch_bounds__(UPD_THREADS) sgd_update_kernel(const UpdateArg
   const int col = cb + tx;
   float acc = 0.f;
   if (col < a.n_out) {
-    for (int r = ty; r < a.rows; r += NY) acc += __bfloat162float(a.delta[(long long)r * a.ldd + col]);
+    if (a.col_partial != nullptr) {
+      if (ty == 0)
+        for (int ch = 0; ch < a.n_chunks; ++ch) acc += a.col_partial[(long long)ch * a.n_out + col];
+    } else {
+      for (int r = ty; r < a.rows; r += NY) acc += __bfloat162float(a.delta[(long long)r * a.ldd + col]);
+    }
   }
   part[ty][tx] = acc;
   __syncthreads();
@@ -230,6 +235,78 @@ cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long
   int blocks = int(std::min<long long>((nvec + 255) / 256, 148 * 16));
   if (blocks < 1) blocks = 1;
   round_to_bf16_kernel<<<blocks, 256, 0, stream>>>(src, dst, nvec);
+  return cudaGetLastError();
+}
+}  // namespace lp
+
+namespace lp {
+// ---------------------------------------------------------------------------
+// 2x2 stride-2 max pool, NHWC, 8 channels (16 bytes) per thread.
+__global__ void maxpool2_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ pooled,
+                                unsigned char* __restrict__ idx, int B, int H, int W, int C) {
+  const int Hp = H / 2, Wp = W / 2, cg = C / 8;
+  const long long total = (long long)B * Hp * Wp * cg;
+  for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+    const int c8 = int(t % cg);
+    long long pp = t / cg;
+    const int pw = int(pp % Wp);
+    const int ph = int((pp / Wp) % Hp);
+    const int n = int(pp / ((long long)Wp * Hp));
+    float best[8];
+    unsigned char bi[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const long long src = (((long long)n * H + 2 * ph + (k >> 1)) * W + 2 * pw + (k & 1)) * C + c8 * 8;
+      const uint4 v = *reinterpret_cast<const uint4*>(a + src);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
+        if (k == 0 || lo > best[2 * j]) { best[2 * j] = lo; bi[2 * j] = (unsigned char)k; }
+        if (k == 0 || hi > best[2 * j + 1]) { best[2 * j + 1] = hi; bi[2 * j + 1] = (unsigned char)k; }
+      }
+    }
+    uint4 o;
+    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      ow[j] = (__float_as_uint(best[2 * j]) >> 16) | (__float_as_uint(best[2 * j + 1]) & 0xFFFF0000u);
+    const long long dst = pp * C + c8 * 8;
+    *reinterpret_cast<uint4*>(pooled + dst) = o;
+    uint2 ib;
+    ib.x = bi[0] | (bi[1] << 8) | (bi[2] << 16) | (bi[3] << 24);
+    ib.y = bi[4] | (bi[5] << 8) | (bi[6] << 16) | (bi[7] << 24);
+    *reinterpret_cast<uint2*>(idx + dst) = ib;
+  }
+}
+cudaError_t launch_maxpool2(const __nv_bfloat16* a, __nv_bfloat16* pooled, unsigned char* idx, int B, int H, int W,
+                            int C, cudaStream_t stream) {
+  const long long total = (long long)B * (H / 2) * (W / 2) * (C / 8);
+  int blocks = int(std::min<long long>((total + 255) / 256, 148 * 16));
+  if (blocks < 1) blocks = 1;
+  maxpool2_kernel<<<blocks, 256, 0, stream>>>(a, pooled, idx, B, H, W, C);
+  return cudaGetLastError();
+}
+
+// partial[chunk][col] = sum over the chunk's rows (in row order, 4-way interleaved like the
+// single-pass bias reduction) of x[row][col]
+__global__ void colsum_partial_kernel(const __nv_bfloat16* __restrict__ x, int rows, int ld, int n_cols,
+                                      float* __restrict__ partial) {
+  __shared__ float part[4][64];
+  const int tx = threadIdx.x % 64, ty = threadIdx.x / 64;
+  const int col = blockIdx.x * 64 + tx;
+  const int r0 = blockIdx.y * kColsumChunk, r1 = min(rows, r0 + kColsumChunk);
+  float acc = 0.f;
+  if (col < n_cols)
+    for (int r = r0 + ty; r < r1; r += 4) acc += __bfloat162float(x[(long long)r * ld + col]);
+  part[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && col < n_cols) partial[(long long)blockIdx.y * n_cols + col] = part[0][tx] + part[1][tx] + part[2][tx] + part[3][tx];
+}
+cudaError_t launch_colsum_partial(const __nv_bfloat16* x, int rows, int ld, int n_cols, float* partial,
+                                  cudaStream_t stream) {
+  dim3 grid((n_cols + 63) / 64, (rows + kColsumChunk - 1) / kColsumChunk);
+  colsum_partial_kernel<<<grid, 256, 0, stream>>>(x, rows, ld, n_cols, partial);
   return cudaGetLastError();
 }
 }  // namespace lp

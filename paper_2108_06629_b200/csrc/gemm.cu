@@ -56,6 +56,30 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64
   return LP_OK;
 }
 
+// NHWC bf16 tensor [N][H][W][C] with channel pitch `pitch_c` (multiple of 8): dimensions
+// (C, W, H, N), box (64 channels, bw, bh, bn pixels).  Coordinates outside the tensor read zero.
+int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
+                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err) {
+  EncodeTiledFn fn = get_encode_fn(err);
+  if (!fn) return LP_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch_c & 7) || bw > 256 || bh > 256 || bn > 256) {
+    if (err) *err = "tensor map: base must be 16-byte aligned, channel pitch a multiple of 8, box <= 256";
+    return LP_ERR_INVALID_ARG;
+  }
+  cuuint64_t dims[4] = {C, W, H, N};
+  cuuint64_t strides[3] = {pitch_c * 2, W * pitch_c * 2, H * W * pitch_c * 2};
+  cuuint32_t box[4] = {64, bw, bh, bn};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled (4-D) failed with CUresult " + std::to_string(int(r));
+    return LP_ERR_CUDA;
+  }
+  return LP_OK;
+}
+
 // ---------------------------------------------------------------------------
 static int g_force_bn = 0;
 static int g_force_stages = 0;
@@ -113,12 +137,13 @@ static int pick_stages(int bn, int K) {
 
 template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
-  if (a.splits < 1 || MODE == EPI_WGRAD_UPDATE || a.partial == nullptr) a.splits = 1;
+  if (a.splits < 1 || a.partial == nullptr) a.splits = 1;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
   a.num_stages = pick_stages(BN, a.kb_per_split * GEMM_BK);
   const size_t smem = GemmSmem<BN>::bytes(a.num_stages);
   dim3 grid((a.M + GEMM_BM - 1) / GEMM_BM, (a.N + BN - 1) / BN, a.splits);
+  if (a.g.kind == GEOM_PIX_K) grid.y = unsigned(a.g.n_per_tap) * unsigned(a.N / a.g.tap_pitch);   // (tap, channel block)
   gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a);
   return cudaGetLastError();
 }
@@ -134,6 +159,7 @@ static cudaError_t configure_one() {
   X(BN, false, false, EPI_FPROP)             \
   X(BN, false, false, EPI_STORE_F32)         \
   X(BN, false, true, EPI_DGRAD)              \
+  X(BN, false, true, EPI_DGRAD_UNPOOL)       \
   X(BN, false, true, EPI_STORE_F32)          \
   X(BN, true, true, EPI_STORE_F32)           \
   X(BN, true, true, EPI_WGRAD_UPDATE)

@@ -4,7 +4,8 @@
 //
 //   warp 0      TMA producer (one elected lane)
 //   warp 1      tensor-memory allocation + MMA issue (one elected lane)
-//   warps 2-5   epilogue: tcgen05.ld -> registers -> bias / activation / f' -> global
+//   warps 2-5   epilogue: tcgen05.ld -> shared-memory transpose -> bias / activation / f' /
+//               update -> coalesced global accesses
 //
 // Operand "major" follows the tensor-core convention: K-major = the contraction index is
 // contiguous in memory, MN-major = the M (or N) index is contiguous.  With W stored
@@ -13,6 +14,11 @@
 //   delta   (Eq. 4)  A = delta  K-major,  B = W      MN-major
 //   G       (Eq. 5)  A = delta  MN-major, B = a      MN-major
 // so one copy of each tensor serves all three.
+//
+// Convolutions (3x3, stride 1, zero padding 1, NHWC activations, weights [Cout][R][S][Cin]) run
+// through the same kernel as implicit GEMMs: the producer addresses the activation tensor
+// through a 4-D tensor map and shifts the pixel box by the filter tap; coordinates outside
+// the image are zero-filled by TMA, which is the padding.  See ConvGeom.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -26,8 +32,29 @@ constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;   // 16 KiB
 constexpr int GEMM_MAX_STAGES = 8;
 
-enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2, EPI_WGRAD_UPDATE = 3 };
+enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2, EPI_WGRAD_UPDATE = 3, EPI_DGRAD_UNPOOL = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
+
+// How the GEMM indices map onto image pixels.
+//   GEOM_PLAIN   ordinary matrices.
+//   GEOM_PIX_M   forward / delta of a convolution: the 128 rows of a tile are a box of
+//                bw x bh x bn pixels (w fastest) of an NHWC tensor; the contraction runs over
+//                (filter tap, 64-channel chunk); the A box is shifted by the tap.
+//   GEOM_PIX_K   G of a convolution: rows = output channels, columns = (tap, input channel),
+//                the contraction runs over boxes of 64 pixels; the B box (activations) is
+//                shifted by the tap of the column tile.
+enum { GEOM_PLAIN = 0, GEOM_PIX_M = 1, GEOM_PIX_K = 2 };
+struct ConvGeom {
+  int kind;
+  int H, W;              // image size of the pixel tensor
+  int lw, lh;            // log2 of the box width / height; images per box = box pixels >> (lw + lh)
+  int tiles_w, tiles_h;  // boxes per image row / column
+  int S, pad;            // filter width (taps = R*S, tap = r*S + s) and padding
+  int flip;              // 0: pixel shift = tap - pad (forward, G); 1: pad - tap (delta)
+  int chunks_per_tap;    // PIX_M: 64-channel chunks of the A tensor per tap
+  int tap_pitch;         // elements between taps inside a row of the weight matrix (padded Cin)
+  int n_per_tap;         // PIX_K: column tiles per tap
+};
 
 struct GemmArgs {
   int M, N, K;
@@ -48,13 +75,20 @@ struct GemmArgs {
   float* mW;
   __nv_bfloat16* ring;
   float lr, mu;
+  // EPI_DGRAD_UNPOOL: the layer below ended in a 2x2 max pool.  Element (row, col) of the product
+  // belongs to pooled pixel row * pool_ppr + col / pool_C, channel col % pool_C; it is routed to
+  // the window position recorded in pool_idx (and gated by the pooled activation in `aux`),
+  // the other three positions of the window receive zero.
+  const unsigned char* pool_idx;
+  int pool_C, pool_ppr, pool_Hp, pool_Wp;
   // split-K (splits > 1): blockIdx.z owns k-blocks [z*kb_per_split, (z+1)*kb_per_split); every CTA
   // writes its fp32 partial tile to `partial`, the last CTA of a tile to arrive (tile_counter)
   // adds the partials in split order -- a fixed order, so results do not depend on timing --
-  // and runs the epilogue.  Not available with EPI_WGRAD_UPDATE.
+  // and runs the epilogue.
   int splits, kb_per_split;
   float* partial;           // [tiles][splits][128][BN]
   unsigned* tile_counter;   // [tiles], zero between launches
+  ConvGeom g;
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -73,17 +107,34 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 
-
 constexpr int EPI_PITCH = 36;                       // floats; 32 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_TILE_BYTES = 4 * 32 * EPI_PITCH * 4;   // one 32 x 32 staging tile per epilogue warp (18 KiB)
 static_assert(EPI_TILE_BYTES <= GEMM_A_BYTES + 64 * GEMM_BK * 2, "staging tiles must fit in one pipeline stage");
 
-// Epilogue for 4 consecutive columns n..n+3 of output row `row`.  Lanes past N inside the
-// last 16-byte (fp32) / 8-element (bf16) group are written as zeros; groups that start
-// beyond that are skipped.
+// Where a tile's rows and columns live in the output.
+struct TileMap {
+  int m0, n0;         // first global row / column (plain)
+  int nlim;           // columns >= nlim do not exist
+  int pn0, ph0, pw0;  // GEOM_PIX_M: first image / row / column of the pixel box
+};
+// Global row index of tile row `tr` (0..127), or -1 if the row does not exist.
+__device__ __forceinline__ int tile_row(const GemmArgs& p, const TileMap& t, int tr) {
+  if (p.g.kind != GEOM_PIX_M) {
+    const int row = t.m0 + tr;
+    return row < p.M ? row : -1;
+  }
+  const int w = t.pw0 + (tr & ((1 << p.g.lw) - 1));
+  const int h = t.ph0 + ((tr >> p.g.lw) & ((1 << p.g.lh) - 1));
+  const int n = t.pn0 + (tr >> (p.g.lw + p.g.lh));
+  const int row = (n * p.g.H + h) * p.g.W + w;
+  return row < p.M ? row : -1;
+}
+
+// Epilogue for 4 consecutive columns n..n+3 of output row `row`.  Lanes past the column limit
+// inside the last 16-byte (fp32) / 8-element (bf16) group are written as zeros; groups that
+// start beyond that are skipped.
 template <int MODE>
-__device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int n, float4 acc) {
-  const int N = p.N;
+__device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int n, int N, float4 acc) {
   float v[4] = {n + 0 < N ? acc.x : 0.f, n + 1 < N ? acc.y : 0.f, n + 2 < N ? acc.z : 0.f, n + 3 < N ? acc.w : 0.f};
   const int n_pad4 = (N + 3) & ~3, n_pad8 = (N + 7) & ~7;
   if (MODE == EPI_STORE_F32) {
@@ -126,10 +177,46 @@ __device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int 
     }
     *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
         make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+  } else if (MODE == EPI_DGRAD_UNPOOL) {
+    // the layer below ended in ReLU + 2x2 max pool: route the gradient to the recorded maximum
+    if (n >= N) return;
+    const int C = p.pool_C;
+    const int pp = row * p.pool_ppr + n / C;     // pooled pixel
+    const int c = n % C;
+    const int pw = pp % p.pool_Wp;
+    const int ph = (pp / p.pool_Wp) % p.pool_Hp;
+    const int pn = pp / (p.pool_Wp * p.pool_Hp);
+    const uint32_t idx = *reinterpret_cast<const uint32_t*>(p.pool_idx + size_t(pp) * C + c);
+    const uint2 av = *reinterpret_cast<const uint2*>(p.aux + size_t(pp) * p.ld_aux + c);
+    const float a[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
+    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int oh = 2 * ph + (k >> 1), ow = 2 * pw + (k & 1);
+      float d[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) d[j] = (((idx >> (8 * j)) & 0xFFu) == uint32_t(k) && a[j] > 0.f) ? v[j] : 0.f;
+      const size_t off = (size_t(pn * 2 * p.pool_Hp + oh) * (2 * p.pool_Wp) + ow) * p.ld_out + c;
+      *reinterpret_cast<uint2*>(o + off) = make_uint2(pack_bf16x2(d[0], d[1]), pack_bf16x2(d[2], d[3]));
+    }
+  } else {  // EPI_WGRAD_UPDATE (plain form, used after a split-K reduction)
+    if (n >= n_pad8) return;
+    const size_t off = size_t(row) * p.ld_out + n;
+    if (p.out != nullptr) __stcs(reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off), make_float4(v[0], v[1], v[2], v[3]));
+    float4 w = __ldcs(reinterpret_cast<const float4*>(p.W + off));
+    float m[4] = {v[0], v[1], v[2], v[3]};
+    if (p.mW != nullptr) {
+      const float4 pm = __ldcs(reinterpret_cast<const float4*>(p.mW + off));
+      m[0] = p.mu * pm.x + v[0]; m[1] = p.mu * pm.y + v[1]; m[2] = p.mu * pm.z + v[2]; m[3] = p.mu * pm.w + v[3];
+      __stcs(reinterpret_cast<float4*>(p.mW + off), make_float4(m[0], m[1], m[2], m[3]));
+    }
+    w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
+    __stcs(reinterpret_cast<float4*>(p.W + off), w);
+    *reinterpret_cast<uint2*>(p.ring + off) = make_uint2(pack_bf16x2(w.x, w.y), pack_bf16x2(w.z, w.w));
   }
 }
 
-// ---- fused G + update epilogue (EPI_WGRAD_UPDATE) -------------------------------------------
+// ---- fused G + update epilogue (EPI_WGRAD_UPDATE, no split-K) -------------------------------
 // The accumulator chunk is G; the epilogue streams the fp32 master (and momentum) tile through
 // registers: m <- mu m + G; W <- W - eta m; ring <- RN(W).  It is an HBM-streaming loop with
 // few warps, so the loads of the NEXT 32 x 32 chunk are issued before the current chunk is
@@ -138,8 +225,8 @@ struct WmRegs {
   float4 w[8];
   float4 m[8];
 };
-__device__ __forceinline__ void load_wm(const GemmArgs& p, int row0, int n, int sub_row, WmRegs& r) {
-  const bool col_ok = n < ((p.N + 7) & ~7);
+__device__ __forceinline__ void load_wm(const GemmArgs& p, int row0, int n, int nlim, int sub_row, WmRegs& r) {
+  const bool col_ok = n < ((nlim + 7) & ~7);
 #pragma unroll
   for (int it = 0; it < 8; ++it) {
     const int row = row0 + it * 4 + sub_row;
@@ -149,16 +236,16 @@ __device__ __forceinline__ void load_wm(const GemmArgs& p, int row0, int n, int 
     if (p.mW != nullptr) r.m[it] = ok ? __ldcs(reinterpret_cast<const float4*>(p.mW + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
 }
-__device__ __forceinline__ void apply_update(const GemmArgs& p, int row0, int n, int sub_row, const float* tile,
-                                             int sub_col, const WmRegs& r) {
-  if (n >= ((p.N + 7) & ~7)) return;
+__device__ __forceinline__ void apply_update(const GemmArgs& p, int row0, int n, int nlim, int sub_row,
+                                             const float* tile, int sub_col, const WmRegs& r) {
+  if (n >= ((nlim + 7) & ~7)) return;
 #pragma unroll
   for (int it = 0; it < 8; ++it) {
     const int rr = it * 4 + sub_row;
     const int row = row0 + rr;
     if (row >= p.M) continue;
     const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
-    float g[4] = {n + 0 < p.N ? acc.x : 0.f, n + 1 < p.N ? acc.y : 0.f, n + 2 < p.N ? acc.z : 0.f, n + 3 < p.N ? acc.w : 0.f};
+    float g[4] = {n + 0 < nlim ? acc.x : 0.f, n + 1 < nlim ? acc.y : 0.f, n + 2 < nlim ? acc.z : 0.f, n + 3 < nlim ? acc.w : 0.f};
     const size_t off = size_t(row) * p.ld_out + n;
     if (p.out != nullptr) __stcs(reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off), make_float4(g[0], g[1], g[2], g[3]));
     float m[4] = {g[0], g[1], g[2], g[3]};
@@ -199,11 +286,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * GEMM_BM;
-  const int n0 = blockIdx.y * BN;
   const int num_kb_total = (p.K + GEMM_BK - 1) / GEMM_BK;
   const int kb_begin = (p.splits > 1) ? int(blockIdx.z) * p.kb_per_split : 0;
   const int num_kb = (p.splits > 1) ? max(0, min(num_kb_total, kb_begin + p.kb_per_split) - kb_begin) : num_kb_total;
+
+  // ---- where this tile sits -----------------------------------------------------------------
+  TileMap tm;
+  tm.m0 = blockIdx.x * GEMM_BM;
+  tm.n0 = blockIdx.y * BN;
+  tm.nlim = p.N;
+  tm.pn0 = tm.ph0 = tm.pw0 = 0;
+  int tap = 0, col0 = tm.n0;      // GEOM_PIX_K: filter tap and first input channel of this column tile
+  if (p.g.kind == GEOM_PIX_M) {
+    const int mt = blockIdx.x;
+    const int tw = mt % p.g.tiles_w, th = (mt / p.g.tiles_w) % p.g.tiles_h, tn = mt / (p.g.tiles_w * p.g.tiles_h);
+    tm.pw0 = tw << p.g.lw;
+    tm.ph0 = th << p.g.lh;
+    tm.pn0 = tn * (GEMM_BM >> (p.g.lw + p.g.lh));
+  } else if (p.g.kind == GEOM_PIX_K) {
+    tap = blockIdx.y / p.g.n_per_tap;
+    col0 = (blockIdx.y % p.g.n_per_tap) * BN;
+    tm.n0 = tap * p.g.tap_pitch + col0;
+    tm.nlim = tap * p.g.tap_pitch + p.g.tap_pitch;     // columns of the next tap belong to another tile
+  }
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
@@ -235,25 +340,69 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t smem0 = smem_u32(smem);
       const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
       uint32_t s = 0, ph = 0;
-      int k0 = kb_begin * GEMM_BK;
-      for (int kb = 0; kb < num_kb; ++kb, k0 += GEMM_BK) {
+      // running position of the contraction
+      int k0 = kb_begin * GEMM_BK;                       // plain: element offset along K
+      int c_tap = 0, c_chunk = 0;                        // PIX_M: filter tap, 64-channel chunk
+      int bw0 = 0, bh0 = 0, bn0 = 0;                     // PIX_K: pixel box of this k-block
+      int dh = 0, dw = 0;                                // PIX_K: pixel shift of this tile's tap
+      if (p.g.kind == GEOM_PIX_M) {
+        c_tap = kb_begin / p.g.chunks_per_tap;
+        c_chunk = kb_begin % p.g.chunks_per_tap;
+      } else if (p.g.kind == GEOM_PIX_K) {
+        const int tw = kb_begin % p.g.tiles_w, th = (kb_begin / p.g.tiles_w) % p.g.tiles_h;
+        bw0 = tw << p.g.lw;
+        bh0 = th << p.g.lh;
+        bn0 = (kb_begin / (p.g.tiles_w * p.g.tiles_h)) * (GEMM_BK >> (p.g.lw + p.g.lh));
+        dh = tap / p.g.S - p.g.pad;
+        dw = tap % p.g.S - p.g.pad;
+      }
+      for (int kb = 0; kb < num_kb; ++kb) {
         ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
         if (!ok) break;
         const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
         const uint32_t sb = sa + GEMM_A_BYTES;
         const uint32_t fb = full0 + 8u * s;
         mbar_arrive_expect_tx_addr(fb, SM::STAGE_BYTES);
-        if (A_MN) {
+        if (p.g.kind == GEOM_PLAIN) {
+          if (A_MN) {
 #pragma unroll
-          for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d_addr(sa + c * 8192, &tmA, fb, m0 + c * 64, k0);
-        } else {
-          tma_load_2d_addr(sa, &tmA, fb, k0, m0);
-        }
-        if (B_MN) {
+            for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, k0);
+          } else {
+            tma_load_2d_addr(sa, &tmA, fb, k0, tm.m0);
+          }
+          if (B_MN) {
 #pragma unroll
-          for (int c = 0; c < BN / 64; ++c) tma_load_2d_addr(sb + c * 8192, &tmB, fb, n0 + c * 64, k0);
+            for (int c = 0; c < BN / 64; ++c) tma_load_2d_addr(sb + c * 8192, &tmB, fb, tm.n0 + c * 64, k0);
+          } else {
+            tma_load_2d_addr(sb, &tmB, fb, k0, tm.n0);
+          }
+          k0 += GEMM_BK;
+        } else if (p.g.kind == GEOM_PIX_M) {
+          // A: 128 pixels x 64 channels of the activation / delta tensor, shifted by the tap
+          const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
+          const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
+          const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;
+          tma_load_4d_addr(sa, &tmA, fb, c_chunk * 64, tm.pw0 + sw, tm.ph0 + sh, tm.pn0);
+          if (B_MN) {   // delta: B[k = (tap, co)][n = ci]: rows co, columns tap*pitch + ci
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c)
+              tma_load_2d_addr(sb + c * 8192, &tmB, fb, c_tap * p.g.tap_pitch + tm.n0 + c * 64, c_chunk * 64);
+          } else {      // forward: B[n = co][k = (tap, ci)]
+            tma_load_2d_addr(sb, &tmB, fb, c_tap * p.g.tap_pitch + c_chunk * 64, tm.n0);
+          }
+          if (++c_chunk == p.g.chunks_per_tap) { c_chunk = 0; ++c_tap; }
         } else {
-          tma_load_2d_addr(sb, &tmB, fb, k0, n0);
+          // G: A = delta (64 pixels x 128 output channels), B = activations shifted by the tap
+#pragma unroll
+          for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_4d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, bw0, bh0, bn0);
+#pragma unroll
+          for (int c = 0; c < BN / 64; ++c) tma_load_4d_addr(sb + c * 8192, &tmB, fb, col0 + c * 64, bw0 + dw, bh0 + dh, bn0);
+          bw0 += 1 << p.g.lw;
+          if (bw0 >= p.g.W) {
+            bw0 = 0;
+            bh0 += 1 << p.g.lh;
+            if (bh0 >= p.g.H) { bh0 = 0; bn0 += GEMM_BK >> (p.g.lw + p.g.lh); }
+          }
         }
         issued = kb + 1;
         if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
@@ -312,15 +461,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     float* tile = epi_tile + q * (32 * EPI_PITCH);
     const int sub_row = lane >> 3;        // 0..3
     const int sub_col = (lane & 7) * 4;   // 0,4,..,28
-    const int row0 = m0 + q * 32;
+    const int row0 = tm.m0 + q * 32;
+    const bool split = p.splits > 1;
     constexpr bool upd = (MODE == EPI_WGRAD_UPDATE);
     WmRegs cur;
-    if constexpr (upd) load_wm(p, row0, n0 + sub_col, sub_row, cur);      // in flight while the main loop runs
+    if constexpr (upd) {
+      if (!split) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
+    }
     bool ok = mbar_wait(acc_bar, 0);
     ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
     if (!ok && lane == 0) atomicExch(p.status, 3);
     tc_fence_after();
-    const bool split = (!upd) && p.splits > 1;
     const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
     float* part = split ? p.partial + (size_t(tile_id) * p.splits + blockIdx.z) * (size_t(GEMM_BM) * BN) : nullptr;
     if (ok) {
@@ -328,29 +479,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         __syncwarp();
-        tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
-        tmem_ld_wait();
+        if (num_kb > 0) {
+          tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = 0u;     // a split without k-blocks contributes zero
+        }
 #pragma unroll
         for (int g = 0; g < 8; ++g)
           *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
         __syncwarp();
-        const int n = n0 + c * 32 + sub_col;
-        if constexpr (upd) {
+        const int n = tm.n0 + c * 32 + sub_col;
+        if (split) {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + sub_row;
+            const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
+            __stcg(reinterpret_cast<float4*>(part + size_t(q * 32 + rr) * BN + c * 32 + sub_col), acc);
+          }
+        } else if constexpr (upd) {
           WmRegs nxt;
-          if (c + 1 < BN / 32) load_wm(p, row0, n + 32, sub_row, nxt);
-          apply_update(p, row0, n, sub_row, tile, sub_col, cur);
+          if (c + 1 < BN / 32) load_wm(p, row0, n + 32, tm.nlim, sub_row, nxt);
+          apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);
           cur = nxt;
         } else {
 #pragma unroll
           for (int it = 0; it < 8; ++it) {
             const int rr = it * 4 + sub_row;
-            const int row = row0 + rr;
+            const int row = tile_row(p, tm, q * 32 + rr);
             const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
-            if (split) {
-              __stcg(reinterpret_cast<float4*>(part + size_t(q * 32 + rr) * BN + c * 32 + sub_col), acc);
-            } else if (row < p.M) {
-              epilogue_store4<MODE>(p, row, n, acc);
-            }
+            if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc);
           }
         }
       }
@@ -371,21 +530,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (*is_last != 0u) {
         const float* base = p.partial + size_t(tile_id) * p.splits * (size_t(GEMM_BM) * BN);
+        const size_t zstride = size_t(GEMM_BM) * BN;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
-          const int n = n0 + c * 32 + sub_col;
-#pragma unroll 2
-          for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + sub_row;
-            const int row = row0 + rr;
-            if (row >= p.M) continue;
-            const float* src = base + size_t(q * 32 + rr) * BN + c * 32 + sub_col;
-            float4 acc = __ldcg(reinterpret_cast<const float4*>(src));
-            for (int z = 1; z < p.splits; ++z) {
-              const float4 t = __ldcg(reinterpret_cast<const float4*>(src + size_t(z) * GEMM_BM * BN));
-              acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+          const int n = tm.n0 + c * 32 + sub_col;
+          // eight independent rows per lane: their loads are issued together for every split,
+          // the additions keep split order
+          float4 acc[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            acc[it] = __ldcg(reinterpret_cast<const float4*>(base + size_t(q * 32 + it * 4 + sub_row) * BN + c * 32 + sub_col));
+          for (int z = 1; z < p.splits; ++z) {
+            float4 t[8];
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+              t[it] = __ldcg(reinterpret_cast<const float4*>(base + z * zstride + size_t(q * 32 + it * 4 + sub_row) * BN + c * 32 + sub_col));
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              acc[it].x += t[it].x; acc[it].y += t[it].y; acc[it].z += t[it].z; acc[it].w += t[it].w;
             }
-            epilogue_store4<MODE>(p, row, n, acc);
+          }
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int row = tile_row(p, tm, q * 32 + it * 4 + sub_row);
+            if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc[it]);
           }
         }
       }

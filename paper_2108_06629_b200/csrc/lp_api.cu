@@ -42,11 +42,33 @@ struct Res {                 // one buffer (or ring slot) the tracker protects
   std::vector<Ev> readers;
 };
 
+struct PixBox {          // box of pixels used as one tile dimension (see ConvGeom)
+  int lw = 0, lh = 0, bw = 1, bh = 1, bn = 1, tiles_w = 1, tiles_h = 1;
+};
+
 struct Layer {
   lp_layer d;
   int stage = 0, delay = 0, slots = 1;
-  int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;
+  int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;   // FC: features; conv: channels (ld = padded to 8)
   int x_slots = 1;
+  // geometry.  FC: H = W = 1, in_rows = out_rows = B.  Conv (3x3, stride 1, pad 1): in_rows =
+  // out_rows = B*H*W; weights are the matrix [Cout][9 * ld_in] (tap-major, padded channels).
+  bool conv = false;
+  int imH = 1, imW = 1, taps = 1;
+  int in_rows = 0, out_rows = 0;
+  int w_rows = 0, w_ld = 0;          // weight matrix [w_rows][w_ld]
+  int pool = 0, Hp = 1, Wp = 1;      // 2x2 max pool after the activation: pooled image size
+  int next_rows = 0;                 // rows of the next layer's input matrix (pooled pixels or B)
+  PixBox box128, box64;              // pixel boxes of 128 (forward / delta) and 64 (G) pixels
+  __nv_bfloat16* a_full = nullptr;   // pool layers: activation before pooling [out_rows][ld_out]
+  unsigned char* pidx = nullptr;     // pool layers: argmax per pooled element, one slot per stash slot of the next layer
+  size_t pidx_elems = 0;
+  float* col_partial = nullptr;      // bias gradient of large layers: partial column sums
+  int col_chunks = 0;
+  int split_g = 1;
+  float* part_g = nullptr;
+  unsigned* cnt_g = nullptr;
+  Res rAfull;
   // device memory (all inside the workspace)
   float *W = nullptr, *mW = nullptr, *b = nullptr, *mb = nullptr, *dW = nullptr, *db = nullptr, *bring = nullptr;
   __nv_bfloat16 *ring = nullptr, *X = nullptr, *Z = nullptr, *delta = nullptr;
@@ -57,7 +79,7 @@ struct Layer {
   float *part_f = nullptr, *part_d = nullptr;   // fp32 partial tiles [tiles][splits][128][BN]
   unsigned *cnt_f = nullptr, *cnt_d = nullptr;  // per-tile arrival counters
   std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
-  std::vector<Res> rX, rZ, rDelta, rRing;
+  std::vector<Res> rX, rZ, rDelta, rRing, rPidx;
   Res rDW;
   Ev last_update;
 };
@@ -116,6 +138,19 @@ static int fail(lp_ctx* h, int code, const std::string& msg) {
       return fail(h, LP_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));         \
   } while (0)
 
+// Factor `pixels` (128 or 64) into a box bw x bh x bn of powers of two with bw | W, bh | H, bn | B,
+// widest in w first (longest contiguous runs).
+static int pick_box(int W, int H, int B, int pixels, PixBox* out) {
+  int bw = 1, lw = 0;
+  while (bw * 2 <= pixels && W % (bw * 2) == 0) { bw *= 2; ++lw; }
+  int bh = 1, lh = 0;
+  while (bw * bh * 2 <= pixels && H % (bh * 2) == 0) { bh *= 2; ++lh; }
+  const int bn = pixels / (bw * bh);
+  if (bn < 1 || B % bn != 0) return LP_ERR_UNSUPPORTED;
+  if (out) { out->lw = lw; out->lh = lh; out->bw = bw; out->bh = bh; out->bn = bn; out->tiles_w = W / bw; out->tiles_h = H / bh; }
+  return LP_OK;
+}
+
 // ---------------------------------------------------------------------------
 static int validate(const lp_layer* layers, int n, const lp_config* cfg, std::string* why) {
   if (!layers || n < 1 || !cfg) { *why = "null layer list or config"; return LP_ERR_INVALID_ARG; }
@@ -128,9 +163,27 @@ static int validate(const lp_layer* layers, int n, const lp_config* cfg, std::st
     if (y.in < 1 || y.out < 1) { *why = "layer sizes must be positive"; return LP_ERR_INVALID_ARG; }
     if (y.act < LP_ACT_NONE || y.act > LP_ACT_GELU) { *why = "unknown activation"; return LP_ERR_INVALID_ARG; }
     if (l == n - 1 && y.act != LP_ACT_NONE) { *why = "last layer must have no activation"; return LP_ERR_INVALID_ARG; }
-    if (y.kind == LP_CONV) { *why = "convolution layers are not built yet"; return LP_ERR_UNSUPPORTED; }
-    if (y.pool != 0) { *why = "pooling needs a convolution layer"; return LP_ERR_INVALID_ARG; }
-    if (l > 0 && layers[l - 1].out != y.in) { *why = "layer sizes do not chain"; return LP_ERR_INVALID_ARG; }
+    if (y.kind == LP_CONV) {
+      if (y.R != 3 || y.S != 3 || y.stride != 1 || y.pad != 1) { *why = "only 3x3 stride-1 pad-1 convolutions are built"; return LP_ERR_UNSUPPORTED; }
+      if (y.H < 1 || y.W < 1) { *why = "bad image size"; return LP_ERR_INVALID_ARG; }
+      if (y.act == LP_ACT_GELU) { *why = "GELU after a convolution is not built"; return LP_ERR_UNSUPPORTED; }
+      if (y.out % 8 != 0) { *why = "convolution output channels must be a multiple of 8"; return LP_ERR_UNSUPPORTED; }
+      if (y.pool != 0 && (y.pool != 2 || y.H % 2 || y.W % 2 || y.act != LP_ACT_RELU)) { *why = "pooling must be 2x2 on even images after ReLU"; return LP_ERR_UNSUPPORTED; }
+      if (l == n - 1) { *why = "the last layer must be fully connected"; return LP_ERR_UNSUPPORTED; }
+      if (pick_box(y.W, y.H, cfg->batch, 128, nullptr) != LP_OK || pick_box(y.W, y.H, cfg->batch, 64, nullptr) != LP_OK) {
+        *why = "image size / batch cannot be tiled into boxes of 128 and 64 pixels"; return LP_ERR_UNSUPPORTED;
+      }
+    } else if (y.pool != 0) { *why = "pooling needs a convolution layer"; return LP_ERR_INVALID_ARG; }
+    if (l > 0) {
+      const lp_layer& pv = layers[l - 1];
+      const int ph = pv.kind == LP_CONV ? pv.H / (pv.pool ? 2 : 1) : 1, pw = pv.kind == LP_CONV ? pv.W / (pv.pool ? 2 : 1) : 1;
+      if (y.kind == LP_CONV) {
+        if (pv.kind != LP_CONV || pv.out != y.in || ph != y.H || pw != y.W) { *why = "layer sizes do not chain"; return LP_ERR_INVALID_ARG; }
+      } else {
+        if ((long long)pv.out * ph * pw != y.in) { *why = "layer sizes do not chain"; return LP_ERR_INVALID_ARG; }
+        if (pv.kind == LP_CONV && pv.act == LP_ACT_GELU) { *why = "GELU after a convolution is not built"; return LP_ERR_UNSUPPORTED; }
+      }
+    }
   }
   return LP_OK;
 }
@@ -182,7 +235,7 @@ static size_t carve(lp_ctx* c, char* base) {
   const int nL = int(c->L.size());
   for (int l = 0; l < nL; ++l) {
     Layer& y = c->L[l];
-    y.w_elems = size_t(y.n_out) * y.ld_in;
+    y.w_elems = size_t(y.w_rows) * y.w_ld;
     y.W = reinterpret_cast<float*>(take(y.w_elems * 4));
     y.mW = mom ? reinterpret_cast<float*>(take(y.w_elems * 4)) : nullptr;
     const bool keep_G = (c->cfg.flags & (LP_CAPTURE_GRADS | LP_UNFUSED_UPDATE)) != 0;
@@ -192,9 +245,9 @@ static size_t carve(lp_ctx* c, char* base) {
     y.mb = mom ? reinterpret_cast<float*>(take(size_t(y.ld_out) * 4)) : nullptr;
     y.db = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4));
     y.bring = reinterpret_cast<float*>(take(size_t(y.ld_out) * 4 * y.slots));
-    y.x_elems = size_t(B) * y.ld_in;
+    y.x_elems = size_t(y.in_rows) * y.ld_in;
     y.X = reinterpret_cast<__nv_bfloat16*>(take(y.x_elems * 2 * y.x_slots));
-    y.delta_elems = size_t(B) * y.ld_out;
+    y.delta_elems = size_t(y.out_rows) * y.ld_out;
     y.delta = reinterpret_cast<__nv_bfloat16*>(take(y.delta_elems * 2 * kDeltaSlots));
     y.z_slots = 0;
     y.Z = nullptr;
@@ -203,6 +256,12 @@ static size_t carve(lp_ctx* c, char* base) {
       y.z_elems = size_t(B) * y.ld_out;
       y.Z = reinterpret_cast<__nv_bfloat16*>(take(y.z_elems * 2 * y.z_slots));
     }
+    if (y.pool && l + 1 < nL) {
+      y.a_full = reinterpret_cast<__nv_bfloat16*>(take(y.delta_elems * 2));
+      y.pidx_elems = size_t(B) * y.Hp * y.Wp * y.ld_out;
+      y.pidx = reinterpret_cast<unsigned char*>(take(y.pidx_elems * c->L[l + 1].x_slots));
+    }
+    if (y.col_chunks > 0) y.col_partial = reinterpret_cast<float*>(take(size_t(y.col_chunks) * y.ld_out * 4));
     auto tiles_of = [&](int M, int N, int bn) { return size_t((M + GEMM_BM - 1) / GEMM_BM) * ((N + bn - 1) / bn); };
     if (y.split_f > 1) {
       const size_t t = tiles_of(B, y.n_out, y.bn_f);
@@ -213,6 +272,11 @@ static size_t carve(lp_ctx* c, char* base) {
       const size_t t = tiles_of(B, y.n_in, y.bn_d);
       y.part_d = reinterpret_cast<float*>(take(t * y.split_d * GEMM_BM * y.bn_d * 4));
       y.cnt_d = reinterpret_cast<unsigned*>(take(t * 4));
+    }
+    if (y.split_g > 1) {
+      const size_t t = size_t((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
+      y.part_g = reinterpret_cast<float*>(take(t * y.split_g * GEMM_BM * y.bn_g * 4));
+      y.cnt_g = reinterpret_cast<unsigned*>(take(t * 4));
     }
   }
   c->zL = reinterpret_cast<float*>(take(size_t(kDeltaSlots) * B * c->ld_cls * 4));
@@ -239,11 +303,38 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     y.ld_out = pad8(y.n_out);
     y.x_slots = y.delay + 1 + kExtraStashSlots;
     const int B = c->cfg.batch;
-    y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
-    y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
-    y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
-    y.split_f = gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
-    y.split_d = gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
+    y.conv = layers[l].kind == LP_CONV;
+    if (y.conv) {
+      y.imH = layers[l].H; y.imW = layers[l].W; y.taps = 9;
+      y.in_rows = y.out_rows = B * y.imH * y.imW;
+      y.w_rows = y.n_out; y.w_ld = y.taps * y.ld_in;
+      y.pool = layers[l].pool;
+      y.Hp = y.pool ? y.imH / 2 : y.imH; y.Wp = y.pool ? y.imW / 2 : y.imW;
+      y.next_rows = (l + 1 < n && layers[l + 1].kind == LP_CONV) ? B * y.Hp * y.Wp : B;
+      pick_box(y.imW, y.imH, B, 128, &y.box128);
+      pick_box(y.imW, y.imH, B, 64, &y.box64);
+      y.bn_f = y.n_out <= 64 ? 64 : 128;
+      y.bn_d = y.ld_in <= 64 ? 64 : 128;
+      y.bn_g = y.ld_in <= 64 ? 64 : 128;
+      y.split_f = y.split_d = 1;
+      // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: split the
+      // pixel range until about two CTAs per SM exist
+      const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
+      const int num_kb = y.in_rows / GEMM_BK;
+      y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), num_kb / 8), 64));
+      const int per = (num_kb + y.split_g - 1) / y.split_g;
+      y.split_g = (num_kb + per - 1) / per;
+    } else {
+      y.in_rows = y.out_rows = y.next_rows = B;
+      y.w_rows = y.n_out; y.w_ld = y.ld_in;
+      y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
+      y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
+      y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
+      y.split_f = gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
+      y.split_d = gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
+      y.split_g = 1;
+    }
+    y.col_chunks = y.out_rows > 8192 ? (y.out_rows + kColsumChunk - 1) / kColsumChunk : 0;
   }
   c->classes = layers[n - 1].out;
   c->ld_cls = pad8(c->classes);
@@ -296,33 +387,57 @@ static int build_tensor_maps(lp_ctx* c) {
     Layer& y = c->L[l];
     uint32_t bA[2], bB[2];
     int rc;
+    y.tm_f_A.resize(y.x_slots);
+    y.tm_f_B.resize(y.slots);
+    y.tm_d_A.resize(kDeltaSlots);
+    y.tm_d_B.resize(y.slots);
+    y.tm_g_A.resize(kDeltaSlots);
+    y.tm_g_B.resize(y.x_slots);
+    if (y.conv) {
+      // forward: A = a^{l-1} as NHWC boxes of 128 pixels; B = W [Cout][9 * ld_in] K-major
+      // delta:   A = delta^l as NHWC boxes of 128 pixels; B = the same W matrix read MN-major
+      // G:       A = delta^l, B = a^{l-1}, both as NHWC boxes of 64 pixels (the contraction index)
+      for (int s = 0; s < y.x_slots; ++s) {
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_f_A[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, y.box128.bw,
+                                      y.box128.bh, y.box128.bn, &err)) != LP_OK) return fail(c, rc, err);
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_g_B[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, y.box64.bw,
+                                      y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
+      }
+      for (int s = 0; s < kDeltaSlots; ++s) {
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
+                                      y.box128.bw, y.box128.bh, y.box128.bn, &err)) != LP_OK) return fail(c, rc, err);
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
+                                      y.box64.bw, y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
+      }
+      for (int s = 0; s < y.slots; ++s) {
+        if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64, y.bn_f, &err)) != LP_OK)
+          return fail(c, rc, err);
+        if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64, 64, &err)) != LP_OK)
+          return fail(c, rc, err);
+      }
+      continue;
+    }
     // forward: A = a^{l-1} [B][in] K-major; B = W [out][in] K-major
     gemm_box_dims(0, y.bn_f, bA, bB);
-    y.tm_f_A.resize(y.x_slots);
     for (int s = 0; s < y.x_slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_f_A[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
-    y.tm_f_B.resize(y.slots);
     for (int s = 0; s < y.slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
     // delta: A = delta^l [B][out] K-major (K = out); B = W [out][in] MN-major (N = in contiguous)
     gemm_box_dims(1, y.bn_d, bA, bB);
-    y.tm_d_A.resize(kDeltaSlots);
     for (int s = 0; s < kDeltaSlots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
-    y.tm_d_B.resize(y.slots);
     for (int s = 0; s < y.slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
     // G: A = delta^l stored [B][out] -> MN-major (M = out contiguous); B = a^{l-1} stored [B][in] -> MN-major
     gemm_box_dims(2, y.bn_g, bA, bB);
-    y.tm_g_A.resize(kDeltaSlots);
     for (int s = 0; s < kDeltaSlots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
-    y.tm_g_B.resize(y.x_slots);
     for (int s = 0; s < y.x_slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_g_B[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
@@ -366,12 +481,31 @@ struct TimedScope {
 
 // ---------------------------------------------------------------------------
 // the kernels of one minibatch
+static ConvGeom conv_geom(const Layer& y, int kind, const PixBox& bx, int flip, int chunks_per_tap, int n_per_tap) {
+  ConvGeom g{};
+  g.kind = kind;
+  g.H = y.imH; g.W = y.imW;
+  g.lw = bx.lw; g.lh = bx.lh;
+  g.tiles_w = bx.tiles_w; g.tiles_h = bx.tiles_h;
+  g.S = 3; g.pad = 1;
+  g.flip = flip;
+  g.chunks_per_tap = chunks_per_tap;
+  g.tap_pitch = y.ld_in;
+  g.n_per_tap = n_per_tap;
+  return g;
+}
+
 static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
   Layer& y = c->L[l];
   const int nL = int(c->L.size());
   const bool last = (l == nL - 1);
   GemmArgs a{};
-  a.M = c->cfg.batch; a.N = y.n_out; a.K = y.n_in;
+  a.M = y.out_rows; a.N = y.n_out; a.K = y.n_in;
+  if (y.conv) {
+    const int cpt = (y.ld_in + 63) / 64;
+    a.K = y.taps * cpt * GEMM_BK;
+    a.g = conv_geom(y, GEOM_PIX_M, y.box128, 0, cpt, 0);
+  }
   a.mode = EPI_FPROP;
   a.act = y.d.act;
   a.bias = y.d.has_bias ? y.bring + size_t(ring_slot) * y.ld_out : nullptr;
@@ -381,10 +515,13 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
     a.out2 = c->zL + size_t(n % kDeltaSlots) * c->cfg.batch * c->ld_cls;
     a.ld_out2 = c->ld_cls;
     a.out2_is_f32 = 1;
+  } else if (y.pool) {
+    a.out = y.a_full;                 // pooled into the next layer's stash by launch_pool
+    a.ld_out = y.ld_out;
   } else {
     Layer& nx = c->L[l + 1];
     a.out = nx.X + size_t(n % nx.x_slots) * nx.x_elems;
-    a.ld_out = nx.ld_in;
+    a.ld_out = y.ld_out;              // = nx.ld_in for conv -> conv and FC -> FC; a flattened conv output keeps its channel pitch
     if (y.Z) {
       a.out2 = y.Z + size_t(n % y.z_slots) * y.z_elems;
       a.ld_out2 = y.ld_out;
@@ -396,21 +533,53 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
 }
 
+// 2x2 max pool of layer l's activation into the next layer's stash slot (+ argmax)
+static cudaError_t launch_pool(lp_ctx* c, int l, long long n, cudaStream_t st) {
+  Layer& y = c->L[l];
+  Layer& nx = c->L[l + 1];
+  ++c->launches;
+  TimedScope ts(c, LP_TASK_FORWARD, st);
+  return launch_maxpool2(y.a_full, nx.X + size_t(n % nx.x_slots) * nx.x_elems, y.pidx + size_t(n % nx.x_slots) * y.pidx_elems,
+                         c->cfg.batch, y.imH, y.imW, y.ld_out, st);
+}
+
 static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
   Layer& y = c->L[l];
   Layer& pv = c->L[l - 1];
   GemmArgs a{};
-  a.M = c->cfg.batch; a.N = y.n_in; a.K = y.n_out;
-  a.mode = EPI_DGRAD;
+  a.M = y.in_rows; a.N = y.n_in; a.K = y.n_out;
+  if (y.conv) {
+    const int cpt = (y.ld_out + 63) / 64;
+    a.K = y.taps * cpt * GEMM_BK;
+    a.g = conv_geom(y, GEOM_PIX_M, y.box128, 1, cpt, 0);
+  }
   a.act = pv.d.act;
   a.out = pv.delta + size_t(n % kDeltaSlots) * pv.delta_elems;
   a.ld_out = pv.ld_out;
-  if (pv.d.act == LP_ACT_GELU) {
-    a.aux = pv.Z + size_t(n % pv.z_slots) * pv.z_elems;   // stored z^{l-1}
+  if (pv.pool) {
+    // the layer below ended in ReLU + max pool: the product lives on the pooled grid and is
+    // routed back through the recorded argmax, gated by the pooled activation
+    a.mode = EPI_DGRAD_UNPOOL;
+    a.pool_idx = pv.pidx + size_t(n % y.x_slots) * pv.pidx_elems;
+    a.pool_C = pv.ld_out;
+    a.pool_ppr = y.conv ? 1 : pv.Hp * pv.Wp;
+    a.pool_Hp = pv.Hp; a.pool_Wp = pv.Wp;
+    a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;
     a.ld_aux = pv.ld_out;
   } else {
-    a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;      // a^{l-1} > 0  <=>  z^{l-1} > 0
-    a.ld_aux = y.ld_in;
+    a.mode = EPI_DGRAD;
+    if (pv.d.act == LP_ACT_GELU) {
+      a.aux = pv.Z + size_t(n % pv.z_slots) * pv.z_elems;   // stored z^{l-1}
+      a.ld_aux = pv.ld_out;
+    } else {
+      a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;      // a^{l-1} > 0  <=>  z^{l-1} > 0
+      a.ld_aux = y.ld_in;
+    }
+    if (!y.conv && pv.conv) {
+      // FC on a flattened (unpooled) conv output: [B][H*W*C] and [B*H*W][C] are the same memory
+      a.ld_out = y.ld_in;
+      a.ld_aux = y.ld_in;
+    }
   }
   a.status = c->status;
   a.splits = y.split_d; a.partial = y.part_d; a.tile_counter = y.cnt_d;
@@ -424,9 +593,14 @@ static inline bool fused_update(const lp_ctx* c) { return (c->cfg.flags & LP_UNF
 static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
   GemmArgs a{};
-  a.M = y.n_out; a.N = y.n_in; a.K = c->cfg.batch;
-  a.ld_out = y.ld_in;
+  a.M = y.n_out; a.N = y.w_ld; a.K = y.in_rows;
+  if (!y.conv) a.N = y.n_in;
+  a.ld_out = y.w_ld;
   a.status = c->status;
+  if (y.conv) {
+    a.g = conv_geom(y, GEOM_PIX_K, y.box64, 0, 0, (y.ld_in + y.bn_g - 1) / y.bn_g);
+    a.splits = y.split_g; a.partial = y.part_g; a.tile_counter = y.cnt_g;
+  }
   if (fused_update(c)) {
     // Eq. 5 and Eq. 6 in one kernel: the accumulator tile is G; the epilogue reads the fp32
     // master (and momentum) tile, applies the update and writes master, momentum and the
@@ -455,9 +629,17 @@ static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st)
   if (u.n_elems == 0 && !y.d.has_bias) return cudaSuccess;  // nothing left to do
   if (y.d.has_bias) {
     u.delta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
-    u.rows = c->cfg.batch; u.ldd = y.ld_out; u.n_out = y.n_out;
+    u.rows = y.out_rows; u.ldd = y.ld_out; u.n_out = y.n_out;
     u.b = y.b; u.mb = y.mb; u.db = y.db;
     u.bring = y.bring + size_t(dst_slot) * y.ld_out;
+    if (y.col_chunks > 0) {
+      // many rows (convolution): column sums in two deterministic passes
+      ++c->launches;
+      cudaError_t e = launch_colsum_partial(u.delta, u.rows, u.ldd, u.n_out, y.col_partial, st);
+      if (e != cudaSuccess) return e;
+      u.col_partial = y.col_partial;
+      u.n_chunks = y.col_chunks;
+    }
   }
   u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
   ++c->launches;
@@ -557,8 +739,10 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
     y.rZ.assign(std::max(y.z_slots, 1), Res{});
     y.rDelta.assign(kDeltaSlots, Res{});
     y.rRing.assign(y.slots, Res{});
+    y.rPidx.assign(l + 1 < n_layers ? c->L[l + 1].x_slots : 1, Res{});
+    // host [out][in] (conv: [Cout][R][S][Cin]) -> device rows of padded pitch ld_in
     LP_CUDA(nullptr, cudaMemcpy2D(y.W, size_t(y.ld_in) * 4, W0_host[l], size_t(y.n_in) * 4, size_t(y.n_in) * 4,
-                                  y.n_out, cudaMemcpyHostToDevice));
+                                  size_t(y.n_out) * y.taps, cudaMemcpyHostToDevice));
     LP_CUDA(nullptr, launch_round_to_bf16(y.W, y.ring, (long long)y.w_elems, 0));
     if (y.d.has_bias && b0_host && b0_host[l]) {
       LP_CUDA(nullptr, cudaMemcpy(y.b, b0_host[l], size_t(y.n_out) * 4, cudaMemcpyHostToDevice));
@@ -643,8 +827,8 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     ++c->launches;
     TimedScope ts(c, LP_TASK_CAST, user);
     LP_CUDA(c, launch_cast_stash(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
-                                 y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.n_in,
-                                 y0.ld_in, user));
+                                 y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, y0.in_rows, B,
+                                 y0.n_in, y0.ld_in, user));
     LP_CUDA(c, task_end(c, user, {}, {rx, rl}, nullptr));
   }
   // ---- forward ---------------------------------------------------------------
@@ -655,9 +839,12 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     Res* rw = &y.rRing[slot[l]];
     Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[n % c->L[l + 1].x_slots];
     Res* rz = y.Z ? &y.rZ[n % y.z_slots] : nullptr;
-    LP_CUDA(c, task_begin(c, st, {rin, rw}, {rout, rz}));
+    Res* rpool = y.pool ? &y.rPidx[n % c->L[l + 1].x_slots] : nullptr;
+    Res* rfull = y.pool ? &y.rAfull : nullptr;
+    LP_CUDA(c, task_begin(c, st, {rin, rw}, {rout, rz, rpool, rfull}));
     LP_CUDA(c, launch_forward(c, l, n, slot[l], st));
-    LP_CUDA(c, task_end(c, st, {rin, rw}, {rout, rz}, nullptr));
+    if (y.pool) LP_CUDA(c, launch_pool(c, l, n, st));
+    LP_CUDA(c, task_end(c, st, {rin, rw}, {rout, rz, rpool, rfull}, nullptr));
   }
   // ---- loss and delta^L --------------------------------------------------------
   {
@@ -681,24 +868,26 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     Res* rnew = &y.rRing[(n + 1) % y.slots];
     Res* rdprev = nullptr;
     Res* raux = nullptr;
+    Res* ridx = nullptr;
     if (l > 0) {
       Layer& pv = c->L[l - 1];
       rdprev = &pv.rDelta[ds];
       raux = (pv.d.act == LP_ACT_GELU) ? &pv.rZ[n % pv.z_slots] : rx;
+      if (pv.pool) ridx = &pv.rPidx[n % y.x_slots];
     }
     if (fusedB) {
       cudaStream_t st = c->sD[y.stage];
-      LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux}, {rdprev, &y.rDW, rnew}));
+      LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}));
       if (l > 0) LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
       LP_CUDA(c, launch_G(c, l, n, st));
       LP_CUDA(c, launch_update(c, l, n, st));
-      LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux}, {rdprev, &y.rDW, rnew}, &y.last_update));
+      LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}, &y.last_update));
     } else {
       if (l > 0) {
         cudaStream_t st = c->sD[y.stage];
-        LP_CUDA(c, task_begin(c, st, {rdl, rw, raux}, {rdprev}));
+        LP_CUDA(c, task_begin(c, st, {rdl, rw, raux, ridx}, {rdprev}));
         LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
-        LP_CUDA(c, task_end(c, st, {rdl, rw, raux}, {rdprev}, nullptr));
+        LP_CUDA(c, task_end(c, st, {rdl, rw, raux, ridx}, {rdprev}, nullptr));
       }
       cudaStream_t sg = c->sG[y.stage];
       if (fused_update(c)) {
@@ -748,8 +937,8 @@ extern "C" int lp_get_weights(lp_handle h, int layer, float* W_out, float* b_out
   Layer& y = h->L[layer];
   if (y.last_update.e) LP_CUDA(h, cudaEventSynchronize(y.last_update.e));
   if (W_out)
-    LP_CUDA(h, cudaMemcpy2D(W_out, size_t(y.n_in) * 4, y.W, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
-                            cudaMemcpyDeviceToHost));
+    LP_CUDA(h, cudaMemcpy2D(W_out, size_t(y.n_in) * 4, y.W, size_t(y.ld_in) * 4, size_t(y.n_in) * 4,
+                            size_t(y.n_out) * y.taps, cudaMemcpyDeviceToHost));
   if (b_out) LP_CUDA(h, cudaMemcpy(b_out, y.b, size_t(y.n_out) * 4, cudaMemcpyDeviceToHost));
   if (version) *version = h->n_steps;
   return LP_OK;
@@ -763,8 +952,8 @@ extern "C" int lp_get_grads(lp_handle h, int layer, long long step, float* dW_ou
   if (dW_out && !y.dW) return fail(h, LP_ERR_NOT_READY, "G is not kept: create the handle with LP_CAPTURE_GRADS");
   if (y.last_update.e) LP_CUDA(h, cudaEventSynchronize(y.last_update.e));
   if (dW_out)
-    LP_CUDA(h, cudaMemcpy2D(dW_out, size_t(y.n_in) * 4, y.dW, size_t(y.ld_in) * 4, size_t(y.n_in) * 4, y.n_out,
-                            cudaMemcpyDeviceToHost));
+    LP_CUDA(h, cudaMemcpy2D(dW_out, size_t(y.n_in) * 4, y.dW, size_t(y.ld_in) * 4, size_t(y.n_in) * 4,
+                            size_t(y.n_out) * y.taps, cudaMemcpyDeviceToHost));
   if (db_out) LP_CUDA(h, cudaMemcpy(db_out, y.db, size_t(y.n_out) * 4, cudaMemcpyDeviceToHost));
   return LP_OK;
 }
@@ -773,7 +962,7 @@ namespace lp {
 struct BufView {
   void* ptr = nullptr;
   int rows = 0, cols = 0, ld = 0;
-  int dtype = 0;   // 0 bf16, 1 f32, 2 i32
+  int dtype = 0;   // 0 bf16, 1 f32, 2 i32, 3 u8
 };
 static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v) {
   const int nL = int(h->L.size());
@@ -787,26 +976,31 @@ static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v)
   if (buffer == LP_BUF_LOSS) { *v = {h->loss + (index % kLossRing), 1, 1, 1, 1}; return LP_OK; }
   if (layer < 0 || layer >= nL) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
   Layer& y = h->L[layer];
+  const int wr = y.n_out * y.taps;     // weight-shaped buffers as [Cout * taps][Cin] with pitch ld_in
   switch (buffer) {
-    case LP_BUF_INPUT: *v = {y.X + size_t(index % y.x_slots) * y.x_elems, B, y.n_in, y.ld_in, 0}; return LP_OK;
+    case LP_BUF_INPUT: *v = {y.X + size_t(index % y.x_slots) * y.x_elems, y.in_rows, y.n_in, y.ld_in, 0}; return LP_OK;
     case LP_BUF_Z:
       if (!y.Z) return fail(h, LP_ERR_NOT_READY, "this layer stores no pre-activation");
       *v = {y.Z + size_t(index % y.z_slots) * y.z_elems, B, y.n_out, y.ld_out, 0};
       return LP_OK;
-    case LP_BUF_DELTA: *v = {y.delta + size_t(index % kDeltaSlots) * y.delta_elems, B, y.n_out, y.ld_out, 0}; return LP_OK;
+    case LP_BUF_DELTA: *v = {y.delta + size_t(index % kDeltaSlots) * y.delta_elems, y.out_rows, y.n_out, y.ld_out, 0}; return LP_OK;
+    case LP_BUF_POOL_IDX:
+      if (!y.pidx) return fail(h, LP_ERR_NOT_READY, "this layer does not pool");
+      *v = {y.pidx + size_t(index % h->L[layer + 1].x_slots) * y.pidx_elems, B * y.Hp * y.Wp, y.n_out, y.ld_out, 3};
+      return LP_OK;
     case LP_BUF_RING_W:
       if (index >= y.slots) return fail(h, LP_ERR_INVALID_ARG, "ring slot out of range");
-      *v = {y.ring + size_t(index) * y.w_elems, y.n_out, y.n_in, y.ld_in, 0};
+      *v = {y.ring + size_t(index) * y.w_elems, wr, y.n_in, y.ld_in, 0};
       return LP_OK;
     case LP_BUF_RING_B:
       if (index >= y.slots) return fail(h, LP_ERR_INVALID_ARG, "ring slot out of range");
       *v = {y.bring + size_t(index) * y.ld_out, 1, y.n_out, y.ld_out, 1};
       return LP_OK;
-    case LP_BUF_MASTER_W: *v = {y.W, y.n_out, y.n_in, y.ld_in, 1}; return LP_OK;
+    case LP_BUF_MASTER_W: *v = {y.W, wr, y.n_in, y.ld_in, 1}; return LP_OK;
     case LP_BUF_MASTER_B: *v = {y.b, 1, y.n_out, y.ld_out, 1}; return LP_OK;
     case LP_BUF_MOM_W:
       if (!y.mW) return fail(h, LP_ERR_NOT_READY, "momentum is off");
-      *v = {y.mW, y.n_out, y.n_in, y.ld_in, 1};
+      *v = {y.mW, wr, y.n_in, y.ld_in, 1};
       return LP_OK;
     case LP_BUF_MOM_B:
       if (!y.mb) return fail(h, LP_ERR_NOT_READY, "momentum is off");
@@ -814,7 +1008,7 @@ static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v)
       return LP_OK;
     case LP_BUF_GRAD_W:
       if (!y.dW) return fail(h, LP_ERR_NOT_READY, "G is not kept: create the handle with LP_CAPTURE_GRADS");
-      *v = {y.dW, y.n_out, y.n_in, y.ld_in, 1};
+      *v = {y.dW, wr, y.n_in, y.ld_in, 1};
       return LP_OK;
     case LP_BUF_GRAD_B: *v = {y.db, 1, y.n_out, y.ld_out, 1}; return LP_OK;
   }
@@ -846,6 +1040,13 @@ extern "C" int lp_debug_read(lp_handle h, int buffer, int layer, long long index
     for (int c = 0; c < v.cols; ++c) out_host[c] = float(tmp[c]);
     return LP_OK;
   }
+  if (v.dtype == 3) {
+    std::vector<unsigned char> tmp(size_t(v.rows) * v.ld);
+    LP_CUDA(h, cudaMemcpy(tmp.data(), v.ptr, tmp.size(), cudaMemcpyDeviceToHost));
+    for (int r = 0; r < v.rows; ++r)
+      for (int c = 0; c < v.cols; ++c) out_host[size_t(r) * v.cols + c] = float(tmp[size_t(r) * v.ld + c]);
+    return LP_OK;
+  }
   std::vector<uint16_t> tmp(size_t(v.rows) * v.ld);
   LP_CUDA(h, cudaMemcpy(tmp.data(), v.ptr, tmp.size() * 2, cudaMemcpyDeviceToHost));
   for (int r = 0; r < v.rows; ++r)
@@ -873,6 +1074,13 @@ extern "C" int lp_debug_write(lp_handle h, int buffer, int layer, long long inde
     LP_CUDA(h, cudaMemcpy(v.ptr, tmp.data(), size_t(v.cols) * 4, cudaMemcpyHostToDevice));
     return LP_OK;
   }
+  if (v.dtype == 3) {
+    std::vector<unsigned char> tmp(size_t(v.rows) * v.ld, 0);
+    for (int r = 0; r < v.rows; ++r)
+      for (int c = 0; c < v.cols; ++c) tmp[size_t(r) * v.ld + c] = (unsigned char)(in_host[size_t(r) * v.cols + c]);
+    LP_CUDA(h, cudaMemcpy(v.ptr, tmp.data(), tmp.size(), cudaMemcpyHostToDevice));
+    return LP_OK;
+  }
   std::vector<uint16_t> tmp(size_t(v.rows) * v.ld, 0);
   for (int r = 0; r < v.rows; ++r)
     for (int c = 0; c < v.cols; ++c) tmp[size_t(r) * v.ld + c] = f32_to_bf16_rn(in_host[size_t(r) * v.cols + c]);
@@ -896,7 +1104,10 @@ extern "C" int lp_debug_run_task(lp_handle h, int task, int layer, long long ste
     slot = int(std::max<long long>(0, step - y.delay) % y.slots);
   }
   switch (task) {
-    case LP_TASK_FORWARD: LP_CUDA(h, launch_forward(h, layer, step, slot, st)); break;
+    case LP_TASK_FORWARD:
+      LP_CUDA(h, launch_forward(h, layer, step, slot, st));
+      if (h->L[layer].pool) LP_CUDA(h, launch_pool(h, layer, step, st));
+      break;
     case LP_TASK_LOSS: {
       Layer& yl = h->L[nL - 1];
       ++h->launches;

@@ -57,6 +57,11 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
             tr.debug_run_task("forward", l, n)
             if l < L - 1:
                 note("a", assert_bf16_close(tr.debug_read("input", l + 1, n), rec["a"][l + 1], "a^%d step %d" % (l + 1, n)))
+                if layers[l].get("pool", 0):
+                    # which window element wins may legitimately differ where two candidates are within
+                    # a rounding of each other; everywhere else the recorded position must agree
+                    same = float((tr.debug_read("pool_idx", l, n) == rec["amax"][l]).mean())
+                    assert same > 0.995, ("pool argmax", l, n, same)
                 if layers[l]["act"] == "gelu":
                     note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n)))
             else:
@@ -76,6 +81,8 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
             if l > 0:
                 if layers[l - 1]["act"] == "gelu":
                     tr.debug_write("z", l - 1, n, rec["zs"][l - 1])
+                if layers[l - 1].get("pool", 0):
+                    tr.debug_write("pool_idx", l - 1, n, rec["amax"][l - 1].astype(np.float32))
                 tr.debug_run_task("delta", l, n)
                 note("delta", assert_bf16_close(tr.debug_read("delta", l - 1, n), rec["delta"][l - 1],
                                                 "delta^%d step %d" % (l - 1, n)))
@@ -148,6 +155,24 @@ def test_tasks_split_k_forward_and_delta():
             run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.9, 4)
         finally:
             lpb.lp_set_tuning(0, 0, 0)
+
+
+def test_tasks_small_convnet():
+    """Conv 3x3 + ReLU (+ 2x2 max pool) layers followed by FC layers: implicit-GEMM forward, delta
+    with the un-pooling epilogue (conv -> conv and conv -> FC), split-K G with the fused update,
+    two-pass bias gradient.  Image sizes 16 / 8 / 4 exercise pixel boxes that span several rows
+    and several images; 3 input channels exercise the padded first layer."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(16, [16, 32, "P", 64, "P", 72, "P"], [40, 10])
+    run_teacher_forced(layers, 16, 4, None, 0.05, 0.9, 4)
+
+
+def test_tasks_vgg_small_32_full_config():
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["vgg_small_32"]
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 8,
+                           check_steps={0, 7})
+    print("worst per-task errors", w)
 
 
 def test_tasks_papers_double_delay_convention():

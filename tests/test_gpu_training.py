@@ -127,6 +127,19 @@ def test_free_running_mlp8_4096_full_size():
             grad_bound=5 * rounding_noise(8), step0_bound=1.5 * rounding_noise(8))
 
 
+def test_free_running_small_convnet_planned_stages():
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(16, [16, 32, "P", 64, "P"], [48, 10])
+    compare("cnn16", layers, 32, 3, None, 0.02, 0.9, 8, grad_bound=0.2, step0_bound=2e-2)
+
+
+def test_free_running_vgg_small_32_full_config():
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["vgg_small_32"]
+    compare("vgg_small_32", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"],
+            wl["steps"], grad_bound=0.2, step0_bound=2e-2)
+
+
 def test_fused_and_unfused_update_agree():
     """The fused epilogue and the separate update kernel evaluate the same expressions on the
     same fp32 accumulators: the two trajectories must be bit-identical."""
