@@ -50,18 +50,22 @@ def work_model(layers, batch, momentum):
     L = len(layers)
     for l, y in enumerate(layers):
         n_in, n_out = y["n_in"], y["n_out"]
-        fl = 2.0 * batch * n_in * n_out
+        conv = y["kind"] == "conv"
+        rows = batch * y["H"] * y["W"] if conv else batch      # pixels (conv) or samples (FC)
+        params = n_in * n_out * (9 if conv else 1)
+        fl = 2.0 * rows * params
         gelu = y["act"] == "gelu"
         last = l == L - 1
-        out["forward"].append(dict(flops=fl, bytes=2.0 * n_in * n_out + 2.0 * batch * n_in +
-                                   (4.0 if last else (4.0 if gelu else 2.0)) * batch * n_out))
+        pool = 1.25 * 2.0 * rows * n_out + 0.25 * rows * n_out if y.get("pool", 0) else 0.0   # re-read a, write pooled + argmax
+        out["forward"].append(dict(flops=fl, bytes=2.0 * params + 2.0 * rows * n_in +
+                                   (4.0 if last else (4.0 if gelu else 2.0)) * rows * n_out + pool))
         if l > 0:
-            out["delta"].append(dict(flops=fl, bytes=2.0 * n_in * n_out + 2.0 * batch * n_out + 4.0 * batch * n_in))
+            out["delta"].append(dict(flops=fl, bytes=2.0 * params + 2.0 * rows * n_out + 4.0 * rows * n_in))
         # G with the update fused into its epilogue: read W (,m), write W (,m) fp32 and the bf16 ring slot
         per_param = 18.0 if momentum != 0.0 else 10.0
-        out["G"].append(dict(flops=fl, bytes=2.0 * batch * (n_in + n_out) + per_param * n_in * n_out))
+        out["G"].append(dict(flops=fl, bytes=2.0 * rows * (n_in + n_out) + per_param * params))
         # what is left of the update: bias gradient (column sums of delta) and the bias update
-        out["update"].append(dict(flops=0.0, bytes=2.0 * batch * n_out + 24.0 * n_out))
+        out["update"].append(dict(flops=0.0, bytes=2.0 * rows * n_out + 24.0 * n_out))
     return out
 
 
