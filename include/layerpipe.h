@@ -209,7 +209,8 @@ int lp_reset_task_times(lp_handle h);
 /* Number of kernels this handle has launched so far. */
 long long lp_kernel_launches(lp_handle h);
 
-/* Tuning hook for experiments: force the GEMM tile width (64, 128, 256; 0 = automatic), the
+/* Tuning hook for experiments: force the GEMM tile width (64, 128, 256, or 512 = 256 x 256 tile on an
+ * SM pair with tcgen05 cta_group::2, plain matrices only; 0 = automatic), the
  * shared-memory pipeline depth (0 = automatic) and the split-K factor of the forward / delta
  * contractions (0 = automatic, 1 = off) for handles created afterwards. */
 int lp_set_tuning(int tile_n, int stages, int split_k);

@@ -23,6 +23,7 @@ int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t
                         uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err);
 
 struct GemmArgs;
+constexpr int GEMM_BN_PAIR = 512;   // tile code: 256 x 256 tile computed by a pair of CTAs (cta_group::2)
 // which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
 // Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
 // (see gemm_box_dims).

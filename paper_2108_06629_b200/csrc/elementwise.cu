@@ -108,12 +108,21 @@ __global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const
     last = (t == unsigned(B) - 1u);
   }
   __syncthreads();
-  if (last && threadIdx.x == 0) {
+  if (last) {
+    // deterministic mean: thread t adds rows t, t + 256, ... in that order, then the 256 partial
+    // sums are added in thread order
     __threadfence();
     float acc = 0.f;
-    for (int i = 0; i < B; ++i) acc += __ldcg(row_loss + i);
-    *loss_out = acc * invB;
-    *ticket = 0u;     // ready for the next launch on this scratch
+    for (int i = threadIdx.x; i < B; i += blockDim.x) acc += __ldcg(row_loss + i);
+    __shared__ float part[256];
+    part[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      for (int i = 0; i < int(blockDim.x); ++i) tot += part[i];
+      *loss_out = tot * invB;
+      *ticket = 0u;     // ready for the next launch on this scratch
+    }
   }
 }
 

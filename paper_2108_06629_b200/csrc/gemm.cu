@@ -1,6 +1,6 @@
 // Host side of the tcgen05 GEMM: tensor-map encoding, tile selection, launch, and the
 // stand-alone lp_gemm_bf16 entry point.
-#include "gemm.cuh"
+#include "gemm2.cuh"
 
 #include <algorithm>
 #include <mutex>
@@ -105,9 +105,11 @@ int gemm_pick_splits(int M, int N, int K, int bn) {
 }
 
 int gemm_pick_bn(int which, int M, int N, int K) {
-  (void)which;
-  if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256) return g_force_bn;
+  if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256 || g_force_bn == GEMM_BN_PAIR) return g_force_bn;
   if (N <= 64) return 64;
+  // tensor-bound shapes: 256 x 256 tiles on SM pairs (code GEMM_BN_PAIR)
+  if (M >= 1024 && N >= 1024 && K >= 1024) return GEMM_BN_PAIR;
+  (void)which;
   // 128 x 256 tiles need 96 B/clk of operands per SM instead of 128 B/clk and measured 1250 vs
   // 1130 TFLOP/s on 2048 x 8192 x 8192; they only pay off when the contraction is long and
   // there are enough tiles to fill two CTAs on every SM
@@ -122,7 +124,7 @@ int gemm_pick_bn(int which, int M, int N, int K) {
 void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
   boxA[0] = 64; boxA[1] = a_mn ? 64 : GEMM_BM;
-  boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(bn);
+  boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(bn == GEMM_BN_PAIR ? 128 : bn);   // a pair CTA stages half of the 256 columns
 }
 
 static int pick_stages(int bn, int K) {
@@ -164,8 +166,49 @@ static cudaError_t configure_one() {
   X(BN, true, true, EPI_STORE_F32)           \
   X(BN, true, true, EPI_WGRAD_UPDATE)
 
+// ---- two-CTA (SM pair) kernel ---------------------------------------------------------------
+template <bool A_MN, bool B_MN, int MODE>
+static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
+  a.splits = 1;
+  const int stage_bytes = 32 * 1024;
+  const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
+  int s = g_force_stages > 0 ? g_force_stages : 3;               // 3 x 32 KiB: two CTAs per SM
+  s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb, 2)));
+  while (s > 2 && size_t(s) * stage_bytes + 1280 > 227 * 1024) --s;
+  a.num_stages = s;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N + GEMM2_BN - 1) / GEMM2_BN, 1);
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = size_t(s) * stage_bytes + 1024 + 256;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE>, tmA, tmB, a);
+}
+template <bool A_MN, bool B_MN, int MODE>
+static cudaError_t configure_pair() {
+  return cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              227 * 1024);
+}
+#define LP_FOR_EACH_PAIR_VARIANT(X)   \
+  X(false, false, EPI_FPROP)          \
+  X(false, false, EPI_STORE_F32)      \
+  X(false, true, EPI_DGRAD)           \
+  X(false, true, EPI_STORE_F32)       \
+  X(true, true, EPI_STORE_F32)        \
+  X(true, true, EPI_WGRAD_UPDATE)
+
 cudaError_t gemm_configure() {
   cudaError_t e;
+#define LP_CFGP(A, B, M) \
+  if ((e = configure_pair<A, B, M>()) != cudaSuccess) return e;
+  LP_FOR_EACH_PAIR_VARIANT(LP_CFGP)
+#undef LP_CFGP
 #define LP_CFG(BN, A, B, M) \
   if ((e = configure_one<BN, A, B, M>()) != cudaSuccess) return e;
   LP_FOR_EACH_VARIANT(LP_CFG, 64)
@@ -178,6 +221,14 @@ cudaError_t gemm_configure() {
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
                         cudaStream_t st) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
+  if (bn == GEMM_BN_PAIR) {
+    if (args.g.kind != GEOM_PLAIN) return cudaErrorInvalidValue;
+#define LP_TRYP(A, B, M) \
+  if (a_mn == A && b_mn == B && args.mode == M) return launch_pair<A, B, M>(tmA, tmB, args, st);
+    LP_FOR_EACH_PAIR_VARIANT(LP_TRYP)
+#undef LP_TRYP
+    return cudaErrorInvalidValue;
+  }
 #define LP_TRY(BN, A, B, M) \
   if (bn == BN && a_mn == A && b_mn == B && args.mode == M) return launch_one<BN, A, B, M>(tmA, tmB, args, st);
   LP_FOR_EACH_VARIANT(LP_TRY, 64)

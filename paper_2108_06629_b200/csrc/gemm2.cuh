@@ -1,0 +1,245 @@
+// Two-CTA variant of the tcgen05 GEMM for tensor-bound shapes: a cluster of two CTAs (an SM
+// pair) computes one 256 x 256 output tile with tcgen05.mma.cta_group::2.  Each CTA stages its
+// own 128 rows of A and only HALF of the B tile (128 of the 256 columns); the tensor cores of
+// both SMs read both halves.  Per k-block an SM therefore loads 32 KiB for 128 x 256 x 64 MACs
+// (64 B/clk at full tensor rate) instead of the 48 KiB (96 B/clk) a 128 x 256 single-CTA tile
+// needs -- the difference between being fed by L2 and starving.
+//
+//   rank 0 ("leader"): TMA producer, MMA issuer for BOTH CTAs, epilogue of its 128 rows
+//   rank 1           : TMA producer (its loads signal the leader's barrier), epilogue of its rows
+//
+// Hand-offs: TMA loads of both CTAs complete on the leader's "full" barrier (the leader arms it
+// with the byte count of both); tcgen05.commit multicasts the "empty" and "accumulator ready"
+// arrivals to the same barrier in both CTAs.  No TMA load uses cluster multicast.
+// Plain matrices only (no convolution geometry, no split-K); epilogues as in gemm.cuh.
+#pragma once
+#include "gemm.cuh"
+
+namespace lp {
+
+constexpr int GEMM2_BN = 256;
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t* smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// 2-D tiled load whose completion is counted on the LEADER's barrier
+__device__ __forceinline__ void tma2_load_2d_addr(uint32_t smem_dst, const CUtensorMap* m, uint32_t leader_bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+      "%4}], [%2];" ::"r"(smem_dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(leader_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma2_f16_lohi(uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(tmem_d),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs once all MMAs issued so far are done
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}" ::"r"(bar)
+      : "memory");
+}
+
+template <bool A_MN, bool B_MN, int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const GemmArgs p) {
+  constexpr int STAGE_BYTES = GEMM_A_BYTES + 128 * GEMM_BK * 2;      // A rows + half of the B tile: 32 KiB
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int S = p.num_stages;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + size_t(S) * STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
+  uint64_t* acc_bar = empty_bar + GEMM_MAX_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+  float* epi_tile = reinterpret_cast<float*>(smem);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int num_kb = (p.K + GEMM_BK - 1) / GEMM_BK;
+
+  TileMap tm;
+  tm.m0 = (blockIdx.x >> 1) * 256 + int(rank) * 128;    // this CTA's 128 rows
+  tm.n0 = blockIdx.y * GEMM2_BN;                        // the pair's 256 columns
+  tm.nlim = p.N;
+  tm.pn0 = tm.ph0 = tm.pw0 = 0;
+  const int nb0 = tm.n0 + int(rank) * 128;              // the half of B this CTA stages
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(acc_bar, 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc2(tmem_slot, GEMM2_BN);
+    tmem_relinquish2();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();          // the peer's barriers exist before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      bool ok = true;
+      int issued = 0;
+      const uint32_t smem0 = smem_u32(smem);
+      const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+      uint32_t s = 0, ph = 0;
+      int k0 = 0;
+      for (int kb = 0; kb < num_kb; ++kb, k0 += GEMM_BK) {
+        ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+        if (!ok) break;
+        const uint32_t sa = smem0 + s * uint32_t(STAGE_BYTES);
+        const uint32_t sb = sa + GEMM_A_BYTES;
+        const uint32_t fb = map_to_cta(full0 + 8u * s, 0);          // the leader's barrier
+        if (rank == 0) mbar_arrive_expect_tx_addr(full0 + 8u * s, 2 * STAGE_BYTES);
+        if (A_MN) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) tma2_load_2d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, k0);
+        } else {
+          tma2_load_2d_addr(sa, &tmA, fb, k0, tm.m0);
+        }
+        if (B_MN) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) tma2_load_2d_addr(sb + c * 8192, &tmB, fb, nb0 + c * 64, k0);
+        } else {
+          tma2_load_2d_addr(sb, &tmB, fb, k0, nb0);
+        }
+        issued = kb + 1;
+        if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) {
+        atomicExch(p.status, 11);
+        if (rank == 0)
+          for (int kb = max(0, issued - S); kb < issued; ++kb) mbar_wait(&full_bar[kb % S], (kb / S) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(256, GEMM2_BN, A_MN, B_MN);
+      const uint64_t dA = A_MN ? make_smem_desc(smem_u32(smem), 8192, 1024) : make_smem_desc(smem_u32(smem), 16, 1024);
+      const uint64_t dB = B_MN ? make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 8192, 1024)
+                               : make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 16, 1024);
+      const uint32_t dA_hi = uint32_t(dA >> 32), dB_hi = uint32_t(dB >> 32);
+      constexpr uint32_t stepA = (A_MN ? 2048 : 32) >> 4, stepB = (B_MN ? 2048 : 32) >> 4;
+      const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+      uint32_t s = 0, ph = 0, acc = 0;
+      uint32_t dA_lo = uint32_t(dA), dB_lo = uint32_t(dB);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        ok = mbar_wait_addr(full0 + 8u * s, ph);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < GEMM_BK / 16; ++j) {
+          umma2_f16_lohi(tmem_base, dA_lo + j * stepA, dA_hi, dB_lo + j * stepB, dB_hi, idesc, acc);
+          acc = 1;
+        }
+        umma2_commit_both(empty0 + 8u * s);
+        dA_lo += uint32_t(STAGE_BYTES >> 4);
+        dB_lo += uint32_t(STAGE_BYTES >> 4);
+        if (++s == uint32_t(S)) {
+          s = 0;
+          ph ^= 1u;
+          dA_lo = uint32_t(dA);
+          dB_lo = uint32_t(dB);
+        }
+      }
+      if (!ok) atomicExch(p.status, 12);
+      umma2_commit_both(smem_u32(acc_bar));
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (both CTAs, own rows)
+    const int q = warp & 3;
+    float* tile = epi_tile + q * (32 * EPI_PITCH);
+    const int sub_row = lane >> 3;
+    const int sub_col = (lane & 7) * 4;
+    const int row0 = tm.m0 + q * 32;
+    constexpr bool upd = (MODE == EPI_WGRAD_UPDATE);
+    WmRegs cur;
+    if constexpr (upd) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);
+    bool ok = mbar_wait(acc_bar, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok && lane == 0) atomicExch(p.status, 13);
+    tc_fence_after();
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < GEMM2_BN / 32; ++c) {
+        uint32_t r[32];
+        __syncwarp();
+        tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+        __syncwarp();
+        const int n = tm.n0 + c * 32 + sub_col;
+        if constexpr (upd) {
+          WmRegs nxt;
+          if (c + 1 < GEMM2_BN / 32) load_wm(p, row0, n + 32, tm.nlim, sub_row, nxt);
+          apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);
+          cur = nxt;
+        } else {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + sub_row;
+            const int row = row0 + rr;
+            const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
+            if (row < p.M) epilogue_store4<MODE>(p, row, n, tm.nlim, acc);
+          }
+        }
+      }
+    }
+  }
+  // neither CTA may release shared or tensor memory while its partner can still touch it
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, GEMM2_BN);
+  }
+}
+
+}  // namespace lp

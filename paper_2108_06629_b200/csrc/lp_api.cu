@@ -330,8 +330,8 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in);
       y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out);
       y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B);
-      y.split_f = gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
-      y.split_d = gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
+      y.split_f = y.bn_f == GEMM_BN_PAIR ? 1 : gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
+      y.split_d = y.bn_d == GEMM_BN_PAIR ? 1 : gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
       y.split_g = 1;
     }
     y.col_chunks = y.out_rows > 8192 ? (y.out_rows + kColsumChunk - 1) / kColsumChunk : 0;
@@ -765,7 +765,7 @@ extern "C" int lp_destroy(lp_handle h) {
 extern "C" const char* lp_last_error(lp_handle h) { return h ? h->err.c_str() : g_err.c_str(); }
 
 extern "C" int lp_set_tuning(int tile_n, int stages, int split_k) {
-  if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) || stages < 0 || stages > GEMM_MAX_STAGES ||
+  if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256 && tile_n != GEMM_BN_PAIR) || stages < 0 || stages > GEMM_MAX_STAGES ||
       split_k < 0 || split_k > 64)
     return LP_ERR_INVALID_ARG;
   gemm_set_tuning(tile_n, stages, split_k);

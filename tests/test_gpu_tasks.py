@@ -175,6 +175,19 @@ def test_tasks_vgg_small_32_full_config():
     print("worst per-task errors", w)
 
 
+def test_tasks_sm_pair_tiles():
+    """All three contractions and the fused update through the two-CTA (cta_group::2) kernel,
+    forced onto shapes with ragged 256 x 256 tiles."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([520, 328, 600, 75], "gelu")
+    lpb.lp_set_tuning(512, 0, 0)
+    try:
+        run_teacher_forced(layers, 300, 3, [2, 1, 0], 0.05, 0.9, 4)
+    finally:
+        lpb.lp_set_tuning(0, 0, 0)
+
+
 def test_tasks_papers_double_delay_convention():
     """Delays = 2 x (stages after the layer), the count Section III-A gives for the retimed graph."""
     from paper_2108_06629_b200 import inputs as I
