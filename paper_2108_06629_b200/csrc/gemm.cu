@@ -127,14 +127,15 @@ void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]) {
   boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(bn == GEMM_BN_PAIR ? 128 : bn);   // a pair CTA stages half of the 256 columns
 }
 
-static int pick_stages(int bn, int K) {
-  const int stage_bytes = GEMM_A_BYTES + bn * GEMM_BK * 2;
-  int s = g_force_stages > 0 ? g_force_stages : (100 * 1024) / stage_bytes;   // two CTAs per SM
-  s = std::min(s, GEMM_MAX_STAGES);
-  const int num_kb = (K + GEMM_BK - 1) / GEMM_BK;
-  s = std::max(2, std::min(s, std::max(num_kb, 2)));
-  while (s > 2 && size_t(s) * stage_bytes + 1280 > 227 * 1024) --s;
-  return s;
+
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+  }
+  return n;
 }
 
 template <int BN, bool A_MN, bool B_MN, int MODE>
@@ -142,17 +143,33 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   if (a.splits < 1 || a.partial == nullptr) a.splits = 1;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
-  a.num_stages = pick_stages(BN, a.kb_per_split * GEMM_BK);
-  const size_t smem = GemmSmem<BN>::bytes(a.num_stages);
-  dim3 grid((a.M + GEMM_BM - 1) / GEMM_BM, (a.N + BN - 1) / BN, a.splits);
-  if (a.g.kind == GEOM_PIX_K) grid.y = unsigned(a.g.n_per_tap) * unsigned(a.N / a.g.tap_pitch);   // (tap, channel block)
-  gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a);
+  // BN <= 128: two persistent CTAs per SM (2 x 2 x BN tensor-memory columns); BN = 256: one
+  const int per_sm = BN <= 128 ? 2 : 1;
+  const int stage_bytes = GEMM_A_BYTES + BN * GEMM_BK * 2;
+  const int budget = (per_sm == 2 ? 113 : 227) * 1024 - 1024 - 256 - EPI_TILE_BYTES - 512;
+  int s = g_force_stages > 0 ? g_force_stages : budget / stage_bytes;
+  s = std::max(2, std::min(s, GEMM_MAX_STAGES));
+  while (s > 2 && size_t(s) * stage_bytes > size_t(227 * 1024 - 1024 - 256 - EPI_TILE_BYTES - 512)) --s;
+  a.num_stages = s;
+  const size_t smem = GemmSmem<BN>::bytes(s);
+  const int tiles_m = (a.M + GEMM_BM - 1) / GEMM_BM;
+  int tiles_n = (a.N + BN - 1) / BN;
+  if (a.g.kind == GEOM_PIX_K) tiles_n = a.g.n_per_tap * (a.N / a.g.tap_pitch);   // (tap, channel block)
+  const long long work = (long long)tiles_m * tiles_n * a.splits;
+  const int grid = int(std::min<long long>(work, (long long)sm_count() * per_sm));
+  if (a.splits > 1)
+    gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, true><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a, tiles_m, tiles_n, int(work));
+  else
+    gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a, tiles_m, tiles_n, int(work));
   return cudaGetLastError();
 }
 
 template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t configure_one() {
-  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               227 * 1024);
 }
 

@@ -265,50 +265,69 @@ template <int BN>
 struct GemmSmem {
   static constexpr int B_BYTES = BN * GEMM_BK * 2;
   static constexpr int STAGE_BYTES = GEMM_A_BYTES + B_BYTES;
-  static constexpr size_t bytes(int stages) { return size_t(stages) * STAGE_BYTES + 1024 /*align slack*/ + 256; }
+  // pipeline stages, barriers (256 B), the epilogue's staging tiles, alignment slack
+  static constexpr size_t bytes(int stages) { return size_t(stages) * STAGE_BYTES + 256 + EPI_TILE_BYTES + 1024; }
 };
 
-template <int BN, bool A_MN, bool B_MN, int MODE>
-__global__ void __launch_bounds__(GEMM_THREADS, 2)
+// One output tile (and, with split-K, one slice of its contraction) of the launch.
+struct TileCtx {
+  TileMap tm;
+  int tap, col0;        // GEOM_PIX_K: filter tap and first input channel of the column tile
+  int kb_begin, num_kb; // k-blocks of this work item
+  int tile_id, z;       // output tile index and split index
+};
+
+template <int BN>
+__device__ __forceinline__ TileCtx decode_tile(const GemmArgs& p, int t, int tiles_m, int tiles_n) {
+  TileCtx c;
+  const int tiles = tiles_m * tiles_n;
+  c.z = t / tiles;
+  c.tile_id = t - c.z * tiles;
+  const int bx = c.tile_id % tiles_m, by = c.tile_id / tiles_m;     // row tiles fastest: neighbours share the B tile
+  const int num_kb_total = (p.K + GEMM_BK - 1) / GEMM_BK;
+  c.kb_begin = (p.splits > 1) ? c.z * p.kb_per_split : 0;
+  c.num_kb = (p.splits > 1) ? max(0, min(num_kb_total, c.kb_begin + p.kb_per_split) - c.kb_begin) : num_kb_total;
+  c.tm.m0 = bx * GEMM_BM;
+  c.tm.n0 = by * BN;
+  c.tm.nlim = p.N;
+  c.tm.pn0 = c.tm.ph0 = c.tm.pw0 = 0;
+  c.tap = 0;
+  c.col0 = c.tm.n0;
+  if (p.g.kind == GEOM_PIX_M) {
+    const int tw = bx % p.g.tiles_w, th = (bx / p.g.tiles_w) % p.g.tiles_h, tn = bx / (p.g.tiles_w * p.g.tiles_h);
+    c.tm.pw0 = tw << p.g.lw;
+    c.tm.ph0 = th << p.g.lh;
+    c.tm.pn0 = tn * (GEMM_BM >> (p.g.lw + p.g.lh));
+  } else if (p.g.kind == GEOM_PIX_K) {
+    c.tap = by / p.g.n_per_tap;
+    c.col0 = (by % p.g.n_per_tap) * BN;
+    c.tm.n0 = c.tap * p.g.tap_pitch + c.col0;
+    c.tm.nlim = c.tap * p.g.tap_pitch + p.g.tap_pitch;     // columns of the next tap belong to another tile
+  }
+  return c;
+}
+
+// Persistent kernel: the grid is sized to the machine (gridDim.x CTAs), CTA b works through
+// tiles b, b + gridDim.x, ...  The accumulator is double-buffered in tensor memory (2 x BN
+// columns) so that the epilogue of one tile overlaps the main loop of the next, and the
+// shared-memory pipeline runs on across tile boundaries.
+template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK>
+__global__ void __launch_bounds__(GEMM_THREADS, BN <= 128 ? 2 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmArgs p) {
+                    const GemmArgs p, const int tiles_m, const int tiles_n, const int total_work) {
   using SM = GemmSmem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int S = p.num_stages;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + size_t(S) * SM::STAGE_BYTES);
   uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
-  uint64_t* acc_bar = empty_bar + GEMM_MAX_STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
-  // the epilogue's staging tiles reuse pipeline stage 0: by the time the accumulator barrier
-  // fires every TMA load has landed and every MMA has finished reading shared memory
-  float* epi_tile = reinterpret_cast<float*>(smem);
+  uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;     // [2] accumulator buffer full  (MMA -> epilogue)
+  uint64_t* acce_bar = accf_bar + 2;                    // [2] accumulator buffer empty (epilogue -> MMA)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce_bar + 2);
+  float* epi_tile = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + 256);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_kb_total = (p.K + GEMM_BK - 1) / GEMM_BK;
-  const int kb_begin = (p.splits > 1) ? int(blockIdx.z) * p.kb_per_split : 0;
-  const int num_kb = (p.splits > 1) ? max(0, min(num_kb_total, kb_begin + p.kb_per_split) - kb_begin) : num_kb_total;
-
-  // ---- where this tile sits -----------------------------------------------------------------
-  TileMap tm;
-  tm.m0 = blockIdx.x * GEMM_BM;
-  tm.n0 = blockIdx.y * BN;
-  tm.nlim = p.N;
-  tm.pn0 = tm.ph0 = tm.pw0 = 0;
-  int tap = 0, col0 = tm.n0;      // GEOM_PIX_K: filter tap and first input channel of this column tile
-  if (p.g.kind == GEOM_PIX_M) {
-    const int mt = blockIdx.x;
-    const int tw = mt % p.g.tiles_w, th = (mt / p.g.tiles_w) % p.g.tiles_h, tn = mt / (p.g.tiles_w * p.g.tiles_h);
-    tm.pw0 = tw << p.g.lw;
-    tm.ph0 = th << p.g.lh;
-    tm.pn0 = tn * (GEMM_BM >> (p.g.lw + p.g.lh));
-  } else if (p.g.kind == GEOM_PIX_K) {
-    tap = blockIdx.y / p.g.n_per_tap;
-    col0 = (blockIdx.y % p.g.n_per_tap) * BN;
-    tm.n0 = tap * p.g.tap_pitch + col0;
-    tm.nlim = tap * p.g.tap_pitch + p.g.tap_pitch;     // columns of the next tap belong to another tile
-  }
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
@@ -317,11 +336,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(acc_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&accf_bar[b], 1);
+      mbar_init(&acce_bar[b], 4);      // one arrival per epilogue warp
+    }
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -336,81 +358,85 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // stays short (a single thread issues at a few cycles per instruction).
     if (lane == 0) {
       bool ok = true;
-      int issued = 0;
+      long long issued = 0;
       const uint32_t smem0 = smem_u32(smem);
       const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
       uint32_t s = 0, ph = 0;
-      // running position of the contraction
-      int k0 = kb_begin * GEMM_BK;                       // plain: element offset along K
-      int c_tap = 0, c_chunk = 0;                        // PIX_M: filter tap, 64-channel chunk
-      int bw0 = 0, bh0 = 0, bn0 = 0;                     // PIX_K: pixel box of this k-block
-      int dh = 0, dw = 0;                                // PIX_K: pixel shift of this tile's tap
-      if (p.g.kind == GEOM_PIX_M) {
-        c_tap = kb_begin / p.g.chunks_per_tap;
-        c_chunk = kb_begin % p.g.chunks_per_tap;
-      } else if (p.g.kind == GEOM_PIX_K) {
-        const int tw = kb_begin % p.g.tiles_w, th = (kb_begin / p.g.tiles_w) % p.g.tiles_h;
-        bw0 = tw << p.g.lw;
-        bh0 = th << p.g.lh;
-        bn0 = (kb_begin / (p.g.tiles_w * p.g.tiles_h)) * (GEMM_BK >> (p.g.lw + p.g.lh));
-        dh = tap / p.g.S - p.g.pad;
-        dw = tap % p.g.S - p.g.pad;
-      }
-      for (int kb = 0; kb < num_kb; ++kb) {
-        ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
-        if (!ok) break;
-        const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
-        const uint32_t sb = sa + GEMM_A_BYTES;
-        const uint32_t fb = full0 + 8u * s;
-        mbar_arrive_expect_tx_addr(fb, SM::STAGE_BYTES);
-        if (p.g.kind == GEOM_PLAIN) {
-          if (A_MN) {
-#pragma unroll
-            for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, k0);
-          } else {
-            tma_load_2d_addr(sa, &tmA, fb, k0, tm.m0);
-          }
-          if (B_MN) {
-#pragma unroll
-            for (int c = 0; c < BN / 64; ++c) tma_load_2d_addr(sb + c * 8192, &tmB, fb, tm.n0 + c * 64, k0);
-          } else {
-            tma_load_2d_addr(sb, &tmB, fb, k0, tm.n0);
-          }
-          k0 += GEMM_BK;
-        } else if (p.g.kind == GEOM_PIX_M) {
-          // A: 128 pixels x 64 channels of the activation / delta tensor, shifted by the tap
-          const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
-          const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
-          const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;
-          tma_load_4d_addr(sa, &tmA, fb, c_chunk * 64, tm.pw0 + sw, tm.ph0 + sh, tm.pn0);
-          if (B_MN) {   // delta: B[k = (tap, co)][n = ci]: rows co, columns tap*pitch + ci
-#pragma unroll
-            for (int c = 0; c < BN / 64; ++c)
-              tma_load_2d_addr(sb + c * 8192, &tmB, fb, c_tap * p.g.tap_pitch + tm.n0 + c * 64, c_chunk * 64);
-          } else {      // forward: B[n = co][k = (tap, ci)]
-            tma_load_2d_addr(sb, &tmB, fb, c_tap * p.g.tap_pitch + c_chunk * 64, tm.n0);
-          }
-          if (++c_chunk == p.g.chunks_per_tap) { c_chunk = 0; ++c_tap; }
-        } else {
-          // G: A = delta (64 pixels x 128 output channels), B = activations shifted by the tap
-#pragma unroll
-          for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_4d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, bw0, bh0, bn0);
-#pragma unroll
-          for (int c = 0; c < BN / 64; ++c) tma_load_4d_addr(sb + c * 8192, &tmB, fb, col0 + c * 64, bw0 + dw, bh0 + dh, bn0);
-          bw0 += 1 << p.g.lw;
-          if (bw0 >= p.g.W) {
-            bw0 = 0;
-            bh0 += 1 << p.g.lh;
-            if (bh0 >= p.g.H) { bh0 = 0; bn0 += GEMM_BK >> (p.g.lw + p.g.lh); }
-          }
+      for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x) {
+        const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
+        const TileMap& tm = tc.tm;
+        // running position of the contraction
+        int k0 = tc.kb_begin * GEMM_BK;                    // plain: element offset along K
+        int c_tap = 0, c_chunk = 0;                        // PIX_M: filter tap, 64-channel chunk
+        int bw0 = 0, bh0 = 0, bn0 = 0;                     // PIX_K: pixel box of this k-block
+        int dh = 0, dw = 0;                                // PIX_K: pixel shift of this tile's tap
+        if (p.g.kind == GEOM_PIX_M) {
+          c_tap = tc.kb_begin / p.g.chunks_per_tap;
+          c_chunk = tc.kb_begin % p.g.chunks_per_tap;
+        } else if (p.g.kind == GEOM_PIX_K) {
+          const int tw = tc.kb_begin % p.g.tiles_w, th = (tc.kb_begin / p.g.tiles_w) % p.g.tiles_h;
+          bw0 = tw << p.g.lw;
+          bh0 = th << p.g.lh;
+          bn0 = (tc.kb_begin / (p.g.tiles_w * p.g.tiles_h)) * (GEMM_BK >> (p.g.lw + p.g.lh));
+          dh = tc.tap / p.g.S - p.g.pad;
+          dw = tc.tap % p.g.S - p.g.pad;
         }
-        issued = kb + 1;
-        if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
+        for (int kb = 0; kb < tc.num_kb; ++kb) {
+          ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+          if (!ok) break;
+          const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
+          const uint32_t sb = sa + GEMM_A_BYTES;
+          const uint32_t fb = full0 + 8u * s;
+          mbar_arrive_expect_tx_addr(fb, SM::STAGE_BYTES);
+          if (p.g.kind == GEOM_PLAIN) {
+            if (A_MN) {
+#pragma unroll
+              for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_2d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, k0);
+            } else {
+              tma_load_2d_addr(sa, &tmA, fb, k0, tm.m0);
+            }
+            if (B_MN) {
+#pragma unroll
+              for (int c = 0; c < BN / 64; ++c) tma_load_2d_addr(sb + c * 8192, &tmB, fb, tm.n0 + c * 64, k0);
+            } else {
+              tma_load_2d_addr(sb, &tmB, fb, k0, tm.n0);
+            }
+            k0 += GEMM_BK;
+          } else if (p.g.kind == GEOM_PIX_M) {
+            // A: 128 pixels x 64 channels of the activation / delta tensor, shifted by the tap
+            const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
+            const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
+            const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;
+            tma_load_4d_addr(sa, &tmA, fb, c_chunk * 64, tm.pw0 + sw, tm.ph0 + sh, tm.pn0);
+            if (B_MN) {   // delta: B[k = (tap, co)][n = ci]: rows co, columns tap*pitch + ci
+#pragma unroll
+              for (int c = 0; c < BN / 64; ++c)
+                tma_load_2d_addr(sb + c * 8192, &tmB, fb, c_tap * p.g.tap_pitch + tm.n0 + c * 64, c_chunk * 64);
+            } else {      // forward: B[n = co][k = (tap, ci)]
+              tma_load_2d_addr(sb, &tmB, fb, c_tap * p.g.tap_pitch + c_chunk * 64, tm.n0);
+            }
+            if (++c_chunk == p.g.chunks_per_tap) { c_chunk = 0; ++c_tap; }
+          } else {
+            // G: A = delta (64 pixels x 128 output channels), B = activations shifted by the tap
+#pragma unroll
+            for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_4d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, bw0, bh0, bn0);
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c) tma_load_4d_addr(sb + c * 8192, &tmB, fb, tc.col0 + c * 64, bw0 + dw, bh0 + dh, bn0);
+            bw0 += 1 << p.g.lw;
+            if (bw0 >= p.g.W) {
+              bw0 = 0;
+              bh0 += 1 << p.g.lh;
+              if (bh0 >= p.g.H) { bh0 = 0; bn0 += GEMM_BK >> (p.g.lw + p.g.lh); }
+            }
+          }
+          ++issued;
+          if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
+        }
       }
       if (!ok) {
         atomicExch(p.status, 1);
         // let copies already in flight land before the CTA's shared memory is released
-        for (int kb = max(0, issued - S); kb < issued; ++kb) mbar_wait(&full_bar[kb % S], (kb / S) & 1);
+        for (long long i = (issued > S ? issued - S : 0); i < issued; ++i) mbar_wait(&full_bar[i % S], uint32_t(i / S) & 1u);
       }
     }
   } else if (warp == 1) {
@@ -425,30 +451,42 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t dA_hi = uint32_t(dA >> 32), dB_hi = uint32_t(dB >> 32);
       constexpr uint32_t stepA = (A_MN ? 2048 : 32) >> 4, stepB = (B_MN ? 2048 : 32) >> 4;
       const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
-      uint32_t s = 0, ph = 0, acc = 0;
+      const uint32_t accf0 = smem_u32(accf_bar), acce0 = smem_u32(acce_bar);
+      uint32_t s = 0, ph = 0;
       uint32_t dA_lo = uint32_t(dA), dB_lo = uint32_t(dB);
       bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        ok = mbar_wait_addr(full0 + 8u * s, ph);
+      uint32_t it = 0;     // tiles done by this CTA
+      for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x, ++it) {
+        const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
+        const uint32_t buf = it & 1u;
+        // the epilogue must have drained this accumulator buffer (tile it - 2)
+        ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t tacc = tmem_base + buf * uint32_t(BN);
+        uint32_t acc = 0;
+        for (int kb = 0; kb < tc.num_kb; ++kb) {
+          ok = mbar_wait_addr(full0 + 8u * s, ph);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-        for (int j = 0; j < GEMM_BK / 16; ++j) {
-          umma_f16_lohi(tmem_base, dA_lo + j * stepA, dA_hi, dB_lo + j * stepB, dB_hi, idesc, acc);
-          acc = 1;
+          for (int j = 0; j < GEMM_BK / 16; ++j) {
+            umma_f16_lohi(tacc, dA_lo + j * stepA, dA_hi, dB_lo + j * stepB, dB_hi, idesc, acc);
+            acc = 1;
+          }
+          umma_commit_addr(empty0 + 8u * s);   // frees the stage once these MMAs have read it
+          dA_lo += uint32_t(SM::STAGE_BYTES >> 4);
+          dB_lo += uint32_t(SM::STAGE_BYTES >> 4);
+          if (++s == uint32_t(S)) {
+            s = 0;
+            ph ^= 1u;
+            dA_lo = uint32_t(dA);
+            dB_lo = uint32_t(dB);
+          }
         }
-        umma_commit_addr(empty0 + 8u * s);   // frees the stage once these MMAs have read it
-        dA_lo += uint32_t(SM::STAGE_BYTES >> 4);
-        dB_lo += uint32_t(SM::STAGE_BYTES >> 4);
-        if (++s == uint32_t(S)) {
-          s = 0;
-          ph ^= 1u;
-          dA_lo = uint32_t(dA);
-          dB_lo = uint32_t(dB);
-        }
+        umma_commit_addr(accf0 + 8u * buf);    // accumulator complete (also releases the epilogue on error)
       }
       if (!ok) atomicExch(p.status, 2);
-      umma_commit(acc_bar);           // accumulator complete (also releases the epilogue on error)
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -461,40 +499,53 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     float* tile = epi_tile + q * (32 * EPI_PITCH);
     const int sub_row = lane >> 3;        // 0..3
     const int sub_col = (lane & 7) * 4;   // 0,4,..,28
-    const int row0 = tm.m0 + q * 32;
-    const bool split = p.splits > 1;
+    constexpr bool split = SPLITK;
     constexpr bool upd = (MODE == EPI_WGRAD_UPDATE);
-    WmRegs cur;
-    if constexpr (upd) {
-      if (!split) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
-    }
-    bool ok = mbar_wait(acc_bar, 0);
-    ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
-    if (!ok && lane == 0) atomicExch(p.status, 3);
-    tc_fence_after();
-    const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
-    float* part = split ? p.partial + (size_t(tile_id) * p.splits + blockIdx.z) * (size_t(GEMM_BM) * BN) : nullptr;
-    if (ok) {
+    const uint32_t accf0 = smem_u32(accf_bar), acce0 = smem_u32(acce_bar);
+    bool ok = true;
+    uint32_t it = 0;
+    for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x, ++it) {
+      const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
+      const TileMap& tm = tc.tm;
+      const uint32_t buf = it & 1u;
+      const uint32_t tacc = tmem_base + buf * uint32_t(BN);
+      const int row0 = tm.m0 + q * 32;
+      WmRegs cur;
+      if constexpr (upd && !split) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
+      ok = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
+      ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
+      if (!ok) {
+        if (lane == 0) atomicExch(p.status, 3);
+        break;
+      }
+      tc_fence_after();
+      float* part = split ? p.partial + (size_t(tc.tile_id) * p.splits + tc.z) * (size_t(GEMM_BM) * BN) : nullptr;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         __syncwarp();
-        if (num_kb > 0) {
-          tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+        if (tc.num_kb > 0) {
+          tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
           tmem_ld_wait();
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) r[j] = 0u;     // a split without k-blocks contributes zero
+        }
+        if (c == BN / 32 - 1) {
+          // last read of this accumulator buffer: hand it back to the MMA issuer
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acce_bar[buf]);
         }
 #pragma unroll
         for (int g = 0; g < 8; ++g)
           *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
         __syncwarp();
         const int n = tm.n0 + c * 32 + sub_col;
-        if (split) {
+        if constexpr (split) {
 #pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + sub_row;
+          for (int i8 = 0; i8 < 8; ++i8) {
+            const int rr = i8 * 4 + sub_row;
             const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
             __stcg(reinterpret_cast<float4*>(part + size_t(q * 32 + rr) * BN + c * 32 + sub_col), acc);
           }
@@ -505,57 +556,58 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           cur = nxt;
         } else {
 #pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + sub_row;
+          for (int i8 = 0; i8 < 8; ++i8) {
+            const int rr = i8 * 4 + sub_row;
             const int row = tile_row(p, tm, q * 32 + rr);
             const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
             if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc);
           }
         }
       }
-    }
-    if (split) {
-      // all four epilogue warps have written their part of the partial tile: publish it, and
-      // let the last CTA of this tile reduce the partials in split order
-      volatile uint32_t* is_last = tmem_slot + 1;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (threadIdx.x == 64) {
-        __threadfence();
-        const unsigned prev = atomicAdd(p.tile_counter + tile_id, 1u);
-        const bool last = (prev == unsigned(p.splits) - 1u);
-        if (last) p.tile_counter[tile_id] = 0u;          // ready for the next launch
-        *is_last = last ? 1u : 0u;
-        __threadfence();
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*is_last != 0u) {
-        const float* base = p.partial + size_t(tile_id) * p.splits * (size_t(GEMM_BM) * BN);
-        const size_t zstride = size_t(GEMM_BM) * BN;
+      if constexpr (split) {
+        // all four epilogue warps have written their part of the partial tile: publish it, and
+        // let the last CTA of this tile reduce the partials in split order
+        volatile uint32_t* is_last = tmem_slot + 1;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64) {
+          __threadfence();
+          const unsigned prev = atomicAdd(p.tile_counter + tc.tile_id, 1u);
+          const bool last = (prev == unsigned(p.splits) - 1u);
+          if (last) p.tile_counter[tc.tile_id] = 0u;          // ready for the next launch
+          *is_last = last ? 1u : 0u;
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*is_last != 0u) {
+          const float* base = p.partial + size_t(tc.tile_id) * p.splits * (size_t(GEMM_BM) * BN);
+          const size_t zstride = size_t(GEMM_BM) * BN;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          const int n = tm.n0 + c * 32 + sub_col;
-          // eight independent rows per lane: their loads are issued together for every split,
-          // the additions keep split order
-          float4 acc[8];
+          for (int c = 0; c < BN / 32; ++c) {
+            const int n = tm.n0 + c * 32 + sub_col;
+            // eight independent rows per lane: their loads are issued together for every split,
+            // the additions keep split order
+            float4 acc[8];
 #pragma unroll
-          for (int it = 0; it < 8; ++it)
-            acc[it] = __ldcg(reinterpret_cast<const float4*>(base + size_t(q * 32 + it * 4 + sub_row) * BN + c * 32 + sub_col));
-          for (int z = 1; z < p.splits; ++z) {
-            float4 t[8];
+            for (int i8 = 0; i8 < 8; ++i8)
+              acc[i8] = __ldcg(reinterpret_cast<const float4*>(base + size_t(q * 32 + i8 * 4 + sub_row) * BN + c * 32 + sub_col));
+            for (int z = 1; z < p.splits; ++z) {
+              float4 tt[8];
 #pragma unroll
-            for (int it = 0; it < 8; ++it)
-              t[it] = __ldcg(reinterpret_cast<const float4*>(base + z * zstride + size_t(q * 32 + it * 4 + sub_row) * BN + c * 32 + sub_col));
+              for (int i8 = 0; i8 < 8; ++i8)
+                tt[i8] = __ldcg(reinterpret_cast<const float4*>(base + z * zstride + size_t(q * 32 + i8 * 4 + sub_row) * BN + c * 32 + sub_col));
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
-              acc[it].x += t[it].x; acc[it].y += t[it].y; acc[it].z += t[it].z; acc[it].w += t[it].w;
+              for (int i8 = 0; i8 < 8; ++i8) {
+                acc[i8].x += tt[i8].x; acc[i8].y += tt[i8].y; acc[i8].z += tt[i8].z; acc[i8].w += tt[i8].w;
+              }
+            }
+#pragma unroll
+            for (int i8 = 0; i8 < 8; ++i8) {
+              const int row = tile_row(p, tm, q * 32 + i8 * 4 + sub_row);
+              if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc[i8]);
             }
           }
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int row = tile_row(p, tm, q * 32 + it * 4 + sub_row);
-            if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc[it]);
-          }
         }
+        asm volatile("bar.sync 1, 128;" ::: "memory");     // is_last is rewritten by the next tile
       }
     }
   }
@@ -563,7 +615,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, BN);
+    tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
