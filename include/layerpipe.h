@@ -212,7 +212,8 @@ long long lp_kernel_launches(lp_handle h);
 /* Tuning hook for experiments: force the GEMM tile width (64, 128, 256, or 512 = 256 x 256 tile on an
  * SM pair with tcgen05 cta_group::2, plain matrices only; 0 = automatic), the
  * shared-memory pipeline depth (0 = automatic) and the split-K factor of the forward / delta
- * contractions (0 = automatic, 1 = off) for handles created afterwards. */
+ * contractions (0 = automatic, 1 = off; adding 256 forces one tile per CTA, adding 512 forces
+ * persistent CTAs that loop over tiles) for handles created afterwards. */
 int lp_set_tuning(int tile_n, int stages, int split_k);
 
 const char* lp_last_error(lp_handle h); /* valid until the next call on h; h may be NULL */

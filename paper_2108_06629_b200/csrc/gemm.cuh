@@ -89,6 +89,7 @@ struct GemmArgs {
   float* partial;           // [tiles][splits][128][BN]
   unsigned* tile_counter;   // [tiles], zero between launches
   ConvGeom g;
+  int persistent;           // CTAs loop over tiles (grid sized to the machine) instead of one tile each
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -266,7 +267,9 @@ struct GemmSmem {
   static constexpr int B_BYTES = BN * GEMM_BK * 2;
   static constexpr int STAGE_BYTES = GEMM_A_BYTES + B_BYTES;
   // pipeline stages, barriers (256 B), the epilogue's staging tiles, alignment slack
-  static constexpr size_t bytes(int stages) { return size_t(stages) * STAGE_BYTES + 256 + EPI_TILE_BYTES + 1024; }
+  static constexpr size_t bytes(int stages, bool persistent) {
+    return size_t(stages) * STAGE_BYTES + 256 + (persistent ? EPI_TILE_BYTES : 0) + 1024;
+  }
 };
 
 // One output tile (and, with split-K, one slice of its contraction) of the launch.
@@ -311,7 +314,7 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmArgs& p, int t, int til
 // tiles b, b + gridDim.x, ...  The accumulator is double-buffered in tensor memory (2 x BN
 // columns) so that the epilogue of one tile overlaps the main loop of the next, and the
 // shared-memory pipeline runs on across tile boundaries.
-template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK>
+template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK, bool PERSIST>
 __global__ void __launch_bounds__(GEMM_THREADS, BN <= 128 ? 2 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmArgs p, const int tiles_m, const int tiles_n, const int total_work) {
@@ -324,7 +327,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;     // [2] accumulator buffer full  (MMA -> epilogue)
   uint64_t* acce_bar = accf_bar + 2;                    // [2] accumulator buffer empty (epilogue -> MMA)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce_bar + 2);
-  float* epi_tile = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + 256);
+  // Staging tiles of the epilogue.  With one tile per CTA they reuse pipeline stage 0 (by the time
+  // the accumulator barrier fires every load has landed and every MMA has read its operands);
+  // a CTA that loops over tiles keeps loading while the epilogue runs and needs its own space.
+  float* epi_tile = PERSIST ? reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + 256)
+                            : reinterpret_cast<float*>(smem);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -343,7 +350,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 2 * BN);
+    tmem_alloc(tmem_slot, PERSIST ? 2 * BN : BN);     // a second accumulator only when tiles follow one another
     tmem_relinquish();
   }
   tc_fence_before();
@@ -362,7 +369,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t smem0 = smem_u32(smem);
       const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
       uint32_t s = 0, ph = 0;
-      for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x) {
+      for (int t = blockIdx.x; t < total_work && ok; t += (PERSIST ? int(gridDim.x) : total_work)) {
         const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
         const TileMap& tm = tc.tm;
         // running position of the contraction
@@ -456,13 +463,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t dA_lo = uint32_t(dA), dB_lo = uint32_t(dB);
       bool ok = true;
       uint32_t it = 0;     // tiles done by this CTA
-      for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x, ++it) {
+      for (int t = blockIdx.x; t < total_work && ok; t += (PERSIST ? int(gridDim.x) : total_work), ++it) {
         const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
-        const uint32_t buf = it & 1u;
-        // the epilogue must have drained this accumulator buffer (tile it - 2)
-        ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u);
-        if (!ok) break;
-        tc_fence_after();
+        const uint32_t buf = PERSIST ? (it & 1u) : 0u;
+        if (PERSIST) {
+          // the epilogue must have drained this accumulator buffer (tile it - 2)
+          ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u);
+          if (!ok) break;
+          tc_fence_after();
+        }
         const uint32_t tacc = tmem_base + buf * uint32_t(BN);
         uint32_t acc = 0;
         for (int kb = 0; kb < tc.num_kb; ++kb) {
@@ -504,10 +513,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t accf0 = smem_u32(accf_bar), acce0 = smem_u32(acce_bar);
     bool ok = true;
     uint32_t it = 0;
-    for (int t = blockIdx.x; t < total_work && ok; t += gridDim.x, ++it) {
+    for (int t = blockIdx.x; t < total_work && ok; t += (PERSIST ? int(gridDim.x) : total_work), ++it) {
       const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
       const TileMap& tm = tc.tm;
-      const uint32_t buf = it & 1u;
+      const uint32_t buf = PERSIST ? (it & 1u) : 0u;
       const uint32_t tacc = tmem_base + buf * uint32_t(BN);
       const int row0 = tm.m0 + q * 32;
       WmRegs cur;
@@ -531,7 +540,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int j = 0; j < 32; ++j) r[j] = 0u;     // a split without k-blocks contributes zero
         }
-        if (c == BN / 32 - 1) {
+        if (PERSIST && c == BN / 32 - 1) {
           // last read of this accumulator buffer: hand it back to the MMA issuer
           tc_fence_before();
           __syncwarp();
@@ -615,7 +624,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * BN);
+    tmem_dealloc(tmem_base, PERSIST ? 2 * BN : BN);
   }
 }
 

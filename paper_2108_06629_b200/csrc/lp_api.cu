@@ -766,7 +766,7 @@ extern "C" const char* lp_last_error(lp_handle h) { return h ? h->err.c_str() : 
 
 extern "C" int lp_set_tuning(int tile_n, int stages, int split_k) {
   if ((tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256 && tile_n != GEMM_BN_PAIR) || stages < 0 || stages > GEMM_MAX_STAGES ||
-      split_k < 0 || split_k > 64)
+      split_k < 0 || (split_k & 0xFF) > 64 || (split_k >> 10) != 0)
     return LP_ERR_INVALID_ARG;
   gemm_set_tuning(tile_n, stages, split_k);
   return LP_OK;
