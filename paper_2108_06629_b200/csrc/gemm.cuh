@@ -90,6 +90,7 @@ struct GemmArgs {
   unsigned* tile_counter;   // [tiles], zero between launches
   ConvGeom g;
   int persistent;           // CTAs loop over tiles (grid sized to the machine) instead of one tile each
+  int l2_ahead;             // plain GEMM: k-blocks of the B operand to pull into L2 ahead of the pipeline (0 = off)
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -388,7 +389,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           dh = tc.tap / p.g.S - p.g.pad;
           dw = tc.tap % p.g.S - p.g.pad;
         }
+        // Weight streaming (small batch): the shared-memory pipeline holds only S k-blocks, not
+        // enough to cover an HBM round trip, so the B operand is additionally requested into L2
+        // l2_ahead k-blocks early; the pipeline then runs at L2-hit latency.
+        const int ahead = (p.g.kind == GEOM_PLAIN) ? p.l2_ahead : 0;
+        for (int kb = 0; kb < min(ahead, tc.num_kb); ++kb) {
+          const int kk = (tc.kb_begin + kb) * GEMM_BK;
+          if (B_MN) {
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c) tma_prefetch_l2_2d(&tmB, tm.n0 + c * 64, kk);
+          } else {
+            tma_prefetch_l2_2d(&tmB, kk, tm.n0);
+          }
+        }
         for (int kb = 0; kb < tc.num_kb; ++kb) {
+          if (ahead > 0 && kb + ahead < tc.num_kb) {
+            const int kk = k0 + ahead * GEMM_BK;
+            if (B_MN) {
+#pragma unroll
+              for (int c = 0; c < BN / 64; ++c) tma_prefetch_l2_2d(&tmB, tm.n0 + c * 64, kk);
+            } else {
+              tma_prefetch_l2_2d(&tmB, kk, tm.n0);
+            }
+          }
           ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
           if (!ok) break;
           const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
@@ -520,7 +543,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t tacc = tmem_base + buf * uint32_t(BN);
       const int row0 = tm.m0 + q * 32;
       WmRegs cur;
-      if constexpr (upd && !split) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
+      if constexpr (upd && !split) {
+        // Pull this warp's 32 rows of the master (and momentum) tile into L2 while the main loop
+        // runs: the register prefetch below only reaches one chunk ahead, and an L2 hit costs a
+        // fraction of an HBM round trip.
+        constexpr int SEGS = BN * 4 / 128;               // 128-byte lines per tile row
+        for (int i = lane; i < 32 * SEGS; i += 32) {
+          const int row = row0 + i / SEGS, col = tm.n0 + (i % SEGS) * 32;
+          if (row < p.M && col < tm.nlim) {
+            const size_t off = size_t(row) * p.ld_out + col;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.W + off));
+            if (p.mW != nullptr) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.mW + off));
+          }
+        }
+        load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
+      }
       ok = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
       ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
       if (!ok) {
