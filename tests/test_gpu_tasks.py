@@ -17,13 +17,13 @@ from gpu_common import assert_bf16_close, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None, fused=True):
+def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None, fused=True, bias=True):
     from oracle import layerpipe_oracle as O
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
     W0, b0 = I.initial_weights(layers, 0)
     rng = np.random.default_rng(5)
-    b0 = [rng.standard_normal(b.shape).astype(np.float32) * 0.1 for b in b0]   # exercise the bias path
+    b0 = [rng.standard_normal(b.shape).astype(np.float32) * 0.1 if bias else None for b in b0]   # exercise the bias path
     flags = lpb.LP_CAPTURE_GRADS | (0 if fused else lpb.LP_UNFUSED_UPDATE)
     tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, flags=flags, W0=W0, b0=b0)
     delays = tr.get_schedule()[1]
@@ -37,9 +37,9 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
     for n in range(steps):
         x, y = I.minibatch(layers, batch, n)
         pre_W = [w.copy() for w in orc.W]
-        pre_b = [b.copy() for b in orc.b]
+        pre_b = [None if b is None else b.copy() for b in orc.b]
         pre_mW = [m.copy() for m in orc.mW]
-        pre_mb = [m.copy() for m in orc.mb]
+        pre_mb = [None if m is None else m.copy() for m in orc.mb]
         stash = [dict(s) for s in orc.stash]
         rec = orc.step(x, y, capture=True)
         if check_steps is not None and n not in check_steps:
@@ -49,7 +49,8 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
         for l in range(L):
             Wv, bv = stash[l][rec["v"][l]]
             tr.debug_write("ring_w", l, slot[l], Wv)
-            tr.debug_write("ring_b", l, slot[l], bv)
+            if bias:
+                tr.debug_write("ring_b", l, slot[l], bv)
         tr.debug_write("labels", 0, n, y.astype(np.float32))
         # forward tasks
         for l in range(L):
@@ -88,10 +89,12 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                                                 "delta^%d step %d" % (l - 1, n)))
             # pre-update state of the oracle; with the fused update the G kernel itself applies Eq. 6
             tr.debug_write("master_w", l, 0, pre_W[l])
-            tr.debug_write("master_b", l, 0, pre_b[l])
+            if bias:
+                tr.debug_write("master_b", l, 0, pre_b[l])
             if mu != 0.0:
                 tr.debug_write("mom_w", l, 0, pre_mW[l])
-                tr.debug_write("mom_b", l, 0, pre_mb[l])
+                if bias:
+                    tr.debug_write("mom_b", l, 0, pre_mb[l])
             tr.debug_run_task("G", l, n)
             r = rel_l2(tr.debug_read("grad_w", l, 0), rec["dW"][l])
             assert r < 2e-5, ("G", l, n, r)
@@ -99,20 +102,23 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
             if not fused:
                 tr.debug_write("grad_w", l, 0, rec["dW"][l])      # Eq. 6 from the oracle's gradient
             tr.debug_run_task("update", l, n)
-            r = rel_l2(tr.debug_read("grad_b", l, 0), rec["db"][l])
-            assert r < 2e-5, ("db", l, n, r)
-            note("db", r)
+            if bias:
+                r = rel_l2(tr.debug_read("grad_b", l, 0), rec["db"][l])
+                assert r < 2e-5, ("db", l, n, r)
+                note("db", r)
             dWn = np.linalg.norm(rec["dW"][l])
             step_err = np.linalg.norm(tr.debug_read("master_w", l, 0) - orc.W[l]) / max(lr * dWn, 1e-30)
             assert step_err < 1e-3, ("update of W relative to the step taken", l, n, step_err)
-            assert rel_l2(tr.debug_read("master_b", l, 0), orc.b[l]) < 1e-5
+            if bias:
+                assert rel_l2(tr.debug_read("master_b", l, 0), orc.b[l]) < 1e-5
             if mu != 0.0:
                 assert rel_l2(tr.debug_read("mom_w", l, 0), orc.mW[l]) < 1e-6
             new_slot = (n + 1) % (delays[l] + 1)
             Wq, bq = orc.stash[l][n + 1]
             note("ring", assert_bf16_close(tr.debug_read("ring_w", l, new_slot), Wq, "ring W^%d step %d" % (l, n),
                                            min_equal=0.995))
-            assert rel_l2(tr.debug_read("ring_b", l, new_slot), bq) < 1e-5
+            if bias:
+                assert rel_l2(tr.debug_read("ring_b", l, new_slot), bq) < 1e-5
     rc, detail = tr.device_status()
     assert rc == 0, detail
     tr.close()
@@ -186,6 +192,18 @@ def test_tasks_sm_pair_tiles():
         run_teacher_forced(layers, 300, 3, [2, 1, 0], 0.05, 0.9, 4)
     finally:
         lpb.lp_set_tuning(0, 0, 0)
+
+
+def test_tasks_degenerate_shapes():
+    """The paper's bias-free Eq. 1; a single layer (no delta task at all); batch 1; one stage with
+    all delays zero (plain backpropagation); a delay larger than the number of steps run."""
+    from paper_2108_06629_b200 import inputs as I
+    nobias = [dict(l, bias=False) for l in I.mlp([72, 40, 24], "relu")]
+    run_teacher_forced(nobias, 24, 2, [1, 0], 0.05, 0.9, 4, bias=False)
+    run_teacher_forced(I.mlp([40, 16], "relu"), 8, 1, [0], 0.05, 0.0, 3)
+    run_teacher_forced(I.mlp([24, 16, 8], "gelu"), 1, 2, [1, 0], 0.05, 0.0, 3)
+    run_teacher_forced(I.mlp([64, 48, 32, 8], "gelu"), 16, 1, [0, 0, 0], 0.05, 0.9, 3)
+    run_teacher_forced(I.mlp([64, 48, 8], "relu"), 16, 2, [9, 0], 0.05, 0.0, 3)
 
 
 def test_tasks_papers_double_delay_convention():

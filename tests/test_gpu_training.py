@@ -144,6 +144,29 @@ def test_free_running_vgg_small_32_full_config():
     # bf16 spacing task by task in test_gpu_tasks.py.)
 
 
+def test_bf16_input_equals_fp32_input_of_the_same_values():
+    """lp_step accepts the minibatch as bf16 as well; values that are already bf16 must give the
+    same bits as their fp32 copies."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([136, 72, 24], "gelu")
+    W0, b0 = I.initial_weights(layers, 0)
+    outs = []
+    for dt in (lpb.LP_F32, lpb.LP_BF16):
+        tr = lpb.Trainer(layers, 20, 2, delays=[1, 0], lr=0.05, momentum=0.9, input_dtype=dt, W0=W0, b0=b0)
+        for n in range(4):
+            x, y = I.minibatch(layers, 20, n)
+            xb = torch.from_numpy(x).cuda().bfloat16()
+            tr.step(xb if dt == lpb.LP_BF16 else xb.float(), torch.from_numpy(y).cuda())
+        tr.flush()
+        torch.cuda.synchronize()
+        outs.append([tr.get_weights(l)[0] for l in range(2)] + [tr.get_loss(3)])
+        tr.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    assert outs[0][2] == outs[1][2]
+
+
 def test_fused_and_unfused_update_agree():
     """The fused epilogue and the separate update kernel evaluate the same expressions on the
     same fp32 accumulators: the two trajectories must be bit-identical."""
