@@ -49,6 +49,8 @@ int plan_layers(const lp_layer* layers, int L, int batch, int Np, PlanResult* ou
 // ---- elementwise.cu ---------------------------------------------------------
 cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
                               int* labels_copy, int rows, int B, int n_in, int ld, cudaStream_t stream);
+cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                                 int* labels_copy, int B, int H, int W, int C, int ld, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
                                 cudaStream_t stream);

@@ -60,6 +60,76 @@ cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* l
 }
 
 // ---------------------------------------------------------------------------
+// First convolution layer with very few input channels (an RGB image): a^0 is stashed as the
+// matrix of 3x3 patches, one row per output pixel, column (r*3 + s)*C + ch = the input at
+// (h + r - 1, w + s - 1, ch) or zero outside the image, padded with zero columns to `ld`.  The
+// layer's contractions (Eq. 1 and Eq. 5 written for a convolution) then run as plain GEMMs over
+// 9*C columns instead of nine taps of a 64-wide k-block that would be 95 % padding.
+// One thread per output pixel; C is a template parameter so that the 9*C gathered values stay in
+// registers and the column arithmetic folds at compile time.
+template <int C>
+__global__ void cast_patch3x3_kernel(const void* __restrict__ batch, int input_is_bf16,
+                                     const int* __restrict__ labels, __nv_bfloat16* __restrict__ x0,
+                                     int* __restrict__ labels_copy, int B, int H, int W) {
+  constexpr int LD = (9 * C + 7) / 8 * 8;
+  const int total = B * H * W;
+  for (int pix = blockIdx.x * blockDim.x + threadIdx.x; pix < total; pix += gridDim.x * blockDim.x) {
+    const int w = pix % W;
+    const int h = (pix / W) % H;
+    float v[LD];
+#pragma unroll
+    for (int k = 0; k < LD; ++k) v[k] = 0.f;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const int hh = h + r - 1;
+      if (hh < 0 || hh >= H) continue;
+#pragma unroll
+      for (int s = 0; s < 3; ++s) {
+        const int ww = w + s - 1;
+        if (ww < 0 || ww >= W) continue;
+        const long long idx = ((long long)pix + (r - 1) * W + (s - 1)) * C;
+#pragma unroll
+        for (int ch = 0; ch < C; ++ch)
+          v[(r * 3 + s) * C + ch] = input_is_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(batch)[idx + ch])
+                                                  : reinterpret_cast<const float*>(batch)[idx + ch];
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(x0 + (long long)pix * LD);
+#pragma unroll
+    for (int g = 0; g < LD / 8; ++g) {
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(v[8 * g + 0], v[8 * g + 1]);
+      __nv_bfloat162 p1 = __floats2bfloat162_rn(v[8 * g + 2], v[8 * g + 3]);
+      __nv_bfloat162 p2 = __floats2bfloat162_rn(v[8 * g + 4], v[8 * g + 5]);
+      __nv_bfloat162 p3 = __floats2bfloat162_rn(v[8 * g + 6], v[8 * g + 7]);
+      uint4 o;
+      o.x = *reinterpret_cast<uint32_t*>(&p0);
+      o.y = *reinterpret_cast<uint32_t*>(&p1);
+      o.z = *reinterpret_cast<uint32_t*>(&p2);
+      o.w = *reinterpret_cast<uint32_t*>(&p3);
+      dst[g] = o;
+    }
+  }
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i < B; i += blockDim.x) labels_copy[i] = labels[i];
+  }
+}
+
+cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                                 int* labels_copy, int B, int H, int W, int C, int ld, cudaStream_t stream) {
+  const long long total = (long long)B * H * W;
+  if (C < 1 || C > 7 || ld != (9 * C + 7) / 8 * 8 || total >= (1ll << 31)) return cudaErrorInvalidValue;
+  int blocks = int(std::min<long long>((total + 255) / 256, 148 * 8));
+  if (blocks < 1) blocks = 1;
+#define LP_PATCH_CASE(c)                                                                                        \
+  case c: cast_patch3x3_kernel<c><<<blocks, 256, 0, stream>>>(batch, input_is_bf16, labels, x0, labels_copy, B, H, W); break;
+  switch (C) {
+    LP_PATCH_CASE(1) LP_PATCH_CASE(2) LP_PATCH_CASE(3) LP_PATCH_CASE(4) LP_PATCH_CASE(5) LP_PATCH_CASE(6) LP_PATCH_CASE(7)
+  }
+#undef LP_PATCH_CASE
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
 // One block per row: p = softmax(z^L), delta^L = RN((p - onehot)/B), row loss; the last
 // block to finish adds the row losses in row order (deterministic mean).
 __device__ __forceinline__ float block_reduce(float v, float* sh, bool is_max) {

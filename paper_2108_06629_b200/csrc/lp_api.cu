@@ -55,6 +55,11 @@ struct Layer {
   // out_rows = B*H*W; weights are the matrix [Cout][9 * ld_in] (tap-major, padded channels).
   bool conv = false;
   int imH = 1, imW = 1, taps = 1;
+  // First convolution layer with few input channels (9 * Cin <= 64): the stash holds 3x3 patches
+  // [B*H*W][9 * Cin] and the layer runs as a plain GEMM over pixel rows; n_in = 9 * Cin, taps = 1,
+  // c_in = the image's channel count.
+  bool patch = false;
+  int c_in = 0;
   int in_rows = 0, out_rows = 0;
   int w_rows = 0, w_ld = 0;          // weight matrix [w_rows][w_ld]
   int pool = 0, Hp = 1, Wp = 1;      // 2x2 max pool after the activation: pooled image size
@@ -306,6 +311,8 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     y.conv = layers[l].kind == LP_CONV;
     if (y.conv) {
       y.imH = layers[l].H; y.imW = layers[l].W; y.taps = 9;
+      y.patch = (l == 0 && 9 * y.n_in <= 64);
+      if (y.patch) { y.c_in = y.n_in; y.n_in = 9 * y.c_in; y.ld_in = pad8(y.n_in); y.taps = 1; }
       y.in_rows = y.out_rows = B * y.imH * y.imW;
       y.w_rows = y.n_out; y.w_ld = y.taps * y.ld_in;
       y.pool = layers[l].pool;
@@ -321,7 +328,8 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       // pixel range until about two CTAs per SM exist
       const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
       const int num_kb = y.in_rows / GEMM_BK;
-      y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), num_kb / 8), 64));
+      // (the patch layer has a single tile: one CTA per SM, each a long run of small k-blocks)
+      y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), num_kb / 8), y.patch ? 148 : 64));
       const int per = (num_kb + y.split_g - 1) / y.split_g;
       y.split_g = (num_kb + per - 1) / per;
     } else {
@@ -393,7 +401,7 @@ static int build_tensor_maps(lp_ctx* c) {
     y.tm_d_B.resize(y.slots);
     y.tm_g_A.resize(kDeltaSlots);
     y.tm_g_B.resize(y.x_slots);
-    if (y.conv) {
+    if (y.conv && !y.patch) {
       // forward: A = a^{l-1} as NHWC boxes of 128 pixels; B = W [Cout][9 * ld_in] K-major
       // delta:   A = delta^l as NHWC boxes of 128 pixels; B = the same W matrix read MN-major
       // G:       A = delta^l, B = a^{l-1}, both as NHWC boxes of 64 pixels (the contraction index)
@@ -417,10 +425,11 @@ static int build_tensor_maps(lp_ctx* c) {
       }
       continue;
     }
+    // (fully connected layers, and the patch layer whose rows are pixels)
     // forward: A = a^{l-1} [B][in] K-major; B = W [out][in] K-major
     gemm_box_dims(0, y.bn_f, bA, bB);
     for (int s = 0; s < y.x_slots; ++s)
-      if ((rc = make_tmap_bf16_2d(&y.tm_f_A[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bA[0], bA[1], &err)) != LP_OK)
+      if ((rc = make_tmap_bf16_2d(&y.tm_f_A[s], y.X + s * y.x_elems, y.n_in, y.in_rows, y.ld_in, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
     for (int s = 0; s < y.slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
@@ -428,7 +437,7 @@ static int build_tensor_maps(lp_ctx* c) {
     // delta: A = delta^l [B][out] K-major (K = out); B = W [out][in] MN-major (N = in contiguous)
     gemm_box_dims(1, y.bn_d, bA, bB);
     for (int s = 0; s < kDeltaSlots; ++s)
-      if ((rc = make_tmap_bf16_2d(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
+      if ((rc = make_tmap_bf16_2d(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.n_out, y.out_rows, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
     for (int s = 0; s < y.slots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
@@ -436,10 +445,10 @@ static int build_tensor_maps(lp_ctx* c) {
     // G: A = delta^l stored [B][out] -> MN-major (M = out contiguous); B = a^{l-1} stored [B][in] -> MN-major
     gemm_box_dims(2, y.bn_g, bA, bB);
     for (int s = 0; s < kDeltaSlots; ++s)
-      if ((rc = make_tmap_bf16_2d(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.n_out, B, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
+      if ((rc = make_tmap_bf16_2d(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.n_out, y.out_rows, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
         return fail(c, rc, err);
     for (int s = 0; s < y.x_slots; ++s)
-      if ((rc = make_tmap_bf16_2d(&y.tm_g_B[s], y.X + s * y.x_elems, y.n_in, B, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
+      if ((rc = make_tmap_bf16_2d(&y.tm_g_B[s], y.X + s * y.x_elems, y.n_in, y.in_rows, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
   }
   return LP_OK;
@@ -501,7 +510,7 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   const bool last = (l == nL - 1);
   GemmArgs a{};
   a.M = y.out_rows; a.N = y.n_out; a.K = y.n_in;
-  if (y.conv) {
+  if (y.conv && !y.patch) {
     const int cpt = (y.ld_in + 63) / 64;
     a.K = y.taps * cpt * GEMM_BK;
     a.g = conv_geom(y, GEOM_PIX_M, y.box128, 0, cpt, 0);
@@ -594,13 +603,11 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
   GemmArgs a{};
   a.M = y.n_out; a.N = y.w_ld; a.K = y.in_rows;
-  if (!y.conv) a.N = y.n_in;
+  if (!y.conv || y.patch) a.N = y.n_in;
   a.ld_out = y.w_ld;
   a.status = c->status;
-  if (y.conv) {
-    a.g = conv_geom(y, GEOM_PIX_K, y.box64, 0, 0, (y.ld_in + y.bn_g - 1) / y.bn_g);
-    a.splits = y.split_g; a.partial = y.part_g; a.tile_counter = y.cnt_g;
-  }
+  if (y.conv && !y.patch) a.g = conv_geom(y, GEOM_PIX_K, y.box64, 0, 0, (y.ld_in + y.bn_g - 1) / y.bn_g);
+  if (y.split_g > 1) { a.splits = y.split_g; a.partial = y.part_g; a.tile_counter = y.cnt_g; }
   if (fused_update(c)) {
     // Eq. 5 and Eq. 6 in one kernel: the accumulator tile is G; the epilogue reads the fp32
     // master (and momentum) tile, applies the update and writes master, momentum and the
@@ -826,9 +833,14 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     LP_CUDA(c, task_begin(c, user, {}, {rx, rl}));
     ++c->launches;
     TimedScope ts(c, LP_TASK_CAST, user);
-    LP_CUDA(c, launch_cast_stash(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
-                                 y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, y0.in_rows, B,
-                                 y0.n_in, y0.ld_in, user));
+    if (y0.patch)
+      LP_CUDA(c, launch_cast_patch3x3(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
+                                      y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.imH,
+                                      y0.imW, y0.c_in, y0.ld_in, user));
+    else
+      LP_CUDA(c, launch_cast_stash(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
+                                   y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, y0.in_rows, B,
+                                   y0.n_in, y0.ld_in, user));
     LP_CUDA(c, task_end(c, user, {}, {rx, rl}, nullptr));
   }
   // ---- forward ---------------------------------------------------------------
@@ -1021,10 +1033,42 @@ static inline uint16_t f32_to_bf16_rn(float f) {
   u += 0x7FFFu + ((u >> 16) & 1u);
   return uint16_t(u >> 16);
 }
+// The patch layer's stash seen from the host as the image it was built from, NHWC [B][H][W][Cin]:
+// a write builds every pixel's 3x3 patch row, a read returns the centre tap.
+static int patch_io(lp_ctx* h, long long index, const float* in_host, float* out_host) {
+  Layer& y = h->L[0];
+  const int B = h->cfg.batch, H = y.imH, W = y.imW, C = y.c_in, ld = y.ld_in;
+  __nv_bfloat16* dev = y.X + size_t(index % y.x_slots) * y.x_elems;
+  std::vector<uint16_t> tmp(y.x_elems, 0);
+  LP_CUDA(h, cudaDeviceSynchronize());
+  if (out_host) {
+    LP_CUDA(h, cudaMemcpy(tmp.data(), dev, tmp.size() * 2, cudaMemcpyDeviceToHost));
+    for (size_t pix = 0; pix < size_t(B) * H * W; ++pix)
+      for (int ch = 0; ch < C; ++ch) {
+        const uint32_t bits = uint32_t(tmp[pix * ld + 4 * C + ch]) << 16;
+        memcpy(&out_host[pix * C + ch], &bits, 4);
+      }
+    return LP_OK;
+  }
+  for (int b = 0; b < B; ++b)
+    for (int hh = 0; hh < H; ++hh)
+      for (int ww = 0; ww < W; ++ww) {
+        uint16_t* row = &tmp[((size_t(b) * H + hh) * W + ww) * ld];
+        for (int tap = 0; tap < 9; ++tap) {
+          const int sh = hh + tap / 3 - 1, sw = ww + tap % 3 - 1;
+          if (sh < 0 || sh >= H || sw < 0 || sw >= W) continue;
+          const float* src = in_host + ((size_t(b) * H + sh) * W + sw) * C;
+          for (int ch = 0; ch < C; ++ch) row[tap * C + ch] = f32_to_bf16_rn(src[ch]);
+        }
+      }
+  LP_CUDA(h, cudaMemcpy(dev, tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice));
+  return LP_OK;
+}
 }  // namespace lp
 
 extern "C" int lp_debug_read(lp_handle h, int buffer, int layer, long long index, float* out_host) {
   if (!h || !out_host) return LP_ERR_INVALID_ARG;
+  if (buffer == LP_BUF_INPUT && layer == 0 && index >= 0 && h->L[0].patch) return patch_io(h, index, nullptr, out_host);
   BufView v;
   int rc = locate(h, buffer, layer, index, &v);
   if (rc != LP_OK) return rc;
@@ -1059,6 +1103,7 @@ extern "C" int lp_debug_read(lp_handle h, int buffer, int layer, long long index
 
 extern "C" int lp_debug_write(lp_handle h, int buffer, int layer, long long index, const float* in_host) {
   if (!h || !in_host) return LP_ERR_INVALID_ARG;
+  if (buffer == LP_BUF_INPUT && layer == 0 && index >= 0 && h->L[0].patch) return patch_io(h, index, in_host, nullptr);
   BufView v;
   int rc = locate(h, buffer, layer, index, &v);
   if (rc != LP_OK) return rc;
