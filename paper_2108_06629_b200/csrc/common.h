@@ -22,15 +22,23 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64
 int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
                         uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err);
 
+// fp32 (elem_bytes 4) or bf16 (2) row-major tensor moved in boxes of 32 columns x box_outer rows
+// (the streamed tiles of the fused update).
+int make_tmap_rows32(CUtensorMap* out, const void* base, int elem_bytes, uint64_t inner, uint64_t outer,
+                     uint64_t pitch_elems, uint32_t box_outer, std::string* err);
+
 struct GemmArgs;
+struct UpdMaps;
 constexpr int GEMM_BN_PAIR = 512;   // tile code: 256 x 256 tile computed by a pair of CTAs (cta_group::2)
 // which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
 // Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
 // (see gemm_box_dims).
 int gemm_pick_bn(int which, int M, int N, int K);
 void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]);
+// um (EPI_WGRAD_UPDATE only): tensor maps of the master, momentum and destination ring slot; when
+// given, and the launch qualifies, the update's tiles are streamed by TMA.
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const GemmArgs& args, cudaStream_t stream);
+                        const GemmArgs& args, cudaStream_t stream, const UpdMaps* um = nullptr);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process
 void gemm_set_tuning(int bn, int stages, int splits);   // 0 = automatic
 int gemm_pick_splits(int M, int N, int K, int bn);

@@ -56,6 +56,32 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64
   return LP_OK;
 }
 
+// Row-major 2-D tensor of 4-byte (fp32) or 2-byte (bf16) elements moved in boxes of 32 columns:
+// 128-byte rows with the 128-byte swizzle, or 64-byte rows with the 64-byte swizzle.
+int make_tmap_rows32(CUtensorMap* out, const void* base, int elem_bytes, uint64_t inner, uint64_t outer,
+                     uint64_t pitch_elems, uint32_t box_outer, std::string* err) {
+  EncodeTiledFn fn = get_encode_fn(err);
+  if (!fn) return LP_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || ((pitch_elems * elem_bytes) & 15) || box_outer > 256 ||
+      (elem_bytes != 4 && elem_bytes != 2)) {
+    if (err) *err = "tensor map: base and pitch must be 16-byte aligned, box <= 256";
+    return LP_ERR_INVALID_ARG;
+  }
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {pitch_elems * elem_bytes};
+  cuuint32_t box[2] = {32, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                  const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  elem_bytes == 4 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled (update tile) failed with CUresult " + std::to_string(int(r));
+    return LP_ERR_CUDA;
+  }
+  return LP_OK;
+}
+
 // NHWC bf16 tensor [N][H][W][C] with channel pitch `pitch_c` (multiple of 8): dimensions
 // (C, W, H, N), box (64 channels, bw, bh, bn pixels).  Coordinates outside the tensor read zero.
 int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
@@ -144,7 +170,8 @@ static int sm_count() {
 }
 
 template <int BN, bool A_MN, bool B_MN, int MODE>
-static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
+static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st,
+                              const UpdMaps* um) {
   if (a.splits < 1 || a.partial == nullptr) a.splits = 1;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
@@ -163,19 +190,24 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   const long long slots = (long long)sm_count() * per_sm;
   a.persistent = (work >= 4 * slots && a.kb_per_split <= 96) ? 1 : 0;
   if (g_force_persistent >= 0) a.persistent = g_force_persistent;
+  // fused update streamed by TMA: plain geometry, no split-K, tiles at least 128 columns wide
+  static const UpdMaps no_maps{};
+  a.upd_tma = (MODE == EPI_WGRAD_UPDATE && um != nullptr && a.splits == 1 && BN >= 128 && a.g.kind == GEOM_PLAIN) ? 1 : 0;
+  if (!a.upd_tma) um = &no_maps;
   const int stage_bytes = GEMM_A_BYTES + BN * GEMM_BK * 2;
-  const int avail = (per_sm == 2 ? 113 : 227) * 1024 - 1024 - 256 - 512 - (a.persistent ? EPI_TILE_BYTES : 0);
+  const int tail = a.upd_tma ? 1024 + UPD_RING_BYTES : 256 + (a.persistent ? EPI_TILE_BYTES : 0);
+  const int avail = (per_sm == 2 ? 113 : 227) * 1024 - 1024 - 512 - tail;
   int s = g_force_stages > 0 ? g_force_stages : avail / stage_bytes;
   s = std::max(2, std::min(s, GEMM_MAX_STAGES));
-  if (!a.persistent) s = std::max(2, std::min(s, std::max(a.kb_per_split, 2)));
-  while (s > 2 && size_t(s) * stage_bytes > size_t(227 * 1024 - 1024 - 256 - 512 - EPI_TILE_BYTES)) --s;
+  if (!a.persistent) s = std::max(2, std::min(s, std::max(a.kb_per_split + (a.upd_tma ? BN / 32 : 0), 2)));
+  while (s > 2 && size_t(s) * stage_bytes > size_t(227 * 1024 - 1024 - 512 - 1024 - EPI_TILE_BYTES)) --s;
   a.num_stages = s;
-  const size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0);
+  const size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0, a.upd_tma != 0);
   const int grid = int(a.persistent ? std::min<long long>(work, slots) : work);
   // single-wave launches stream their weights once: request them into L2 well ahead of the pipeline
   a.l2_ahead = (a.g.kind == GEOM_PLAIN && work <= slots && a.kb_per_split >= 8) ? g_l2_ahead : 0;
 #define LP_LAUNCH(SPL, PER) \
-  gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, SPL, PER><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, a, tiles_m, tiles_n, int(work))
+  gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, SPL, PER><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, *um, a, tiles_m, tiles_n, int(work))
   if (a.splits > 1) { if (a.persistent) LP_LAUNCH(true, true); else LP_LAUNCH(true, false); }
   else              { if (a.persistent) LP_LAUNCH(false, true); else LP_LAUNCH(false, false); }
 #undef LP_LAUNCH
@@ -257,7 +289,7 @@ cudaError_t gemm_configure() {
 }
 
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
-                        cudaStream_t st) {
+                        cudaStream_t st, const UpdMaps* um) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
   if (bn == GEMM_BN_PAIR) {
     if (args.g.kind != GEOM_PLAIN) return cudaErrorInvalidValue;
@@ -268,7 +300,7 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
     return cudaErrorInvalidValue;
   }
 #define LP_TRY(BN, A, B, M) \
-  if (bn == BN && a_mn == A && b_mn == B && args.mode == M) return launch_one<BN, A, B, M>(tmA, tmB, args, st);
+  if (bn == BN && a_mn == A && b_mn == B && args.mode == M) return launch_one<BN, A, B, M>(tmA, tmB, args, st, um);
   LP_FOR_EACH_VARIANT(LP_TRY, 64)
   LP_FOR_EACH_VARIANT(LP_TRY, 128)
   LP_FOR_EACH_VARIANT(LP_TRY, 256)

@@ -91,6 +91,7 @@ struct GemmArgs {
   ConvGeom g;
   int persistent;           // CTAs loop over tiles (grid sized to the machine) instead of one tile each
   int l2_ahead;             // plain GEMM: k-blocks of the B operand to pull into L2 ahead of the pipeline (0 = off)
+  int upd_tma;              // EPI_WGRAD_UPDATE: master / momentum / ring tiles move by TMA through the stage ring
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -263,13 +264,25 @@ __device__ __forceinline__ void apply_update(const GemmArgs& p, int row0, int n,
   }
 }
 
+// Tensor maps of the fused update's streamed tiles: fp32 master and momentum (boxes of 32
+// columns x 128 rows, 128-byte swizzle) and the bf16 ring slot being written (same box,
+// 64-byte swizzle).
+struct UpdMaps {
+  CUtensorMap W, M, R;
+};
+constexpr int UPD_CHUNK_BYTES = GEMM_BM * 32 * 4;     // one fp32 chunk: 128 rows x 32 columns (16 KiB)
+constexpr int UPD_RING_BYTES = GEMM_BM * 32 * 2;      // its bf16 image (8 KiB)
+
 template <int BN>
 struct GemmSmem {
   static constexpr int B_BYTES = BN * GEMM_BK * 2;
   static constexpr int STAGE_BYTES = GEMM_A_BYTES + B_BYTES;
-  // pipeline stages, barriers (256 B), the epilogue's staging tiles, alignment slack
-  static constexpr size_t bytes(int stages, bool persistent) {
-    return size_t(stages) * STAGE_BYTES + 256 + (persistent ? EPI_TILE_BYTES : 0) + 1024;
+  // pipeline stages; then a block of barriers followed by either the epilogue's transposition
+  // tiles (persistent CTAs; a one-tile CTA reuses stage 0) or, 1 KiB in, the bf16 staging tile
+  // of the TMA update path; alignment slack
+  static constexpr size_t bytes(int stages, bool persistent, bool upd_tma = false) {
+    const size_t tail = upd_tma ? size_t(1024 + UPD_RING_BYTES) : size_t(256 + (persistent ? EPI_TILE_BYTES : 0));
+    return size_t(stages) * STAGE_BYTES + tail + 1024;
   }
 };
 
@@ -318,7 +331,8 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmArgs& p, int t, int til
 template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK, bool PERSIST>
 __global__ void __launch_bounds__(GEMM_THREADS, BN <= 128 ? 2 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmArgs p, const int tiles_m, const int tiles_n, const int total_work) {
+                    const __grid_constant__ UpdMaps um, const GemmArgs p, const int tiles_m, const int tiles_n,
+                    const int total_work) {
   using SM = GemmSmem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -336,10 +350,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // Fused update by TMA (one tile = its k-blocks followed by BN / 32 "chunk fills" of the same
+  // stage ring: 128 x 32 fp32 of the master and of the momentum).  The epilogue updates a chunk
+  // in place in shared memory and a TMA store writes it back, so the HBM stream of Eq. 6 is
+  // queued by the copy engine, many chunks deep, instead of by the registers of four warps.
+  constexpr bool kUpdTmaOk = (MODE == EPI_WGRAD_UPDATE) && !SPLITK && BN >= 128 && (BN * GEMM_BK * 2 >= UPD_CHUNK_BYTES);
+  const bool upd_tma = kUpdTmaOk && p.upd_tma != 0;
+  constexpr int kChunks = BN / 32;
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if (upd_tma) {
+      tma_prefetch_desc(&um.W);
+      if (p.mW != nullptr) tma_prefetch_desc(&um.M);
+      tma_prefetch_desc(&um.R);
+    }
     for (int s = 0; s < S; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
@@ -462,6 +488,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           ++issued;
           if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
         }
+        if constexpr (kUpdTmaOk) {
+          if (upd_tma && ok) {
+            const uint32_t bytes = p.mW != nullptr ? 2u * UPD_CHUNK_BYTES : uint32_t(UPD_CHUNK_BYTES);
+            for (int c = 0; c < kChunks; ++c) {
+              ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+              if (!ok) break;
+              const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
+              const uint32_t fb = full0 + 8u * s;
+              mbar_arrive_expect_tx_addr(fb, bytes);
+              tma_load_2d_addr(sa, &um.W, fb, tm.n0 + c * 32, tm.m0);
+              if (p.mW != nullptr) tma_load_2d_addr(sa + UPD_CHUNK_BYTES, &um.M, fb, tm.n0 + c * 32, tm.m0);
+              ++issued;
+              if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
+            }
+          }
+        }
       }
       if (!ok) {
         atomicExch(p.status, 1);
@@ -517,6 +559,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
         umma_commit_addr(accf0 + 8u * buf);    // accumulator complete (also releases the epilogue on error)
+        if constexpr (kUpdTmaOk) {
+          if (upd_tma) {
+            // The tile's chunk fills pass through the ring without this warp.  A CTA that goes on
+            // to another tile still has to SEE each of them complete: a parity wait only tells
+            // adjacent phases apart, and a stage may not run two phases ahead of a waiter.
+            for (int c = 0; c < kChunks; ++c) {
+              if (PERSIST) {
+                ok = mbar_wait_addr(full0 + 8u * s, ph);
+                if (!ok) break;
+              }
+              dA_lo += uint32_t(SM::STAGE_BYTES >> 4);
+              dB_lo += uint32_t(SM::STAGE_BYTES >> 4);
+              if (++s == uint32_t(S)) {
+                s = 0;
+                ph ^= 1u;
+                dA_lo = uint32_t(dA);
+                dB_lo = uint32_t(dB);
+              }
+            }
+          }
+        }
       }
       if (!ok) atomicExch(p.status, 2);
     }
@@ -536,12 +599,132 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t accf0 = smem_u32(accf_bar), acce0 = smem_u32(acce_bar);
     bool ok = true;
     uint32_t it = 0;
+    // TMA update path: position in the stage ring, and the store whose source has not been released yet
+    uint32_t us = 0, uph = 0, pending_stage = 0;
+    bool pending = false, good = true;
     for (int t = blockIdx.x; t < total_work && ok; t += (PERSIST ? int(gridDim.x) : total_work), ++it) {
       const TileCtx tc = decode_tile<BN>(p, t, tiles_m, tiles_n);
       const TileMap& tm = tc.tm;
       const uint32_t buf = PERSIST ? (it & 1u) : 0u;
       const uint32_t tacc = tmem_base + buf * uint32_t(BN);
       const int row0 = tm.m0 + q * 32;
+      if constexpr (kUpdTmaOk) {
+        if (upd_tma) {
+          // Every one of the 128 epilogue threads runs the same number of named barriers whatever
+          // happens: after a wait that ran out, the remaining chunks only keep the barrier count.
+          const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+          const uint32_t ringbuf = full0 + 1024u;
+          const int trow = q * 32 + lane;            // row of the tile this lane owns (tensor-memory lane)
+          if (good) {
+            good = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
+            good = __all_sync(0xffffffffu, good);
+            if (!good && lane == 0) atomicExch(p.status, 3);
+          }
+          tc_fence_after();
+          for (int kb = 0; kb < tc.num_kb; ++kb)       // the operand fills of this tile
+            if (++us == uint32_t(S)) { us = 0; uph ^= 1u; }
+#pragma unroll 1
+          for (int c = 0; c < kChunks; ++c) {
+            const uint32_t sW = smem0 + us * uint32_t(SM::STAGE_BYTES);
+            const uint32_t sM = sW + UPD_CHUNK_BYTES;
+            if (good) {
+              good = mbar_wait_addr(full0 + 8u * us, uph);
+              good = __all_sync(0xffffffffu, good);
+              if (!good && lane == 0) atomicExch(p.status, 4);
+            }
+            uint32_t packed[16];
+            if (good) {
+              uint32_t r[32];
+              if (tc.num_kb > 0) {
+                tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+                tmem_ld_wait();
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+              }
+              if (PERSIST && c == kChunks - 1) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acce_bar[buf]);
+              }
+              const uint32_t rowoff = uint32_t(trow) * 128u;
+              const uint32_t swz = uint32_t(trow & 7);
+              const int grow = tm.m0 + trow;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const uint32_t off = rowoff + ((uint32_t(j) ^ swz) << 4);
+                float g[4] = {__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                              __uint_as_float(r[4 * j + 3])};
+                const int n = tm.n0 + c * 32 + 4 * j;
+                if (p.out != nullptr && grow < p.M && n < tm.nlim) {
+                  float* dst = reinterpret_cast<float*>(p.out) + size_t(grow) * p.ld_out + n;
+                  if (n + 3 < tm.nlim) {
+                    __stcs(reinterpret_cast<float4*>(dst), make_float4(g[0], g[1], g[2], g[3]));
+                  } else {
+                    for (int e = 0; e < 4; ++e) if (n + e < tm.nlim) dst[e] = g[e];
+                  }
+                }
+                float m[4] = {g[0], g[1], g[2], g[3]};
+                if (p.mW != nullptr) {
+                  float4 mm;
+                  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(mm.x), "=f"(mm.y), "=f"(mm.z), "=f"(mm.w) : "r"(sM + off));
+                  m[0] = p.mu * mm.x + g[0]; m[1] = p.mu * mm.y + g[1];
+                  m[2] = p.mu * mm.z + g[2]; m[3] = p.mu * mm.w + g[3];
+                  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sM + off), "f"(m[0]), "f"(m[1]), "f"(m[2]), "f"(m[3]) : "memory");
+                }
+                float4 w;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w) : "r"(sW + off));
+                w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sW + off), "f"(w.x), "f"(w.y), "f"(w.z), "f"(w.w) : "memory");
+                packed[2 * j] = pack_bf16x2(w.x, w.y);
+                packed[2 * j + 1] = pack_bf16x2(w.z, w.w);
+              }
+            }
+            // the bf16 staging tile is free once the previous chunk's stores have read it; the
+            // same wait releases that chunk's stage to the producer
+            if (threadIdx.x == 64 && pending) {
+              tma_store_wait_read0();
+              mbar_arrive_addr(empty0 + 8u * pending_stage);
+              pending = false;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (good) {
+              const uint32_t roff = ringbuf + uint32_t(trow) * 64u;
+              const uint32_t rs = uint32_t(trow >> 1) & 3u;
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(roff + ((uint32_t(u) ^ rs) << 4)), "r"(packed[4 * u]),
+                             "r"(packed[4 * u + 1]), "r"(packed[4 * u + 2]), "r"(packed[4 * u + 3])
+                             : "memory");
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) {
+              if (good) {
+                const int n = tm.n0 + c * 32;
+                tma_store_2d_addr(&um.W, sW, n, tm.m0);
+                if (p.mW != nullptr) tma_store_2d_addr(&um.M, sM, n, tm.m0);
+                tma_store_2d_addr(&um.R, ringbuf, n, tm.m0);
+                tma_store_commit();
+                pending = true;
+                pending_stage = us;
+                if (PERSIST && c == kChunks - 1) {
+                  // A tile's last stage is released before the next tile is touched: the next
+                  // accumulator can only complete if the producer gets this stage back, so
+                  // deferring the release to the next tile's first chunk would be a cycle.
+                  tma_store_wait_read0();
+                  mbar_arrive_addr(empty0 + 8u * us);
+                  pending = false;
+                }
+              } else {
+                mbar_arrive_addr(empty0 + 8u * us);   // keep the producer's bounded waits short
+              }
+            }
+            if (++us == uint32_t(S)) { us = 0; uph ^= 1u; }
+          }
+          continue;
+        }
+      }
       WmRegs cur;
       if constexpr (upd && !split) {
         // Pull this warp's 32 rows of the master (and momentum) tile into L2 while the main loop
@@ -654,6 +837,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");     // is_last is rewritten by the next tile
+      }
+    }
+    if constexpr (kUpdTmaOk) {
+      if (pending) {                       // (thread 64 only) shared memory must outlive the last stores' reads
+        tma_store_wait_read0();
+        mbar_arrive_addr(smem_u32(empty_bar) + 8u * pending_stage);
       }
     }
   }

@@ -84,6 +84,9 @@ struct Layer {
   float *part_f = nullptr, *part_d = nullptr;   // fp32 partial tiles [tiles][splits][128][BN]
   unsigned *cnt_f = nullptr, *cnt_d = nullptr;  // per-tile arrival counters
   std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
+  bool upd_maps = false;                        // fused update streamed by TMA (fully connected layers, 128-wide tiles)
+  CUtensorMap tm_u_W, tm_u_M;                   // fp32 master / momentum as 32-column boxes
+  std::vector<CUtensorMap> tm_u_R;              // each ring slot as 32-column bf16 boxes
   std::vector<Res> rX, rZ, rDelta, rRing, rPidx;
   Res rDW;
   Ev last_update;
@@ -443,6 +446,15 @@ static int build_tensor_maps(lp_ctx* c) {
       if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
     // G: A = delta^l stored [B][out] -> MN-major (M = out contiguous); B = a^{l-1} stored [B][in] -> MN-major
+    y.upd_maps = (y.bn_g == 128 || y.bn_g == 256) && y.split_g == 1;
+    if (y.upd_maps) {
+      if ((rc = make_tmap_rows32(&y.tm_u_W, y.W, 4, y.n_in, y.n_out, y.w_ld, GEMM_BM, &err)) != LP_OK) return fail(c, rc, err);
+      if (y.mW && (rc = make_tmap_rows32(&y.tm_u_M, y.mW, 4, y.n_in, y.n_out, y.w_ld, GEMM_BM, &err)) != LP_OK) return fail(c, rc, err);
+      y.tm_u_R.resize(y.slots);
+      for (int s = 0; s < y.slots; ++s)
+        if ((rc = make_tmap_rows32(&y.tm_u_R[s], y.ring + s * y.w_elems, 2, y.n_in, y.n_out, y.w_ld, GEMM_BM, &err)) != LP_OK)
+          return fail(c, rc, err);
+    }
     gemm_box_dims(2, y.bn_g, bA, bB);
     for (int s = 0; s < kDeltaSlots; ++s)
       if ((rc = make_tmap_bf16_2d(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.n_out, y.out_rows, y.ld_out, bA[0], bA[1], &err)) != LP_OK)
@@ -623,6 +635,13 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   }
   ++c->launches;
   TimedScope ts(c, LP_TASK_G, st);
+  if (y.upd_maps && a.mode == EPI_WGRAD_UPDATE) {
+    UpdMaps um;
+    um.W = y.tm_u_W;
+    um.M = y.mW ? y.tm_u_M : y.tm_u_W;
+    um.R = y.tm_u_R[(n + 1) % y.slots];
+    return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st, &um);
+  }
   return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st);
 }
 

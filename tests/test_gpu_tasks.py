@@ -163,6 +163,21 @@ def test_tasks_split_k_forward_and_delta():
             lpb.lp_set_tuning(0, 0, 0)
 
 
+def test_tasks_persistent_tile_loop():
+    """Forced persistent CTAs on a layer with more tiles (21 x 18) than resident CTAs: every CTA
+    walks several tiles, so the pipeline, the double-buffered accumulator and the streamed
+    update tiles (Eq. 6 in the G epilogue) run across tile boundaries.  With and without momentum."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([2200, 2600, 520, 75], "gelu")
+    lpb.lp_set_tuning(0, 0, 512)
+    try:
+        run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.9, 3)
+        run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.0, 3)
+    finally:
+        lpb.lp_set_tuning(0, 0, 0)
+
+
 def test_tasks_small_convnet():
     """Conv 3x3 + ReLU (+ 2x2 max pool) layers followed by FC layers: implicit-GEMM forward, delta
     with the un-pooling epilogue (conv -> conv and conv -> FC), split-K G with the fused update,
