@@ -11,6 +11,8 @@ independent replicas, one process per GPU, and adds their throughput.
 import argparse
 import json
 import os
+
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")  # one hardware queue per scheduler stream; read when the CUDA context is created
 import statistics
 import subprocess
 import sys

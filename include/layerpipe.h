@@ -114,7 +114,12 @@ int lp_workspace_size(const lp_layer* layers, int n_layers, int n_stages, const 
  * d_l + 1 bf16 versions.  W0_host[l] (fp32, [out][in]) and b0_host[l] (fp32 [out], may be
  * NULL = zeros or has_bias = 0) are copied before the call returns.  workspace_dev:
  * device, 256-byte aligned, >= lp_workspace_size bytes; zeroed by this call.
- * Uses the current CUDA device; creates its own streams and events.
+ * Uses the current CUDA device; creates its own streams and events: three streams (forward,
+ * delta, G + update) per group of stages.  Streams overlap only while each owns a hardware
+ * work queue, and a process has CUDA_DEVICE_MAX_CONNECTIONS of those (8 if unset, at most 32),
+ * fixed when its CUDA context is created: set the variable to 32 before the first CUDA call.
+ * lp_create reads the variable and folds the stages onto (value - 2) / 3 stream triples so that
+ * no two of its streams share a queue.
  */
 int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, int n_stages,
               const int* stage, const int* delays, const lp_config* cfg,
@@ -205,6 +210,11 @@ int lp_device_status(lp_handle h, int* detail);
 enum { LP_TASK_CAST = 5 };
 int lp_get_task_time(lp_handle h, int task, long long* launches, double* total_ms);
 int lp_reset_task_times(lp_handle h);
+/* Needs LP_TIME_TASKS.  The timeline behind lp_get_task_time: for the first min(capacity, launches)
+ * timed launches of `task`, in launch order, start_ms[i] and end_ms[i] (host arrays) receive the
+ * kernel's begin and end in milliseconds after the first event timed since the last reset (of any
+ * task kind).  *count_out = entries written.  Blocks until the device is idle. */
+int lp_get_task_timeline(lp_handle h, int task, int capacity, float* start_ms, float* end_ms, int* count_out);
 
 /* Number of kernels this handle has launched so far. */
 long long lp_kernel_launches(lp_handle h);

@@ -74,6 +74,7 @@ def lib():
         "lp_device_status": [vp, ip],
         "lp_get_task_time": [vp, C.c_int, llp, _P(C.c_double)],
         "lp_reset_task_times": [vp],
+        "lp_get_task_timeline": [vp, C.c_int, C.c_int, _P(C.c_float), _P(C.c_float), _P(C.c_int)],
         "lp_set_tuning": [C.c_int, C.c_int, C.c_int],
         "lp_destroy": [vp],
         "lp_gemm_bf16": [C.c_int, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, vp],
@@ -93,7 +94,7 @@ def lib():
 
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
            "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
-           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
+           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
            "lp_gemm_bf16", "lp_softmax_xent_static"]
 
 
@@ -291,6 +292,17 @@ class Trainer:
         n, ms = C.c_longlong(), C.c_double()
         _check(lib().lp_get_task_time(self.h, k, C.byref(n), C.byref(ms)), self.h)
         return n.value, ms.value
+
+    def task_timeline(self, task, capacity=4096):
+        """(start_ms, end_ms) arrays of the timed launches of one task kind, in launch order,
+        relative to the first event timed since the last reset; needs flags=LP_TIME_TASKS."""
+        k = dict(self.TASK, cast=5)[task]
+        st = np.zeros(capacity, dtype=np.float32)
+        en = np.zeros(capacity, dtype=np.float32)
+        n = C.c_int()
+        _check(lib().lp_get_task_timeline(self.h, k, capacity, st.ctypes.data_as(_P(C.c_float)),
+                                          en.ctypes.data_as(_P(C.c_float)), C.byref(n)), self.h)
+        return st[:n.value], en[:n.value]
 
     def reset_task_times(self):
         _check(lib().lp_reset_task_times(self.h), self.h)

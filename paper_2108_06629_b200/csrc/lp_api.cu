@@ -15,6 +15,7 @@
 //   Fused-B schedule: delta_l, G_l, U_l run back to back as ONE task on the stage's
 //   backward stream and delta^{l-1} is released only when the whole task has finished.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <memory>
 
@@ -99,6 +100,7 @@ struct lp_ctx {
   lp_config cfg{};
   int n_stages = 0;
   int stages_used = 0;
+  int n_groups = 1;             // stream triples; stage s runs on triple s % n_groups
   int classes = 0, ld_cls = 0;
   // shared buffers
   float* zL = nullptr;          // [kDeltaSlots][B][ld_cls] fp32
@@ -738,10 +740,19 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   // (measured on the 8 x 4096 workload: this ordering 0.90 ms per step; G as urgent as forward,
   // all equal, or G above delta: 1.03 ms -- the paper's rule of putting delta first holds here)
   const int pD = greatest, pF = std::min(least, greatest + 1), pG = least;
-  c->sF.assign(used, nullptr);
-  c->sD.assign(used, nullptr);
-  c->sG.assign(used, nullptr);
-  for (int s = 0; s < used; ++s) {
+  // Streams only run concurrently while each has a hardware work queue of its own; the process
+  // has CUDA_DEVICE_MAX_CONNECTIONS of them (8 unless the variable was set, up to 32, before the
+  // CUDA context was created).  Streams that share a queue serialise in enqueue order, which
+  // stalls tasks behind unrelated event waits (measured on the 8 x 4096 workload: 24 streams on 8
+  // queues 838 us per step, on 32 queues 591 us).  So the stages share as many stream triples as
+  // the queues allow, two queues being left to the caller's stream and the default stream.
+  int conn = 8;
+  if (const char* e = getenv("CUDA_DEVICE_MAX_CONNECTIONS")) conn = std::max(1, std::min(32, atoi(e)));
+  c->n_groups = std::max(1, std::min(used, (conn - 2) / 3));
+  c->sF.assign(c->n_groups, nullptr);
+  c->sD.assign(c->n_groups, nullptr);
+  c->sG.assign(c->n_groups, nullptr);
+  for (int s = 0; s < c->n_groups; ++s) {
     LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sF[s], cudaStreamNonBlocking, pF));
     LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sD[s], cudaStreamNonBlocking, pD));
     LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sG[s], cudaStreamNonBlocking, pG));
@@ -813,6 +824,25 @@ extern "C" int lp_get_task_time(lp_handle h, int task, long long* launches, doub
   return LP_OK;
 }
 
+extern "C" int lp_get_task_timeline(lp_handle h, int task, int capacity, float* start_ms, float* end_ms, int* count_out) {
+  if (!h || task < 0 || task > LP_TASK_CAST || capacity < 0 || !count_out || (capacity > 0 && (!start_ms || !end_ms)))
+    return LP_ERR_INVALID_ARG;
+  if (!(h->cfg.flags & LP_TIME_TASKS)) return fail(h, LP_ERR_NOT_READY, "handle was created without LP_TIME_TASKS");
+  LP_CUDA(h, cudaDeviceSynchronize());
+  *count_out = 0;
+  if (h->tpool_next == 0) return LP_OK;
+  cudaEvent_t base = h->tpool[0];      // events are handed out in order: the first one since the reset
+  int n = 0;
+  for (auto& pr : h->timed[task]) {
+    if (n >= capacity) break;
+    LP_CUDA(h, cudaEventElapsedTime(&start_ms[n], base, pr.first));
+    LP_CUDA(h, cudaEventElapsedTime(&end_ms[n], base, pr.second));
+    ++n;
+  }
+  *count_out = n;
+  return LP_OK;
+}
+
 extern "C" int lp_reset_task_times(lp_handle h) {
   if (!h) return LP_ERR_INVALID_ARG;
   LP_CUDA(h, cudaDeviceSynchronize());
@@ -865,7 +895,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   // ---- forward ---------------------------------------------------------------
   for (int l = 0; l < nL; ++l) {
     Layer& y = c->L[l];
-    cudaStream_t st = c->sF[y.stage];
+    cudaStream_t st = c->sF[y.stage % c->n_groups];
     Res* rin = &y.rX[n % y.x_slots];
     Res* rw = &y.rRing[slot[l]];
     Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[n % c->L[l + 1].x_slots];
@@ -880,7 +910,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   // ---- loss and delta^L --------------------------------------------------------
   {
     Layer& yl = c->L[nL - 1];
-    cudaStream_t st = c->sD[yl.stage];
+    cudaStream_t st = c->sD[yl.stage % c->n_groups];
     Res* rd = &yl.rDelta[ds];
     LP_CUDA(c, task_begin(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}));
     ++c->launches;
@@ -907,7 +937,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
       if (pv.pool) ridx = &pv.rPidx[n % y.x_slots];
     }
     if (fusedB) {
-      cudaStream_t st = c->sD[y.stage];
+      cudaStream_t st = c->sD[y.stage % c->n_groups];
       LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}));
       if (l > 0) LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
       LP_CUDA(c, launch_G(c, l, n, st));
@@ -915,12 +945,12 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
       LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}, &y.last_update));
     } else {
       if (l > 0) {
-        cudaStream_t st = c->sD[y.stage];
+        cudaStream_t st = c->sD[y.stage % c->n_groups];
         LP_CUDA(c, task_begin(c, st, {rdl, rw, raux, ridx}, {rdprev}));
         LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
         LP_CUDA(c, task_end(c, st, {rdl, rw, raux, ridx}, {rdprev}, nullptr));
       }
-      cudaStream_t sg = c->sG[y.stage];
+      cudaStream_t sg = c->sG[y.stage % c->n_groups];
       if (fused_update(c)) {
         // G + update of W in one kernel, then the bias update: one task that writes the ring
         // slot of version n+1 (the slot delta_l(n) reads, so the tracker orders it after it)

@@ -1,4 +1,6 @@
 import os
+
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")  # one hardware queue per scheduler stream; read when the CUDA context is created
 import sys
 
 import pytest
