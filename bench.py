@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
 # ncu capture summarised under profiles/ (None until a capture exists for that pair).
 NCU_TRAFFIC_BYTES = {
-    # profiles/gemm_G_fused_update_mlp8_4096.md: 138.77 MB read + 110.34 MB written inside the kernel window
-    ("mlp8_4096", "G"): 249.12e6,
+    # profiles/gemm_G_fused_update_mlp8_4096.md: 139.54 MB read + 111.93 MB written inside the kernel window
+    ("mlp8_4096", "G"): 251.47e6,
 }
 
 
@@ -326,22 +326,35 @@ def run_ours(args, wl):
 
     line = None
     if rank == 0:
-        # ---- per-kernel times for the roofline (separate handle with timing events) ----------
-        trp = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
-                          schedule=sched, flags=lpb.LP_TIME_TASKS, W0=W0, b0=b0, device=dev)
-        for k in range(prewarm):
-            trp.step(xs[k % P], ys[k % P])
-        trp.flush()
-        torch.cuda.synchronize()
-        trp.reset_task_times()
-        nprof = min(args.steps, 32768 // (6 * len(layers)))
-        timed_loop(torch, trp, xs, ys, nprof, stream)
-        kinds = {}
-        for kind in ("forward", "delta", "G", "update", "loss", "cast"):
-            n, tot = trp.task_time(kind)
-            kinds[kind] = dict(launches=n, total_ms=tot, avg_us=1e3 * tot / max(n, 1))
-        trp.close()
-        del trp
+        # ---- per-kernel times for the roofline (separate handles with timing events) ----------
+        # In the real schedule up to a dozen kernels share the GPU, so a kernel's event-timed
+        # duration there is the time it spent sharing, not its own cost.  The roofline therefore
+        # uses a second pass of the same steps with every task on one stream (LP_SERIAL_TASKS: the
+        # same kernels, launches and operands, none overlapping); the overlapped averages are
+        # reported beside it.
+        def kernel_times(flags):
+            trp = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                              schedule=sched, flags=flags, W0=W0, b0=b0, device=dev)
+            for k in range(prewarm):
+                trp.step(xs[k % P], ys[k % P])
+            trp.flush()
+            torch.cuda.synchronize()
+            trp.reset_task_times()
+            nprof = min(args.steps, 32768 // (6 * len(layers)))
+            timed_loop(torch, trp, xs, ys, nprof, stream)
+            out = {}
+            for kind in ("forward", "delta", "G", "update", "loss", "cast"):
+                n, tot = trp.task_time(kind)
+                out[kind] = dict(launches=n, total_ms=tot, avg_us=1e3 * tot / max(n, 1))
+            trp.close()
+            del trp
+            torch.cuda.empty_cache()
+            return out
+
+        kinds_live = kernel_times(lpb.LP_TIME_TASKS)
+        kinds = kernel_times(lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS)
+        for kind in kinds:
+            kinds[kind]["avg_us_overlapped"] = kinds_live[kind]["avg_us"]
         peaks = load_peaks()
         wm = work_model(layers, B, wl["momentum"])
         dom = max(("forward", "delta", "G", "update"), key=lambda k: kinds[k]["total_ms"])
@@ -361,6 +374,9 @@ def run_ours(args, wl):
                           "G": "gemm_tcgen05_kernel<G>", "update": "sgd_update_kernel"}[dom]
         roof["peak_source"] = "of " + peaks["_source"]
         roof["avg_launch_us"] = kinds[dom]["avg_us"]
+        roof["avg_launch_us_overlapped"] = kinds[dom]["avg_us_overlapped"]
+        roof["timing"] = ("CUDA events around every launch of the kernel in a pass of the same steps with all tasks on "
+                          "one stream; avg_launch_us_overlapped is the same measurement under the concurrent schedule")
         roof["algorithmic_per_launch"] = {"bytes": avg_bytes, "flops": avg_flops}
         # whole-step figures against both roofs
         step_flops = sum(p["flops"] for k in ("forward", "delta", "G") for p in wm[k])

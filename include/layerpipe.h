@@ -50,9 +50,11 @@ enum { LP_SCHED_LAYERPIPE = 0, /* delta and G of a layer are separate concurrent
 enum { LP_F32 = 0, LP_BF16 = 1 };
 enum { LP_CAPTURE_GRADS = 1u, /* keep G of the latest step readable by lp_get_grads            */
        LP_TIME_TASKS = 2u,     /* bracket every kernel with timing events (see lp_get_task_time) */
-       LP_UNFUSED_UPDATE = 4u }; /* write G to memory and run Eq. 6 as a separate kernel. Default:  */
+       LP_UNFUSED_UPDATE = 4u, /* write G to memory and run Eq. 6 as a separate kernel. Default:  */
                                /* the update is fused into the epilogue of the G contraction and  */
                                /* G is only stored when LP_CAPTURE_GRADS is set                    */
+       LP_SERIAL_TASKS = 8u };  /* measurement aid: enqueue every task on the caller's stream, so  */
+                               /* that no two kernels overlap and LP_TIME_TASKS times each alone  */
 
 /* One layer of the chain (Eqs. 1-2: z = W a (+ b), a = f(z)). */
 typedef struct {

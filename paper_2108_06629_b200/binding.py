@@ -23,6 +23,7 @@ LP_F32, LP_BF16 = 0, 1
 LP_CAPTURE_GRADS = 1
 LP_TIME_TASKS = 2
 LP_UNFUSED_UPDATE = 4
+LP_SERIAL_TASKS = 8
 
 
 class lp_layer(C.Structure):

@@ -208,6 +208,15 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   a.l2_ahead = (a.g.kind == GEOM_PLAIN && work <= slots && a.kb_per_split >= 8) ? g_l2_ahead : 0;
 #define LP_LAUNCH(SPL, PER) \
   gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, SPL, PER><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, *um, a, tiles_m, tiles_n, int(work))
+  if constexpr (MODE == EPI_WGRAD_UPDATE && BN >= 128) {
+    if (a.upd_tma) {
+      if (a.persistent)
+        gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false, true, true><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, *um, a, tiles_m, tiles_n, int(work));
+      else
+        gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false, false, true><<<grid, GEMM_THREADS, smem, st>>>(tmA, tmB, *um, a, tiles_m, tiles_n, int(work));
+      return cudaGetLastError();
+    }
+  }
   if (a.splits > 1) { if (a.persistent) LP_LAUNCH(true, true); else LP_LAUNCH(true, false); }
   else              { if (a.persistent) LP_LAUNCH(false, true); else LP_LAUNCH(false, false); }
 #undef LP_LAUNCH
@@ -223,6 +232,14 @@ static cudaError_t configure_one() {
     return e;
   LP_ATTR(false, false) LP_ATTR(false, true) LP_ATTR(true, false) LP_ATTR(true, true)
 #undef LP_ATTR
+  if constexpr (MODE == EPI_WGRAD_UPDATE && BN >= 128) {
+    if ((e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false, false, true>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess)
+      return e;
+    if ((e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BN, A_MN, B_MN, MODE, false, true, true>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess)
+      return e;
+  }
   return cudaSuccess;
 }
 

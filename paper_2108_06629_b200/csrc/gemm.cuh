@@ -328,7 +328,7 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmArgs& p, int t, int til
 // tiles b, b + gridDim.x, ...  The accumulator is double-buffered in tensor memory (2 x BN
 // columns) so that the epilogue of one tile overlaps the main loop of the next, and the
 // shared-memory pipeline runs on across tile boundaries.
-template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK, bool PERSIST>
+template <int BN, bool A_MN, bool B_MN, int MODE, bool SPLITK, bool PERSIST, bool UTMA = false>
 __global__ void __launch_bounds__(GEMM_THREADS, BN <= 128 ? 2 : 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ UpdMaps um, const GemmArgs p, const int tiles_m, const int tiles_n,
@@ -354,8 +354,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // stage ring: 128 x 32 fp32 of the master and of the momentum).  The epilogue updates a chunk
   // in place in shared memory and a TMA store writes it back, so the HBM stream of Eq. 6 is
   // queued by the copy engine, many chunks deep, instead of by the registers of four warps.
-  constexpr bool kUpdTmaOk = (MODE == EPI_WGRAD_UPDATE) && !SPLITK && BN >= 128 && (BN * GEMM_BK * 2 >= UPD_CHUNK_BYTES);
-  const bool upd_tma = kUpdTmaOk && p.upd_tma != 0;
+  // (UTMA is a template parameter, not a flag: the register-path update keeps 128 registers of
+  // prefetched tiles per thread, and a kernel that contains both forms is allocated for the larger --
+  // two resident CTAs then own the whole register file and no other stream's block fits beside them.)
+  static_assert(!UTMA || ((MODE == EPI_WGRAD_UPDATE) && !SPLITK && BN >= 128 && (BN * GEMM_BK * 2 >= UPD_CHUNK_BYTES)),
+                "the TMA update needs an unsplit update tile at least 128 columns wide");
+  constexpr bool kUpdTmaOk = UTMA;
+  constexpr bool upd_tma = UTMA;
   constexpr int kChunks = BN / 32;
 
   if (threadIdx.x == 0) {
@@ -726,7 +731,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
       WmRegs cur;
-      if constexpr (upd && !split) {
+      if constexpr (upd && !split && !UTMA) {
         // Pull this warp's 32 rows of the master (and momentum) tile into L2 while the main loop
         // runs: the register prefetch below only reaches one chunk ahead, and an L2 hit costs a
         // fraction of an HBM round trip.
@@ -778,7 +783,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
             __stcg(reinterpret_cast<float4*>(part + size_t(q * 32 + rr) * BN + c * 32 + sub_col), acc);
           }
-        } else if constexpr (upd) {
+        } else if constexpr (upd && !UTMA) {
           WmRegs nxt;
           if (c + 1 < BN / 32) load_wm(p, row0, n + 32, tm.nlim, sub_row, nxt);
           apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);

@@ -863,6 +863,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   const int nL = int(c->L.size());
   const int B = c->cfg.batch;
   const bool fusedB = (c->cfg.schedule == LP_SCHED_FUSED_B);
+  const bool serial = (c->cfg.flags & LP_SERIAL_TASKS) != 0;   // every task on the caller's stream
   const int ds = int(n % kDeltaSlots);
 
   // version bookkeeping (the integers the parity tests compare bit-exactly)
@@ -895,7 +896,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   // ---- forward ---------------------------------------------------------------
   for (int l = 0; l < nL; ++l) {
     Layer& y = c->L[l];
-    cudaStream_t st = c->sF[y.stage % c->n_groups];
+    cudaStream_t st = (serial ? user : c->sF[y.stage % c->n_groups]);
     Res* rin = &y.rX[n % y.x_slots];
     Res* rw = &y.rRing[slot[l]];
     Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[n % c->L[l + 1].x_slots];
@@ -910,7 +911,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   // ---- loss and delta^L --------------------------------------------------------
   {
     Layer& yl = c->L[nL - 1];
-    cudaStream_t st = c->sD[yl.stage % c->n_groups];
+    cudaStream_t st = (serial ? user : c->sD[yl.stage % c->n_groups]);
     Res* rd = &yl.rDelta[ds];
     LP_CUDA(c, task_begin(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}));
     ++c->launches;
@@ -937,7 +938,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
       if (pv.pool) ridx = &pv.rPidx[n % y.x_slots];
     }
     if (fusedB) {
-      cudaStream_t st = c->sD[y.stage % c->n_groups];
+      cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
       LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}));
       if (l > 0) LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
       LP_CUDA(c, launch_G(c, l, n, st));
@@ -945,12 +946,12 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
       LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}, &y.last_update));
     } else {
       if (l > 0) {
-        cudaStream_t st = c->sD[y.stage % c->n_groups];
+        cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
         LP_CUDA(c, task_begin(c, st, {rdl, rw, raux, ridx}, {rdprev}));
         LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
         LP_CUDA(c, task_end(c, st, {rdl, rw, raux, ridx}, {rdprev}, nullptr));
       }
-      cudaStream_t sg = c->sG[y.stage % c->n_groups];
+      cudaStream_t sg = (serial ? user : c->sG[y.stage % c->n_groups]);
       if (fused_update(c)) {
         // G + update of W in one kernel, then the bias update: one task that writes the ring
         // slot of version n+1 (the slot delta_l(n) reads, so the tracker orders it after it)
