@@ -53,6 +53,7 @@ struct PlanResult {
   int rounds = 0;
 };
 int plan_layers(const lp_layer* layers, int L, int batch, int Np, PlanResult* out);
+int layer_macs(const lp_layer& y, int batch, long long* macs);   // the planner's cost of one contraction of the layer
 
 // ---- elementwise.cu ---------------------------------------------------------
 cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,

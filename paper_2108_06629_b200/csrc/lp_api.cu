@@ -9,9 +9,9 @@
 // weight version max(0, n - d_l), tasks of consecutive minibatches overlap on the device
 // exactly as far as the delays allow -- the pipelining of Section III-A -- while the
 // results stay those of the minibatch-by-minibatch recursion.
-//   LayerPipe schedule: per stage three streams -- delta (highest priority: it carries
-//   the critical loop), forward, and G+update (lowest) -- so delta_l and G_l of one layer
-//   run concurrently and delta^{l-1} is released as soon as delta_l is done.
+//   LayerPipe schedule: per stage group three streams -- G+update (highest priority: it
+//   hands buffers back to later minibatches), delta, forward -- so delta_l and G_l of one
+//   layer run concurrently and delta^{l-1} is released as soon as delta_l is done.
 //   Fused-B schedule: delta_l, G_l, U_l run back to back as ONE task on the stage's
 //   backward stream and delta^{l-1} is released only when the whole task has finished.
 #include <cstdio>
@@ -24,7 +24,7 @@
 
 namespace lp {
 
-constexpr int kDeltaSlots = 2;
+constexpr int kDeltaSlots = 4;
 constexpr int kLossRing = 256;
 constexpr int kLogRing = 4096;
 constexpr int kEventPool = 2048;
@@ -734,12 +734,26 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   lp_ctx* h = c.get();
   LP_CUDA(nullptr, cudaMemset(c->ws, 0, need));
   LP_CUDA(nullptr, gemm_configure());
-  // streams: delta highest priority, forward next, G + update lowest
   int least = 0, greatest = 0;
   LP_CUDA(nullptr, cudaDeviceGetStreamPriorityRange(&least, &greatest));
-  // (measured on the 8 x 4096 workload: this ordering 0.90 ms per step; G as urgent as forward,
-  // all equal, or G above delta: 1.03 ms -- the paper's rule of putting delta first holds here)
-  const int pD = greatest, pF = std::min(least, greatest + 1), pG = least;
+  // Priorities: G + update highest, delta next, forward lowest.  The paper puts delta first because
+  // it carries the critical loop between processors; on one GPU the step time is set by how full
+  // the SMs are kept, and the G + update task is the one that hands buffers back (the delta slot,
+  // the ring slot of the next version), so starving it stalls later minibatches.  Measured per step
+  // with every stream on its own hardware queue and four delta slots, (delta > forward > G) against
+  // this order: 8 x 4096 MLP 589 / 588 us, small VGG 478 / 384 us, VGG-16 9.43 / 9.20 ms, 16 x 8192
+  // MLP 11.11 / 10.89 ms; all priorities equal lies in between.
+  // A network whose kernels are too small to fill the GPU (the 784-256-256-256-10 MLP at batch
+  // 32: 0.110 ms per step with delta first, 0.130 ms with G first) is bound by the latency of the
+  // delta chain instead, and keeps the paper's order.
+  long long step_macs = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    long long m = 0;
+    if (layer_macs(layers[l], cfg->batch, &m) == LP_OK) step_macs += 3 * m;
+  }
+  const bool g_first = step_macs >= 1000000000ll;
+  const int pMid = std::min(least, greatest + 1);
+  const int pG = g_first ? greatest : least, pD = g_first ? pMid : greatest, pF = g_first ? least : pMid;
   // Streams only run concurrently while each has a hardware work queue of its own; the process
   // has CUDA_DEVICE_MAX_CONNECTIONS of them (8 unless the variable was set, up to 32, before the
   // CUDA context was created).  Streams that share a queue serialise in enqueue order, which
