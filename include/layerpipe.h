@@ -171,7 +171,9 @@ int lp_get_grads(lp_handle h, int layer, long long step, float* dW_out, float* d
  *   LP_BUF_MASTER_W/B, LP_BUF_MOM_W/B, LP_BUF_GRAD_W/B   [out][in] / [out]   (index ignored)
  *   LP_BUF_POOL_IDX   [pooled pixels][channels]  position 0..3 of the maximum in its 2x2 window   minibatch
  * For convolution layers "batch" rows become batch*H*W pixel rows (NHWC) and [out][in] becomes
- * [Cout][R][S][Cin].
+ * [Cout][R][S][Cin].  A first convolution layer with 9*Cin <= 64 stores its input as the matrix of
+ * 3x3 patches; LP_BUF_INPUT of that layer is still exchanged as the image [batch][H][W][Cin]
+ * (a write builds every pixel's patch row, a read returns the centre taps).
  */
 enum { LP_BUF_INPUT = 0, LP_BUF_Z = 1, LP_BUF_DELTA = 2, LP_BUF_LOGITS = 3, LP_BUF_LABELS = 4, LP_BUF_LOSS = 5,
        LP_BUF_RING_W = 6, LP_BUF_RING_B = 7, LP_BUF_MASTER_W = 8, LP_BUF_MASTER_B = 9, LP_BUF_MOM_W = 10,

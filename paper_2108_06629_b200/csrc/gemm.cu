@@ -3,6 +3,7 @@
 #include "gemm2.cuh"
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.h"

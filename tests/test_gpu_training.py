@@ -183,6 +183,76 @@ def test_fused_and_unfused_update_agree():
     assert a["loss"] == b["loss"]
 
 
+def test_serial_tasks_agree_and_timeline_is_consistent():
+    """LP_SERIAL_TASKS runs the same kernels on one stream: bit-identical tensors.  With
+    LP_TIME_TASKS the timeline lists every launch of a task kind in order, and on one stream no
+    two kernels overlap."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 40], "gelu")
+    steps = 6
+    a, W0, b0 = free_run(layers, 56, 3, [2, 1, 0], 0.02, 0.9, steps, lpb.LP_SCHED_LAYERPIPE)
+    b, _, _ = free_run(layers, 56, 3, [2, 1, 0], 0.02, 0.9, steps, lpb.LP_SCHED_LAYERPIPE,
+                       extra_flags=lpb.LP_SERIAL_TASKS)
+    for l in range(len(layers)):
+        assert np.array_equal(a["W"][l][0], b["W"][l][0]) and np.array_equal(a["W"][l][1], b["W"][l][1])
+    assert a["loss"] == b["loss"]
+
+    tr = lpb.Trainer(layers, 56, 3, delays=[2, 1, 0], lr=0.02, momentum=0.9,
+                     flags=lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS, W0=W0, b0=b0)
+    for n in range(steps):
+        x, y = I.minibatch(layers, 56, n)
+        tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    tr.flush()
+    torch.cuda.synchronize()
+    L = len(layers)
+    expect = dict(cast=steps, forward=steps * L, loss=steps, delta=steps * (L - 1), G=steps * L, update=steps * L)
+    spans = []
+    for kind, count in expect.items():
+        st, en = tr.task_timeline(kind)
+        n, tot = tr.task_time(kind)
+        assert len(st) == count == n
+        assert np.all(en >= st) and np.all(np.diff(st) > 0)
+        assert abs(float(np.sum(en - st)) - tot) <= 1e-3 * max(tot, 1e-3) + 1e-3
+        spans += list(zip(st.tolist(), en.tolist()))
+    spans.sort()
+    assert spans[0][0] == 0.0                      # times are relative to the first timed event
+    for (s0, e0), (s1, e1) in zip(spans, spans[1:]):
+        assert s1 >= e0 - 2e-3                     # one stream: the next kernel starts after the previous one ended (2 us of event resolution)
+    tr.close()
+
+
+def test_patch_matrix_of_the_first_convolution_layer():
+    """A first convolution layer with three input channels keeps its input as the matrix of 3x3
+    patches.  After one step the first layer's output (the second layer's stashed input) must be
+    the oracle's a^1 for the same weights and image -- this goes through the patch cast kernel,
+    which the task-by-task tests bypass -- and the stash read back as an image is RN_bf16(x)."""
+    import torch
+    from oracle import layerpipe_oracle as O
+    from oracle.bf16 import rn_bf16
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    from gpu_common import assert_bf16_close
+    layers = I.vgg(16, [16, 32, "P"], [10])
+    B = 8
+    W0, b0 = I.initial_weights(layers, 0)
+    b0 = [np.linspace(-0.2, 0.2, l["n_out"]).astype(np.float32) for l in layers]
+    tr = lpb.Trainer(layers, B, 2, lr=0.01, momentum=0.0, W0=W0, b0=b0)
+    x, y = I.minibatch(layers, B, 0)
+    tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    tr.flush()
+    torch.cuda.synchronize()
+    got_x = tr.debug_read("input", 0, 0)
+    assert np.array_equal(got_x, rn_bf16(x))
+    orc = O.DelayedGradientTrainer(layers, [0, 0, 0], 0.01, 0.0, W0, b0, mirror=True, dtype=np.float32)
+    rec = orc.step(x, y, capture=True)
+    a1 = np.asarray(rec["a"][1], dtype=np.float32)
+    got_a1 = tr.debug_read("input", 1, 0)
+    assert_bf16_close(got_a1, a1, "a^1 through the patch matrix")
+    tr.close()
+
+
 def test_step_rejects_bad_arguments_without_side_effects():
     import torch
     from paper_2108_06629_b200 import binding as lpb
