@@ -39,6 +39,12 @@ void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]);
 // given, and the launch qualifies, the update's tiles are streamed by TMA.
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, cudaStream_t stream, const UpdMaps* um = nullptr);
+// 3x3 convolution forward (which = 0) / delta (which = 1) with at most 64 channels on both sides:
+// tmA = NHWC tensor map with a 64 x 16 x 18 x 1 box, tmB = the layer's weight map (64 x 64 boxes);
+// args.g describes 8 x 16 pixel tiles (lw = 3, lh = 4).  tmO (forward only; any valid map otherwise): the
+// NHWC output with a 64 x 8 x 16 x 1 box, written by TMA stores.
+cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
+                             const GemmArgs& args, cudaStream_t stream);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process
 void gemm_set_tuning(int bn, int stages, int splits);   // 0 = automatic
 int gemm_pick_splits(int M, int N, int K, int bn);

@@ -1,0 +1,266 @@
+// 3x3 convolution contractions over few channels (at most 64 on both sides): forward
+// (Eqs. 1-2) and delta (Eqs. 3-4) as an implicit GEMM whose activation operand is fetched ONCE
+// per tile.
+//
+// The general kernel loads a 128-pixel x 64-channel box per filter tap, i.e. nine shifted copies
+// of nearly the same pixels; with only 64 output columns per tile the tensor cores then wait on
+// the ~64 B/clk one SM can pull from L2.  Here a tile is 8 x 16 pixels of one image; its
+// 10 x 18 halo box (the pixels the nine taps touch) lands in shared memory once (22.5 KiB), and
+// the operand of tap (r, s) is a VIEW of it: the matrix descriptor starts r * 10 + s pixel rows
+// into the box, eight consecutive pixels of an image row form one 8-row swizzle group and the
+// next group is one box row (10 pixels = 1280 bytes) further.  The
+// 128-byte swizzle is a function of the absolute shared-memory address for TMA and for the
+// tensor core alike, so a view that starts at any 128-byte row of the box needs nothing else
+// (checked tap by tap with one-hot weights: exact with the descriptor's base-offset field left
+// zero, chunk-permuted when it is set to the start row).  All nine 64 x 64 weight taps stay resident in shared memory (72 KiB) for the whole
+// persistent CTA.  Per tile the SM now reads 22.5 KiB instead of 216 KiB; four boxes are in flight.
+#pragma once
+#include "gemm.cuh"
+
+namespace lp {
+
+constexpr int HALO_W = 10, HALO_H = 18;                       // box: pixels per row (pitch) x rows
+constexpr int HALO_STAGES = 4;
+constexpr int HALO_BYTES = HALO_W * HALO_H * 128;             // 64 bf16 channels per pixel
+constexpr int HALO_TAP_BYTES = 64 * 64 * 2;                   // one weight tap: 64 x 64 bf16
+constexpr int HALO_OUT_BYTES = GEMM_BM * 128;                 // forward: one output tile, 128 pixels x 64 bf16 channels
+constexpr int HALO_SMEM_BYTES = 9 * HALO_TAP_BYTES + HALO_STAGES * HALO_BYTES + 2 * HALO_OUT_BYTES + EPI_TILE_BYTES + 256 + 1024;
+static_assert((HALO_STAGES * HALO_BYTES) % 1024 == 0, "the buffers behind the halo boxes stay 1 KiB aligned");
+
+template <bool B_MN, int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmO, const GemmArgs p, const int tiles_total) {
+  constexpr int BN = 64;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sB = smem;                                   // [9][64 x 64] weight taps
+  uint8_t* sA = smem + 9 * HALO_TAP_BYTES;              // [HALO_STAGES] halo boxes
+  uint8_t* sO = sA + HALO_STAGES * HALO_BYTES;                    // [2] output tiles of the forward epilogue (TMA store sources)
+  float* epi_tile = reinterpret_cast<float*>(sO + 2 * HALO_OUT_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(epi_tile) + EPI_TILE_BYTES);
+  uint64_t* wfull = bars;          // weights resident
+  uint64_t* afull = bars + 1;                       // [HALO_STAGES] halo box landed
+  uint64_t* aempty = afull + HALO_STAGES;           // [HALO_STAGES] halo box consumed
+  uint64_t* accf = aempty + HALO_STAGES;            // [2] accumulator complete
+  uint64_t* acce = accf + 2;                        // [2] accumulator drained
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    if (MODE == EPI_FPROP) tma_prefetch_desc(&tmO);
+    mbar_init(wfull, 1);
+    for (int b = 0; b < HALO_STAGES; ++b) {
+      mbar_init(&afull[b], 1);
+      mbar_init(&aempty[b], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&accf[b], 1);
+      mbar_init(&acce[b], 4);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 2 * BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // CTA b works through the contiguous tile range [t_begin, t_end): neighbouring tiles share halo
+  // pixels in L2, and the tile coordinates advance without divisions.
+  const int tiles_per_image = p.g.tiles_w * p.g.tiles_h;
+  const int per_cta = (tiles_total + int(gridDim.x) - 1) / int(gridDim.x);
+  const int t_begin = min(int(blockIdx.x) * per_cta, tiles_total);
+  const int t_end = min(t_begin + per_cta, tiles_total);
+  const int tw_begin = t_begin % p.g.tiles_w, th_begin = (t_begin / p.g.tiles_w) % p.g.tiles_h, tn_begin = t_begin / tiles_per_image;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int issued = 0;
+      mbar_arrive_expect_tx(wfull, 9 * HALO_TAP_BYTES);
+      for (int tap = 0; tap < 9; ++tap) tma_load_2d(sB + tap * HALO_TAP_BYTES, &tmB, wfull, tap * p.g.tap_pitch, 0);
+      uint32_t st = 0, sph = 0;
+      int tw = tw_begin, th = th_begin, n = tn_begin;
+      for (int t = t_begin; t < t_end; ++t) {
+        ok = mbar_wait(&aempty[st], sph ^ 1u);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&afull[st], HALO_BYTES);
+        // the box starts one pixel left of and above the tile; pixels outside the image read zero (= the padding)
+        tma_load_4d(sA + st * HALO_BYTES, &tmA, &afull[st], 0, tw * 8 - 1, th * 16 - 1, n);
+        ++issued;
+        if (++st == uint32_t(HALO_STAGES)) { st = 0; sph ^= 1u; }
+        if (++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++n; } }
+      }
+      if (!ok) {
+        atomicExch(p.status, 1);
+        mbar_wait(wfull, 0);
+        for (int i = (issued > HALO_STAGES ? issued - HALO_STAGES : 0); i < issued; ++i)
+          mbar_wait(&afull[i % HALO_STAGES], uint32_t(i / HALO_STAGES) & 1u);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(GEMM_BM, BN, false, B_MN);
+      constexpr uint32_t stepB = (B_MN ? 2048 : 32) >> 4;
+      // One thread issues 36 MMAs per tile, so everything that can be is computed once: the
+      // descriptors of box 0 / tap 0, and per tap the start-address offset of its view (the
+      // address field counts 16-byte units and never carries out of the low word).
+      const uint64_t dA = make_smem_desc(smem_u32(sA), 16, HALO_W * 128);
+      const uint64_t dB = B_MN ? make_smem_desc(smem_u32(sB), 8192, 1024) : make_smem_desc(smem_u32(sB), 16, 1024);
+      const uint32_t dA_lo0 = uint32_t(dA), dA_hi = uint32_t(dA >> 32), dB_lo0 = uint32_t(dB), dB_hi = uint32_t(dB >> 32);
+      uint32_t tap_off[9];
+#pragma unroll
+      for (int tap = 0; tap < 9; ++tap) {
+        int r = tap / 3, s = tap % 3;
+        if (p.g.flip) { r = 2 - r; s = 2 - s; }        // delta: the tap's shift is mirrored
+        tap_off[tap] = uint32_t(r * HALO_W + s) * (128u >> 4);
+      }
+      bool ok = mbar_wait(wfull, 0);
+      uint32_t it = 0, st = 0, sph = 0;
+      for (int t = t_begin; t < t_end && ok; ++t, ++it) {
+        const uint32_t buf = it & 1u;
+        ok = mbar_wait(&acce[buf], ((it >> 1) & 1u) ^ 1u);
+        if (!ok) break;
+        ok = mbar_wait(&afull[st], sph);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + buf * uint32_t(BN);
+        const uint32_t a_lo = dA_lo0 + st * uint32_t(HALO_BYTES >> 4);
+        uint32_t acc = 0;
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) {
+#pragma unroll
+          for (int j = 0; j < GEMM_BK / 16; ++j) {
+            umma_f16_lohi(tacc, a_lo + tap_off[tap] + uint32_t(j * 2), dA_hi,
+                          dB_lo0 + uint32_t(tap) * uint32_t(HALO_TAP_BYTES >> 4) + uint32_t(j) * stepB, dB_hi, idesc, acc);
+            acc = 1;
+          }
+        }
+        umma_commit(&aempty[st]);
+        umma_commit(&accf[buf]);
+        if (++st == uint32_t(HALO_STAGES)) { st = 0; sph ^= 1u; }
+      }
+      if (!ok) atomicExch(p.status, 2);
+    }
+  } else {
+    const int q = warp & 3;
+    float* tile = epi_tile + q * (32 * EPI_PITCH);
+    const int sub_row = lane >> 3;
+    const int sub_col = (lane & 7) * 4;
+    uint32_t it = 0;
+    bool dead = false;      // a wait ran out: keep the named-barrier count, touch nothing else
+    int tw = tw_begin - 1, th = th_begin, tn = tn_begin;
+    for (int t = t_begin; t < t_end; ++t, ++it) {
+      const uint32_t buf = it & 1u;
+      if (++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++tn; } }
+      TileMap tm;
+      tm.m0 = 0;
+      tm.n0 = 0;
+      tm.nlim = p.N;
+      tm.pw0 = tw * 8;
+      tm.ph0 = th * 16;
+      tm.pn0 = tn;
+      if (!dead) {
+        bool ok = mbar_wait(&accf[buf], (it >> 1) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {
+          if (lane == 0) atomicExch(p.status, 3);
+          dead = true;
+        }
+      }
+      if (dead && MODE != EPI_FPROP) break;      // only the forward epilogue has CTA-wide barriers
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + buf * uint32_t(BN);
+      if constexpr (MODE == EPI_FPROP) {
+        // Forward: a lane keeps its accumulator row (one pixel), adds the bias, applies f, and
+        // writes the 64 bf16 channels as one 128-byte swizzled row of a shared-memory tile that a
+        // TMA store sends to the NHWC output (8 x 16 pixel box) -- no transposition, no address
+        // arithmetic per element, and the global writes are whole lines.
+        const int trow = q * 32 + lane;
+        const uint32_t so = smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES) + uint32_t(trow) * 128u;
+        const uint32_t swz = uint32_t(trow & 7);
+        uint32_t packed[32];
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) {
+          if (dead) break;
+          uint32_t r[32];
+          tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+          tmem_ld_wait();
+          if (c == BN / 32 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acce[buf]);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const int n = c * 32 + j;
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.bias != nullptr && n < p.N) b = __ldg(reinterpret_cast<const float4*>(p.bias + n));   // bias rows are padded to 8 with zeros
+            float v[4] = {__uint_as_float(r[j]) + b.x, __uint_as_float(r[j + 1]) + b.y, __uint_as_float(r[j + 2]) + b.z,
+                          __uint_as_float(r[j + 3]) + b.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (n + e >= p.N) v[e] = 0.f;
+              else if (p.act == ACT_RELU) v[e] = fmaxf(v[e], 0.f);
+            }
+            packed[(n >> 1)] = pack_bf16x2(v[0], v[1]);
+            packed[(n >> 1) + 1] = pack_bf16x2(v[2], v[3]);
+          }
+        }
+        // the staging tile of two tiles ago must have been read by its store
+        if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (!dead) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(so + ((uint32_t(u) ^ swz) << 4)), "r"(packed[4 * u]),
+                         "r"(packed[4 * u + 1]), "r"(packed[4 * u + 2]), "r"(packed[4 * u + 3])
+                         : "memory");
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64 && !dead) {
+          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                           reinterpret_cast<uint64_t>(&tmO)),
+                       "r"(smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES)), "r"(0), "r"(tm.pw0), "r"(tm.ph0), "r"(tm.pn0)
+                       : "memory");
+          tma_store_commit();
+        }
+        continue;
+      }
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        __syncwarp();
+        tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+        tmem_ld_wait();
+        if (c == BN / 32 - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acce[buf]);
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+        __syncwarp();
+        const int n = c * 32 + sub_col;
+        epilogue_rows8<MODE>(p, tm, tile, q, sub_row, sub_col, n);
+      }
+    }
+  }
+  if (MODE == EPI_FPROP && threadIdx.x == 64) tma_store_wait_read0();   // shared memory must outlive the stores' reads
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+}  // namespace lp

@@ -1,6 +1,7 @@
 // Host side of the tcgen05 GEMM: tensor-map encoding, tile selection, launch, and the
 // stand-alone lp_gemm_bf16 entry point.
 #include "gemm2.cuh"
+#include "conv_halo.cuh"
 
 #include <algorithm>
 #include <cstdlib>
@@ -291,8 +292,35 @@ static cudaError_t configure_pair() {
   X(true, true, EPI_STORE_F32)        \
   X(true, true, EPI_WGRAD_UPDATE)
 
+// ---- halo-tile convolution (3x3, at most 64 channels on both sides) ------------------------------
+#define LP_FOR_EACH_HALO_VARIANT(X) \
+  X(false, EPI_FPROP)               \
+  X(true, EPI_DGRAD)                \
+  X(true, EPI_DGRAD_UNPOOL)
+
+cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
+                             const GemmArgs& args, cudaStream_t st) {
+  const bool b_mn = (which != 0);
+  const int tiles = args.g.tiles_w * args.g.tiles_h * (args.M / (args.g.H * args.g.W));
+  const int grid = std::min(tiles, sm_count());
+#define LP_TRYH(B, M)                                                                                          \
+  if (b_mn == B && args.mode == M) {                                                                           \
+    conv_halo_kernel<B, M><<<grid, GEMM_THREADS, HALO_SMEM_BYTES, st>>>(tmA, tmB, tmO, args, tiles);                \
+    return cudaGetLastError();                                                                                 \
+  }
+  LP_FOR_EACH_HALO_VARIANT(LP_TRYH)
+#undef LP_TRYH
+  return cudaErrorInvalidValue;
+}
+
 cudaError_t gemm_configure() {
   cudaError_t e;
+#define LP_CFGH(B, M)                                                                                          \
+  if ((e = cudaFuncSetAttribute(conv_halo_kernel<B, M>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
+                                HALO_SMEM_BYTES)) != cudaSuccess)                                              \
+    return e;
+  LP_FOR_EACH_HALO_VARIANT(LP_CFGH)
+#undef LP_CFGH
 #define LP_CFGP(A, B, M) \
   if ((e = configure_pair<A, B, M>()) != cudaSuccess) return e;
   LP_FOR_EACH_PAIR_VARIANT(LP_CFGP)

@@ -133,6 +133,51 @@ __device__ __forceinline__ int tile_row(const GemmArgs& p, const TileMap& t, int
   return row < p.M ? row : -1;
 }
 
+// Bias of four consecutive output columns (zero where there is none).
+__device__ __forceinline__ void load_bias4(const GemmArgs& p, int n, int N, float b[4]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) b[j] = (p.bias != nullptr && n + j < N) ? __ldg(p.bias + n + j) : 0.f;
+}
+// Forward epilogue for columns n..n+3 of one row: z = acc + b; z^L / stored z; a = f(z).
+__device__ __forceinline__ void fprop_store4(const GemmArgs& p, int row, int n, int N, const float acc[4], const float b[4]) {
+  const int n_pad4 = (N + 3) & ~3;
+  float v[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) v[j] = acc[j] + b[j];
+  if (p.out2 != nullptr) {
+    if (p.out2_is_f32) {
+      if (n < n_pad4)
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out2) + size_t(row) * p.ld_out2 + n) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out2) + size_t(row) * p.ld_out2 + n) =
+          make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+    }
+  }
+  if (p.out != nullptr) {
+    if (p.act == ACT_RELU) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
+    } else if (p.act == ACT_GELU) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = gelu_fwd(v[j]);
+    }
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
+        make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+  }
+}
+// Delta epilogue: delta^{l-1} = (delta^l W) (.) f'(z^{l-1}), one rounding; av = the four stored
+// values of z^{l-1} (GELU) or a^{l-1} (ReLU: a > 0 <=> z > 0) at this position.
+__device__ __forceinline__ void dgrad_store4(const GemmArgs& p, int row, int n, const float acc[4], uint2 av) {
+  float v[4] = {acc[0], acc[1], acc[2], acc[3]};
+  if (p.act != ACT_NONE) {
+    const float z[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = (p.act == ACT_RELU) ? (z[j] > 0.f ? v[j] : 0.f) : v[j] * gelu_grad(z[j]);
+  }
+  *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
+      make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+}
+
 // Epilogue for 4 consecutive columns n..n+3 of output row `row`.  Lanes past the column limit
 // inside the last 16-byte (fp32) / 8-element (bf16) group are written as zeros; groups that
 // start beyond that are skipped.
@@ -145,41 +190,14 @@ __device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int 
     *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + size_t(row) * p.ld_out + n) = make_float4(v[0], v[1], v[2], v[3]);
   } else if (MODE == EPI_FPROP) {
     if (n >= n_pad8) return;
-    if (p.bias != nullptr) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) if (n + j < N) v[j] += __ldg(p.bias + n + j);
-    }
-    if (p.out2 != nullptr) {
-      if (p.out2_is_f32) {
-        if (n < n_pad4)
-          *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out2) + size_t(row) * p.ld_out2 + n) = make_float4(v[0], v[1], v[2], v[3]);
-      } else {
-        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out2) + size_t(row) * p.ld_out2 + n) =
-            make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
-      }
-    }
-    if (p.out != nullptr) {
-      if (p.act == ACT_RELU) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
-      } else if (p.act == ACT_GELU) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = gelu_fwd(v[j]);
-      }
-      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
-          make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
-    }
+    float b[4];
+    load_bias4(p, n, N, b);
+    fprop_store4(p, row, n, N, v, b);
   } else if (MODE == EPI_DGRAD) {
-    // delta^{l-1} = (delta^l W) (.) f'(z^{l-1}), one rounding
     if (n >= n_pad8) return;
-    if (p.act != ACT_NONE) {
-      const uint2 av = *reinterpret_cast<const uint2*>(p.aux + size_t(row) * p.ld_aux + n);
-      const float z[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) v[j] = (p.act == ACT_RELU) ? (z[j] > 0.f ? v[j] : 0.f) : v[j] * gelu_grad(z[j]);
-    }
-    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + size_t(row) * p.ld_out + n) =
-        make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+    uint2 av = make_uint2(0u, 0u);
+    if (p.act != ACT_NONE) av = *reinterpret_cast<const uint2*>(p.aux + size_t(row) * p.ld_aux + n);
+    dgrad_store4(p, row, n, v, av);
   } else if (MODE == EPI_DGRAD_UNPOOL) {
     // the layer below ended in ReLU + 2x2 max pool: route the gradient to the recorded maximum
     if (n >= N) return;
@@ -216,6 +234,53 @@ __device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int 
     w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
     __stcs(reinterpret_cast<float4*>(p.W + off), w);
     *reinterpret_cast<uint2*>(p.ring + off) = make_uint2(pack_bf16x2(w.x, w.y), pack_bf16x2(w.z, w.w));
+  }
+}
+
+// One lane's share of a transposed 32 x 32 chunk: columns n..n+3 of the eight tile rows
+// q*32 + i*4 + sub_row.  The four epilogue warps of a CTA are all the latency hiding there is,
+// so what does not depend on the row is fetched once (the bias) and what does is fetched for
+// all eight rows before the first store (f' operands): a store may alias a later load as far as
+// the compiler knows, and would otherwise serialise eight global round trips.
+template <int MODE>
+__device__ __forceinline__ void epilogue_rows8(const GemmArgs& p, const TileMap& tm, const float* tile, int q,
+                                               int sub_row, int sub_col, int n) {
+  int rows[8];
+#pragma unroll
+  for (int i8 = 0; i8 < 8; ++i8) rows[i8] = tile_row(p, tm, q * 32 + i8 * 4 + sub_row);
+  const int N = tm.nlim;
+  const int n_pad8 = (N + 7) & ~7;
+  if constexpr (MODE == EPI_FPROP) {
+    if (n >= n_pad8) return;
+    float b[4];
+    load_bias4(p, n, N, b);
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8) {
+      if (rows[i8] < 0) continue;
+      const float4 a = *reinterpret_cast<const float4*>(tile + (i8 * 4 + sub_row) * EPI_PITCH + sub_col);
+      const float v[4] = {n + 0 < N ? a.x : 0.f, n + 1 < N ? a.y : 0.f, n + 2 < N ? a.z : 0.f, n + 3 < N ? a.w : 0.f};
+      fprop_store4(p, rows[i8], n, N, v, b);
+    }
+  } else if constexpr (MODE == EPI_DGRAD) {
+    if (n >= n_pad8) return;
+    uint2 av[8];
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8)
+      av[i8] = (p.act != ACT_NONE && rows[i8] >= 0) ? *reinterpret_cast<const uint2*>(p.aux + size_t(rows[i8]) * p.ld_aux + n)
+                                                    : make_uint2(0u, 0u);
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8) {
+      if (rows[i8] < 0) continue;
+      const float4 a = *reinterpret_cast<const float4*>(tile + (i8 * 4 + sub_row) * EPI_PITCH + sub_col);
+      const float v[4] = {n + 0 < N ? a.x : 0.f, n + 1 < N ? a.y : 0.f, n + 2 < N ? a.z : 0.f, n + 3 < N ? a.w : 0.f};
+      dgrad_store4(p, rows[i8], n, v, av[i8]);
+    }
+  } else {
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8) {
+      const float4 a = *reinterpret_cast<const float4*>(tile + (i8 * 4 + sub_row) * EPI_PITCH + sub_col);
+      if (rows[i8] >= 0) epilogue_store4<MODE>(p, rows[i8], n, N, a);
+    }
   }
 }
 
@@ -789,13 +854,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);
           cur = nxt;
         } else {
-#pragma unroll
-          for (int i8 = 0; i8 < 8; ++i8) {
-            const int rr = i8 * 4 + sub_row;
-            const int row = tile_row(p, tm, q * 32 + rr);
-            const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
-            if (row >= 0) epilogue_store4<MODE>(p, row, n, tm.nlim, acc);
-          }
+          epilogue_rows8<MODE>(p, tm, tile, q, sub_row, sub_col, n);
         }
       }
       if constexpr (split) {

@@ -21,6 +21,7 @@
 
 #include "common.h"
 #include "gemm.cuh"
+#include "conv_halo.cuh"
 
 namespace lp {
 
@@ -85,6 +86,11 @@ struct Layer {
   float *part_f = nullptr, *part_d = nullptr;   // fp32 partial tiles [tiles][splits][128][BN]
   unsigned *cnt_f = nullptr, *cnt_d = nullptr;  // per-tile arrival counters
   std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
+  // 3x3 layers with at most 64 channels on both sides and images tiled by 8 x 16 pixels: the
+  // activation / delta box is fetched once per tile with its halo (see conv_halo.cuh)
+  bool halo_f = false, halo_d = false;
+  std::vector<CUtensorMap> tm_hf_A, tm_hd_A;    // halo boxes over the stash slots / the delta slots
+  std::vector<CUtensorMap> tm_hf_O;             // forward output (next layer's stash slots, or the pre-pool buffer) as 8 x 16 pixel boxes
   bool upd_maps = false;                        // fused update streamed by TMA (fully connected layers, 128-wide tiles)
   CUtensorMap tm_u_W, tm_u_M;                   // fp32 master / momentum as 32-column boxes
   std::vector<CUtensorMap> tm_u_R;              // each ring slot as 32-column bf16 boxes
@@ -329,6 +335,9 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.bn_d = y.ld_in <= 64 ? 64 : 128;
       y.bn_g = y.ld_in <= 64 ? 64 : 128;
       y.split_f = y.split_d = 1;
+      const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
+      y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
+      y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
       // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: split the
       // pixel range until about two CTAs per SM exist
       const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
@@ -421,6 +430,29 @@ static int build_tensor_maps(lp_ctx* c) {
                                       y.box128.bw, y.box128.bh, y.box128.bn, &err)) != LP_OK) return fail(c, rc, err);
         if ((rc = make_tmap_bf16_nhwc(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
                                       y.box64.bw, y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
+      }
+      if (y.halo_f) {
+        y.tm_hf_A.resize(y.x_slots);
+        for (int s = 0; s < y.x_slots; ++s)
+          if ((rc = make_tmap_bf16_nhwc(&y.tm_hf_A[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, HALO_W, HALO_H, 1,
+                                        &err)) != LP_OK) return fail(c, rc, err);
+      }
+      if (y.halo_f) {
+        // the layer's output: NHWC [B][H][W][ld_out], one map per destination
+        Layer& nx = c->L[l + 1];
+        const int n_dst = y.pool ? 1 : nx.x_slots;
+        y.tm_hf_O.resize(n_dst);
+        for (int s = 0; s < n_dst; ++s) {
+          const __nv_bfloat16* dst = y.pool ? y.a_full : nx.X + size_t(s) * nx.x_elems;
+          if ((rc = make_tmap_bf16_nhwc(&y.tm_hf_O[s], dst, y.ld_out, y.imW, y.imH, B, y.ld_out, 8, 16, 1, &err)) != LP_OK)
+            return fail(c, rc, err);
+        }
+      }
+      if (y.halo_d) {
+        y.tm_hd_A.resize(kDeltaSlots);
+        for (int s = 0; s < kDeltaSlots; ++s)
+          if ((rc = make_tmap_bf16_nhwc(&y.tm_hd_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out, HALO_W,
+                                        HALO_H, 1, &err)) != LP_OK) return fail(c, rc, err);
       }
       for (int s = 0; s < y.slots; ++s) {
         if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64, y.bn_f, &err)) != LP_OK)
@@ -518,6 +550,20 @@ static ConvGeom conv_geom(const Layer& y, int kind, const PixBox& bx, int flip, 
   return g;
 }
 
+// geometry of the halo-tile kernel: 8 x 16 pixel tiles of one image
+static ConvGeom halo_geom(const Layer& y, int flip) {
+  ConvGeom g{};
+  g.kind = GEOM_PIX_M;
+  g.H = y.imH; g.W = y.imW;
+  g.lw = 3; g.lh = 4;
+  g.tiles_w = y.imW / 8; g.tiles_h = y.imH / 16;
+  g.S = 3; g.pad = 1;
+  g.flip = flip;
+  g.chunks_per_tap = 1;
+  g.tap_pitch = y.ld_in;
+  return g;
+}
+
 static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
   Layer& y = c->L[l];
   const int nL = int(c->L.size());
@@ -553,6 +599,11 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   a.splits = y.split_f; a.partial = y.part_f; a.tile_counter = y.cnt_f;
   ++c->launches;
   TimedScope ts(c, LP_TASK_FORWARD, st);
+  if (y.halo_f) {
+    a.g = halo_geom(y, 0);
+    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
+    return conv_halo_launch(0, y.tm_hf_A[n % y.x_slots], y.tm_f_B[ring_slot], tmo, a, st);
+  }
   return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
 }
 
@@ -608,6 +659,10 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
   a.splits = y.split_d; a.partial = y.part_d; a.tile_counter = y.cnt_d;
   ++c->launches;
   TimedScope ts(c, LP_TASK_DELTA, st);
+  if (y.halo_d) {
+    a.g = halo_geom(y, 1);
+    return conv_halo_launch(1, y.tm_hd_A[n % kDeltaSlots], y.tm_d_B[ring_slot], y.tm_hd_A[0], a, st);
+  }
   return gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
 }
 

@@ -186,6 +186,10 @@ def test_tasks_small_convnet():
     from paper_2108_06629_b200 import inputs as I
     layers = I.vgg(16, [16, 32, "P", 64, "P", 72, "P"], [40, 10])
     run_teacher_forced(layers, 16, 4, None, 0.05, 0.9, 4)
+    # 32 x 32 and 16 x 16 images with at most 64 channels: the halo-tile kernel (one fetch of the
+    # activation box per 8 x 16 pixel tile) for forward and delta, the latter also behind a pool
+    layers = I.vgg(32, [16, "P", 32, 24, "P"], [10])
+    run_teacher_forced(layers, 4, 3, None, 0.05, 0.9, 3)
 
 
 def test_tasks_vgg_small_32_full_config():
