@@ -24,11 +24,14 @@ constexpr int HALO_STAGES = 4;
 constexpr int HALO_BYTES = HALO_W * HALO_H * 128;             // 64 bf16 channels per pixel
 constexpr int HALO_TAP_BYTES = 64 * 64 * 2;                   // one weight tap: 64 x 64 bf16
 constexpr int HALO_OUT_BYTES = GEMM_BM * 128;                 // forward: one output tile, 128 pixels x 64 bf16 channels
-constexpr int HALO_SMEM_BYTES = 9 * HALO_TAP_BYTES + HALO_STAGES * HALO_BYTES + 2 * HALO_OUT_BYTES + EPI_TILE_BYTES + 256 + 1024;
+constexpr int HALO_THREADS = 320;                             // producer warp, MMA warp, eight epilogue warps
+constexpr int HALO_EPI_BYTES = 2 * EPI_TILE_BYTES;            // forward: two output tiles (32 KiB); delta: eight transposition tiles (36 KiB)
+static_assert(HALO_EPI_BYTES >= 2 * HALO_OUT_BYTES, "the epilogue area holds two output tiles");
+constexpr int HALO_SMEM_BYTES = 9 * HALO_TAP_BYTES + HALO_STAGES * HALO_BYTES + HALO_EPI_BYTES + 256 + 1024;
 static_assert((HALO_STAGES * HALO_BYTES) % 1024 == 0, "the buffers behind the halo boxes stay 1 KiB aligned");
 
 template <bool B_MN, int MODE>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(HALO_THREADS, 1)
 conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmO, const GemmArgs p, const int tiles_total) {
   constexpr int BN = 64;
@@ -36,9 +39,9 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sB = smem;                                   // [9][64 x 64] weight taps
   uint8_t* sA = smem + 9 * HALO_TAP_BYTES;              // [HALO_STAGES] halo boxes
-  uint8_t* sO = sA + HALO_STAGES * HALO_BYTES;                    // [2] output tiles of the forward epilogue (TMA store sources)
-  float* epi_tile = reinterpret_cast<float*>(sO + 2 * HALO_OUT_BYTES);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(epi_tile) + EPI_TILE_BYTES);
+  uint8_t* sO = sA + HALO_STAGES * HALO_BYTES;                    // forward: [2] output tiles (TMA store sources)
+  float* epi_tile = reinterpret_cast<float*>(sO);                 // delta: one transposition tile per epilogue warp (same area)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sO + HALO_EPI_BYTES);
   uint64_t* wfull = bars;          // weights resident
   uint64_t* afull = bars + 1;                       // [HALO_STAGES] halo box landed
   uint64_t* aempty = afull + HALO_STAGES;           // [HALO_STAGES] halo box consumed
@@ -59,7 +62,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&accf[b], 1);
-      mbar_init(&acce[b], 4);
+      mbar_init(&acce[b], 8);      // one arrival per epilogue warp
     }
     fence_barrier_init();
   }
@@ -149,12 +152,24 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!ok) atomicExch(p.status, 2);
     }
   } else {
+    // Eight warps: warp w reads tensor-memory lanes 32 * (w % 4) (the rows of its quarter of the
+    // tile) and takes columns 32 * half .. + 32.  With one warp per scheduler there is nothing to
+    // hide an instruction's latency behind, so the epilogue is spread as wide as the tile allows.
     const int q = warp & 3;
-    float* tile = epi_tile + q * (32 * EPI_PITCH);
+    const int half = (warp - 2) >> 2;
+    float* tile = epi_tile + (warp - 2) * (32 * EPI_PITCH);
     const int sub_row = lane >> 3;
     const int sub_col = (lane & 7) * 4;
     uint32_t it = 0;
     bool dead = false;      // a wait ran out: keep the named-barrier count, touch nothing else
+    // the bias of this warp's 32 output channels does not depend on the tile (rows are padded to 8 with zeros)
+    float4 bias4[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const int n = half * 32 + 4 * g;
+      bias4[g] = (MODE == EPI_FPROP && p.bias != nullptr && n < p.N) ? __ldg(reinterpret_cast<const float4*>(p.bias + n))
+                                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     int tw = tw_begin - 1, th = th_begin, tn = tn_begin;
     for (int t = t_begin; t < t_end; ++t, ++it) {
       const uint32_t buf = it & 1u;
@@ -185,46 +200,40 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int trow = q * 32 + lane;
         const uint32_t so = smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES) + uint32_t(trow) * 128u;
         const uint32_t swz = uint32_t(trow & 7);
-        uint32_t packed[32];
-#pragma unroll
-        for (int c = 0; c < BN / 32; ++c) {
-          if (dead) break;
+        uint32_t packed[16];
+        if (!dead) {
           uint32_t r[32];
-          tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+          tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(half * 32), r);
           tmem_ld_wait();
-          if (c == BN / 32 - 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acce[buf]);
-          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acce[buf]);
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const int n = c * 32 + j;
-            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (p.bias != nullptr && n < p.N) b = __ldg(reinterpret_cast<const float4*>(p.bias + n));   // bias rows are padded to 8 with zeros
-            float v[4] = {__uint_as_float(r[j]) + b.x, __uint_as_float(r[j + 1]) + b.y, __uint_as_float(r[j + 2]) + b.z,
-                          __uint_as_float(r[j + 3]) + b.w};
+          for (int g = 0; g < 8; ++g) {
+            const int n = half * 32 + 4 * g;
+            float v[4] = {__uint_as_float(r[4 * g]) + bias4[g].x, __uint_as_float(r[4 * g + 1]) + bias4[g].y,
+                          __uint_as_float(r[4 * g + 2]) + bias4[g].z, __uint_as_float(r[4 * g + 3]) + bias4[g].w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               if (n + e >= p.N) v[e] = 0.f;
               else if (p.act == ACT_RELU) v[e] = fmaxf(v[e], 0.f);
             }
-            packed[(n >> 1)] = pack_bf16x2(v[0], v[1]);
-            packed[(n >> 1) + 1] = pack_bf16x2(v[2], v[3]);
+            packed[2 * g] = pack_bf16x2(v[0], v[1]);
+            packed[2 * g + 1] = pack_bf16x2(v[2], v[3]);
           }
         }
         // the staging tile of two tiles ago must have been read by its store
         if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (!dead) {
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(so + ((uint32_t(u) ^ swz) << 4)), "r"(packed[4 * u]),
+          for (int u = 0; u < 4; ++u)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(so + ((uint32_t(half * 4 + u) ^ swz) << 4)), "r"(packed[4 * u]),
                          "r"(packed[4 * u + 1]), "r"(packed[4 * u + 2]), "r"(packed[4 * u + 3])
                          : "memory");
         }
         fence_proxy_async_smem();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (threadIdx.x == 64 && !dead) {
           asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
                            reinterpret_cast<uint64_t>(&tmO)),
@@ -234,17 +243,15 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         continue;
       }
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      {
+        const int c = half;
         uint32_t r[32];
         __syncwarp();
         tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
         tmem_ld_wait();
-        if (c == BN / 32 - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&acce[buf]);
-        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acce[buf]);
 #pragma unroll
         for (int g = 0; g < 8; ++g)
           *reinterpret_cast<uint4*>(tile + lane * EPI_PITCH + g * 4) = make_uint4(r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);

@@ -305,7 +305,7 @@ cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMa
   const int grid = std::min(tiles, sm_count());
 #define LP_TRYH(B, M)                                                                                          \
   if (b_mn == B && args.mode == M) {                                                                           \
-    conv_halo_kernel<B, M><<<grid, GEMM_THREADS, HALO_SMEM_BYTES, st>>>(tmA, tmB, tmO, args, tiles);                \
+    conv_halo_kernel<B, M><<<grid, HALO_THREADS, HALO_SMEM_BYTES, st>>>(tmA, tmB, tmO, args, tiles);                \
     return cudaGetLastError();                                                                                 \
   }
   LP_FOR_EACH_HALO_VARIANT(LP_TRYH)
