@@ -42,7 +42,8 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
 // 3x3 convolution forward (which = 0) / delta (which = 1) with at most 64 channels on both sides:
 // tmA = NHWC tensor map with a 64 x 16 x 18 x 1 box, tmB = the layer's weight map (64 x 64 boxes);
 // args.g describes 8 x 16 pixel tiles (lw = 3, lh = 4).  tmO (forward only; any valid map otherwise): the
-// NHWC output with a 64 x 8 x 16 x 1 box, written by TMA stores.
+// NHWC output with a 64 x 8 x 16 x 1 box, written by TMA stores.  With plain geometry (which = 0 only) the
+// call is a forward GEMM with K <= 64 and N <= 64: tmA and tmO are 2-D maps with 64 x 128 boxes.
 cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
                              const GemmArgs& args, cudaStream_t stream);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process

@@ -14,6 +14,12 @@
 // (checked tap by tap with one-hot weights: exact with the descriptor's base-offset field left
 // zero, chunk-permuted when it is set to the start row).  All nine 64 x 64 weight taps stay resident in shared memory (72 KiB) for the whole
 // persistent CTA.  Per tile the SM now reads 22.5 KiB instead of 216 KiB; four boxes are in flight.
+//
+// The same pipeline also runs the forward GEMM of a layer whose whole contraction fits one
+// k-block and whose output is at most 64 columns wide (plain geometry: the patch-matrix form of
+// a first convolution layer): one weight "tap", tiles of 128 consecutive rows fetched through a
+// 2-D map, the output tile stored through a 2-D map.  Such a layer is 25 000 tiles of a single
+// k-block each, and what it needs is this kernel's epilogue.
 #pragma once
 #include "gemm.cuh"
 
@@ -76,29 +82,37 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   // CTA b works through the contiguous tile range [t_begin, t_end): neighbouring tiles share halo
   // pixels in L2, and the tile coordinates advance without divisions.
-  const int tiles_per_image = p.g.tiles_w * p.g.tiles_h;
+  const bool plain = (p.g.kind == GEOM_PLAIN);          // one tap, 128 consecutive rows per tile
+  const int ntaps = plain ? 1 : 9;
+  const int tiles_per_image = plain ? 1 : p.g.tiles_w * p.g.tiles_h;
   const int per_cta = (tiles_total + int(gridDim.x) - 1) / int(gridDim.x);
   const int t_begin = min(int(blockIdx.x) * per_cta, tiles_total);
   const int t_end = min(t_begin + per_cta, tiles_total);
-  const int tw_begin = t_begin % p.g.tiles_w, th_begin = (t_begin / p.g.tiles_w) % p.g.tiles_h, tn_begin = t_begin / tiles_per_image;
+  const int tw_begin = plain ? 0 : t_begin % p.g.tiles_w, th_begin = plain ? 0 : (t_begin / p.g.tiles_w) % p.g.tiles_h;
+  const int tn_begin = t_begin / tiles_per_image;
 
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
       int issued = 0;
-      mbar_arrive_expect_tx(wfull, 9 * HALO_TAP_BYTES);
-      for (int tap = 0; tap < 9; ++tap) tma_load_2d(sB + tap * HALO_TAP_BYTES, &tmB, wfull, tap * p.g.tap_pitch, 0);
+      mbar_arrive_expect_tx(wfull, uint32_t(ntaps) * HALO_TAP_BYTES);
+      for (int tap = 0; tap < ntaps; ++tap) tma_load_2d(sB + tap * HALO_TAP_BYTES, &tmB, wfull, tap * p.g.tap_pitch, 0);
       uint32_t st = 0, sph = 0;
       int tw = tw_begin, th = th_begin, n = tn_begin;
       for (int t = t_begin; t < t_end; ++t) {
         ok = mbar_wait(&aempty[st], sph ^ 1u);
         if (!ok) break;
-        mbar_arrive_expect_tx(&afull[st], HALO_BYTES);
-        // the box starts one pixel left of and above the tile; pixels outside the image read zero (= the padding)
-        tma_load_4d(sA + st * HALO_BYTES, &tmA, &afull[st], 0, tw * 8 - 1, th * 16 - 1, n);
+        if (plain) {
+          mbar_arrive_expect_tx(&afull[st], GEMM_A_BYTES);
+          tma_load_2d(sA + st * HALO_BYTES, &tmA, &afull[st], 0, t * GEMM_BM);
+        } else {
+          mbar_arrive_expect_tx(&afull[st], HALO_BYTES);
+          // the box starts one pixel left of and above the tile; pixels outside the image read zero (= the padding)
+          tma_load_4d(sA + st * HALO_BYTES, &tmA, &afull[st], 0, tw * 8 - 1, th * 16 - 1, n);
+          if (++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++n; } }
+        }
         ++issued;
         if (++st == uint32_t(HALO_STAGES)) { st = 0; sph ^= 1u; }
-        if (++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++n; } }
       }
       if (!ok) {
         atomicExch(p.status, 1);
@@ -114,7 +128,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       // One thread issues 36 MMAs per tile, so everything that can be is computed once: the
       // descriptors of box 0 / tap 0, and per tap the start-address offset of its view (the
       // address field counts 16-byte units and never carries out of the low word).
-      const uint64_t dA = make_smem_desc(smem_u32(sA), 16, HALO_W * 128);
+      const uint64_t dA = make_smem_desc(smem_u32(sA), 16, plain ? 1024 : HALO_W * 128);
       const uint64_t dB = B_MN ? make_smem_desc(smem_u32(sB), 8192, 1024) : make_smem_desc(smem_u32(sB), 16, 1024);
       const uint32_t dA_lo0 = uint32_t(dA), dA_hi = uint32_t(dA >> 32), dB_lo0 = uint32_t(dB), dB_hi = uint32_t(dB >> 32);
       uint32_t tap_off[9];
@@ -138,6 +152,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t acc = 0;
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap) {
+          if (tap >= ntaps) break;
 #pragma unroll
           for (int j = 0; j < GEMM_BK / 16; ++j) {
             umma_f16_lohi(tacc, a_lo + tap_off[tap] + uint32_t(j * 2), dA_hi,
@@ -173,9 +188,9 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int tw = tw_begin - 1, th = th_begin, tn = tn_begin;
     for (int t = t_begin; t < t_end; ++t, ++it) {
       const uint32_t buf = it & 1u;
-      if (++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++tn; } }
+      if (!plain && ++tw == p.g.tiles_w) { tw = 0; if (++th == p.g.tiles_h) { th = 0; ++tn; } }
       TileMap tm;
-      tm.m0 = 0;
+      tm.m0 = t * GEMM_BM;            // (plain geometry)
       tm.n0 = 0;
       tm.nlim = p.N;
       tm.pw0 = tw * 8;
@@ -235,10 +250,14 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         fence_proxy_async_smem();
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (threadIdx.x == 64 && !dead) {
-          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
-                           reinterpret_cast<uint64_t>(&tmO)),
-                       "r"(smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES)), "r"(0), "r"(tm.pw0), "r"(tm.ph0), "r"(tm.pn0)
-                       : "memory");
+          if (plain) {
+            tma_store_2d_addr(&tmO, smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES), 0, tm.m0);
+          } else {
+            asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                             reinterpret_cast<uint64_t>(&tmO)),
+                         "r"(smem_u32(sO) + buf * uint32_t(HALO_OUT_BYTES)), "r"(0), "r"(tm.pw0), "r"(tm.ph0), "r"(tm.pn0)
+                         : "memory");
+          }
           tma_store_commit();
         }
         continue;

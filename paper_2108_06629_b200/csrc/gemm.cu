@@ -301,7 +301,8 @@ static cudaError_t configure_pair() {
 cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
                              const GemmArgs& args, cudaStream_t st) {
   const bool b_mn = (which != 0);
-  const int tiles = args.g.tiles_w * args.g.tiles_h * (args.M / (args.g.H * args.g.W));
+  const int tiles = args.g.kind == GEOM_PLAIN ? (args.M + GEMM_BM - 1) / GEMM_BM
+                                               : args.g.tiles_w * args.g.tiles_h * (args.M / (args.g.H * args.g.W));
   const int grid = std::min(tiles, sm_count());
 #define LP_TRYH(B, M)                                                                                          \
   if (b_mn == B && args.mode == M) {                                                                           \

@@ -89,6 +89,7 @@ struct Layer {
   // 3x3 layers with at most 64 channels on both sides and images tiled by 8 x 16 pixels: the
   // activation / delta box is fetched once per tile with its halo (see conv_halo.cuh)
   bool halo_f = false, halo_d = false;
+  bool lean_f = false;                          // patch-matrix layer with at most 64 output channels: forward through the same kernel
   std::vector<CUtensorMap> tm_hf_A, tm_hd_A;    // halo boxes over the stash slots / the delta slots
   std::vector<CUtensorMap> tm_hf_O;             // forward output (next layer's stash slots, or the pre-pool buffer) as 8 x 16 pixel boxes
   bool upd_maps = false;                        // fused update streamed by TMA (fully connected layers, 128-wide tiles)
@@ -338,6 +339,7 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
       y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
+      y.lean_f = y.patch && y.n_out <= 64 && y.ld_in <= 64 && l + 1 < n;
       // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: split the
       // pixel range until about two CTAs per SM exist
       const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
@@ -461,6 +463,16 @@ static int build_tensor_maps(lp_ctx* c) {
           return fail(c, rc, err);
       }
       continue;
+    }
+    if (y.lean_f) {
+      Layer& nx = c->L[l + 1];
+      const int n_dst = y.pool ? 1 : nx.x_slots;
+      y.tm_hf_O.resize(n_dst);
+      for (int s = 0; s < n_dst; ++s) {
+        const __nv_bfloat16* dst = y.pool ? y.a_full : nx.X + size_t(s) * nx.x_elems;
+        if ((rc = make_tmap_bf16_2d(&y.tm_hf_O[s], dst, y.ld_out, y.out_rows, y.ld_out, 64, GEMM_BM, &err)) != LP_OK)
+          return fail(c, rc, err);
+      }
     }
     // (fully connected layers, and the patch layer whose rows are pixels)
     // forward: A = a^{l-1} [B][in] K-major; B = W [out][in] K-major
@@ -599,6 +611,10 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   a.splits = y.split_f; a.partial = y.part_f; a.tile_counter = y.cnt_f;
   ++c->launches;
   TimedScope ts(c, LP_TASK_FORWARD, st);
+  if (y.lean_f) {
+    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
+    return conv_halo_launch(0, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], tmo, a, st);
+  }
   if (y.halo_f) {
     a.g = halo_geom(y, 0);
     const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
