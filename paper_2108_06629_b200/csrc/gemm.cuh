@@ -178,6 +178,37 @@ __device__ __forceinline__ void dgrad_store4(const GemmArgs& p, int row, int n, 
       make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
 }
 
+// The layer below ended in ReLU + 2x2 max pool: output row `row`, column n of the delta product
+// lives on the pooled grid; pooled pixel pp, channel c, and the 2x2 window it came from.
+struct UnpoolPos {
+  int pp, c, pn, ph, pw;
+};
+__device__ __forceinline__ UnpoolPos unpool_pos(const GemmArgs& p, int row, int n) {
+  UnpoolPos u;
+  const int C = p.pool_C;
+  u.pp = row * p.pool_ppr + n / C;
+  u.c = n % C;
+  u.pw = u.pp % p.pool_Wp;
+  u.ph = (u.pp / p.pool_Wp) % p.pool_Hp;
+  u.pn = u.pp / (p.pool_Wp * p.pool_Hp);
+  return u;
+}
+// Routes four channels of the gradient to the recorded maximum of the window (idx: one byte per
+// channel, 0..3), gated by the pooled activation av (ReLU); the three other positions get zeros.
+__device__ __forceinline__ void unpool_store4(const GemmArgs& p, const UnpoolPos& u, const float v[4], uint32_t idx, uint2 av) {
+  const float a[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
+  __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int oh = 2 * u.ph + (k >> 1), ow = 2 * u.pw + (k & 1);
+    float d[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) d[j] = (((idx >> (8 * j)) & 0xFFu) == uint32_t(k) && a[j] > 0.f) ? v[j] : 0.f;
+    const size_t off = (size_t(u.pn * 2 * p.pool_Hp + oh) * (2 * p.pool_Wp) + ow) * p.ld_out + u.c;
+    *reinterpret_cast<uint2*>(o + off) = make_uint2(pack_bf16x2(d[0], d[1]), pack_bf16x2(d[2], d[3]));
+  }
+}
+
 // Epilogue for 4 consecutive columns n..n+3 of output row `row`.  Lanes past the column limit
 // inside the last 16-byte (fp32) / 8-element (bf16) group are written as zeros; groups that
 // start beyond that are skipped.
@@ -199,27 +230,11 @@ __device__ __forceinline__ void epilogue_store4(const GemmArgs& p, int row, int 
     if (p.act != ACT_NONE) av = *reinterpret_cast<const uint2*>(p.aux + size_t(row) * p.ld_aux + n);
     dgrad_store4(p, row, n, v, av);
   } else if (MODE == EPI_DGRAD_UNPOOL) {
-    // the layer below ended in ReLU + 2x2 max pool: route the gradient to the recorded maximum
     if (n >= N) return;
-    const int C = p.pool_C;
-    const int pp = row * p.pool_ppr + n / C;     // pooled pixel
-    const int c = n % C;
-    const int pw = pp % p.pool_Wp;
-    const int ph = (pp / p.pool_Wp) % p.pool_Hp;
-    const int pn = pp / (p.pool_Wp * p.pool_Hp);
-    const uint32_t idx = *reinterpret_cast<const uint32_t*>(p.pool_idx + size_t(pp) * C + c);
-    const uint2 av = *reinterpret_cast<const uint2*>(p.aux + size_t(pp) * p.ld_aux + c);
-    const float a[4] = {bf16_lo(av.x), bf16_hi(av.x), bf16_lo(av.y), bf16_hi(av.y)};
-    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int oh = 2 * ph + (k >> 1), ow = 2 * pw + (k & 1);
-      float d[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) d[j] = (((idx >> (8 * j)) & 0xFFu) == uint32_t(k) && a[j] > 0.f) ? v[j] : 0.f;
-      const size_t off = (size_t(pn * 2 * p.pool_Hp + oh) * (2 * p.pool_Wp) + ow) * p.ld_out + c;
-      *reinterpret_cast<uint2*>(o + off) = make_uint2(pack_bf16x2(d[0], d[1]), pack_bf16x2(d[2], d[3]));
-    }
+    const UnpoolPos u = unpool_pos(p, row, n);
+    const uint32_t idx = *reinterpret_cast<const uint32_t*>(p.pool_idx + size_t(u.pp) * p.pool_C + u.c);
+    const uint2 av = *reinterpret_cast<const uint2*>(p.aux + size_t(u.pp) * p.ld_aux + u.c);
+    unpool_store4(p, u, v, idx, av);
   } else {  // EPI_WGRAD_UPDATE (plain form, used after a split-K reduction)
     if (n >= n_pad8) return;
     const size_t off = size_t(row) * p.ld_out + n;
@@ -274,6 +289,25 @@ __device__ __forceinline__ void epilogue_rows8(const GemmArgs& p, const TileMap&
       const float4 a = *reinterpret_cast<const float4*>(tile + (i8 * 4 + sub_row) * EPI_PITCH + sub_col);
       const float v[4] = {n + 0 < N ? a.x : 0.f, n + 1 < N ? a.y : 0.f, n + 2 < N ? a.z : 0.f, n + 3 < N ? a.w : 0.f};
       dgrad_store4(p, rows[i8], n, v, av[i8]);
+    }
+  } else if constexpr (MODE == EPI_DGRAD_UNPOOL) {
+    if (n >= N) return;
+    UnpoolPos u[8];
+    uint32_t idx[8];
+    uint2 av[8];
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8) {
+      if (rows[i8] < 0) continue;
+      u[i8] = unpool_pos(p, rows[i8], n);
+      idx[i8] = *reinterpret_cast<const uint32_t*>(p.pool_idx + size_t(u[i8].pp) * p.pool_C + u[i8].c);
+      av[i8] = *reinterpret_cast<const uint2*>(p.aux + size_t(u[i8].pp) * p.ld_aux + u[i8].c);
+    }
+#pragma unroll
+    for (int i8 = 0; i8 < 8; ++i8) {
+      if (rows[i8] < 0) continue;
+      const float4 a = *reinterpret_cast<const float4*>(tile + (i8 * 4 + sub_row) * EPI_PITCH + sub_col);
+      const float v[4] = {n + 0 < N ? a.x : 0.f, n + 1 < N ? a.y : 0.f, n + 2 < N ? a.z : 0.f, n + 3 < N ? a.w : 0.f};
+      unpool_store4(p, u[i8], v, idx[i8], av[i8]);
     }
   } else {
 #pragma unroll
