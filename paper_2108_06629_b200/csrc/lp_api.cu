@@ -183,6 +183,7 @@ static int validate(const lp_layer* layers, int n, const lp_config* cfg, std::st
     if (y.kind == LP_CONV) {
       if (y.R != 3 || y.S != 3 || y.stride != 1 || y.pad != 1) { *why = "only 3x3 stride-1 pad-1 convolutions are built"; return LP_ERR_UNSUPPORTED; }
       if (y.H < 1 || y.W < 1) { *why = "bad image size"; return LP_ERR_INVALID_ARG; }
+      if ((long long)cfg->batch * y.H * y.W >= (1ll << 31) / 64) { *why = "batch x image size too large (pixel rows are indexed with 32 bits)"; return LP_ERR_UNSUPPORTED; }
       if (y.act == LP_ACT_GELU) { *why = "GELU after a convolution is not built"; return LP_ERR_UNSUPPORTED; }
       if (y.out % 8 != 0) { *why = "convolution output channels must be a multiple of 8"; return LP_ERR_UNSUPPORTED; }
       if (y.pool != 0 && (y.pool != 2 || y.H % 2 || y.W % 2 || y.act != LP_ACT_RELU)) { *why = "pooling must be 2x2 on even images after ReLU"; return LP_ERR_UNSUPPORTED; }

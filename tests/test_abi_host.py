@@ -89,6 +89,18 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(lpb.LayerPipeError) as e:
         lpb.lp_workspace_size(wl["layers"], 4, None, [3, 2, 1, -1], wl["batch"])
     assert e.value.code == lpb.LP_ERR_INVALID_ARG
+    # pixel rows are indexed with 32 bits: batch x image size beyond that is refused, not wrapped
+    big = I.vgg(2048, [64, "P"], [10])
+    with pytest.raises(lpb.LayerPipeError) as e:
+        lpb.lp_workspace_size(big, 1, None, None, 16)
+    assert e.value.code == lpb.LP_ERR_UNSUPPORTED
+    # a first convolution layer with three channels keeps 3x3 patch rows of 32 bf16 per pixel
+    small = I.vgg(16, [16, 32], [10])
+    sz = lpb.lp_workspace_size(small, 1, None, None, 8)
+    assert sz >= 2 * 8 * 16 * 16 * 32
+    # timeline access without a handle
+    n = __import__("ctypes").c_int()
+    assert lpb.lib().lp_get_task_timeline(None, 0, 0, None, None, n) == lpb.LP_ERR_INVALID_ARG
     lib = lpb.lib()
     assert lib.lp_step(None, None, None, None) == lpb.LP_ERR_INVALID_ARG
     assert lib.lp_destroy(None) == lpb.LP_ERR_INVALID_ARG
