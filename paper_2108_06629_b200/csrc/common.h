@@ -92,8 +92,10 @@ cudaError_t launch_sgd_update(const UpdateArgs& a, cudaStream_t stream);
 cudaError_t launch_maxpool2(const __nv_bfloat16* a, __nv_bfloat16* pooled, unsigned char* idx, int B, int H, int W,
                             int C, cudaStream_t stream);
 // Column sums of a [rows][ld] bf16 matrix in two deterministic passes: partial[chunk][col] over
-// chunks of kColsumChunk rows, then (inside launch_sgd_update) the chunks in order.
-constexpr int kColsumChunk = 2048;
+// chunks of colsum_chunk_rows(rows) rows, then (inside launch_sgd_update) the chunk sums on four
+// interleaved thread rows.  One pass (a serial loop over rows / 4 per thread) only up to 512 rows.
+inline int colsum_chunk_rows(int rows) { return rows <= 131072 ? 256 : 2048; }
+inline int colsum_chunks(int rows) { return rows > 512 ? (rows + colsum_chunk_rows(rows) - 1) / colsum_chunk_rows(rows) : 0; }
 cudaError_t launch_colsum_partial(const __nv_bfloat16* x, int rows, int ld, int n_cols, float* partial,
                                   cudaStream_t stream);
 cudaError_t launch_round_to_bf16(const float* src, __nv_bfloat16* dst, long long n_elems, cudaStream_t stream);

@@ -371,12 +371,12 @@ cudaError_t launch_maxpool2(const __nv_bfloat16* a, __nv_bfloat16* pooled, unsig
 
 // partial[chunk][col] = sum over the chunk's rows (in row order, 4-way interleaved like the
 // single-pass bias reduction) of x[row][col]
-__global__ void colsum_partial_kernel(const __nv_bfloat16* __restrict__ x, int rows, int ld, int n_cols,
+__global__ void colsum_partial_kernel(const __nv_bfloat16* __restrict__ x, int rows, int ld, int n_cols, int chunk_rows,
                                       float* __restrict__ partial) {
   __shared__ float part[4][64];
   const int tx = threadIdx.x % 64, ty = threadIdx.x / 64;
   const int col = blockIdx.x * 64 + tx;
-  const int r0 = blockIdx.y * kColsumChunk, r1 = min(rows, r0 + kColsumChunk);
+  const int r0 = blockIdx.y * chunk_rows, r1 = min(rows, r0 + chunk_rows);
   float acc = 0.f;
   if (col < n_cols)
     for (int r = r0 + ty; r < r1; r += 4) acc += __bfloat162float(x[(long long)r * ld + col]);
@@ -386,8 +386,9 @@ __global__ void colsum_partial_kernel(const __nv_bfloat16* __restrict__ x, int r
 }
 cudaError_t launch_colsum_partial(const __nv_bfloat16* x, int rows, int ld, int n_cols, float* partial,
                                   cudaStream_t stream) {
-  dim3 grid((n_cols + 63) / 64, (rows + kColsumChunk - 1) / kColsumChunk);
-  colsum_partial_kernel<<<grid, 256, 0, stream>>>(x, rows, ld, n_cols, partial);
+  const int chunk = colsum_chunk_rows(rows);
+  dim3 grid((n_cols + 63) / 64, (rows + chunk - 1) / chunk);
+  colsum_partial_kernel<<<grid, 256, 0, stream>>>(x, rows, ld, n_cols, chunk, partial);
   return cudaGetLastError();
 }
 }  // namespace lp

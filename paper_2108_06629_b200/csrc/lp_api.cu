@@ -359,7 +359,7 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.split_d = y.bn_d == GEMM_BN_PAIR ? 1 : gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
       y.split_g = 1;
     }
-    y.col_chunks = y.out_rows > 8192 ? (y.out_rows + kColsumChunk - 1) / kColsumChunk : 0;
+    y.col_chunks = colsum_chunks(y.out_rows);
   }
   c->classes = layers[n - 1].out;
   c->ld_cls = pad8(c->classes);
