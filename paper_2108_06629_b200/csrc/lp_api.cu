@@ -14,6 +14,7 @@
 //   layer run concurrently and delta^{l-1} is released as soon as delta_l is done.
 //   Fused-B schedule: delta_l, G_l, U_l run back to back as ONE task on the stage's
 //   backward stream and delta^{l-1} is released only when the whole task has finished.
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -341,12 +342,16 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
       y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
       y.lean_f = y.patch && y.n_out <= 64 && y.ld_in <= 64 && l + 1 < n;
-      // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: split the
-      // pixel range until about two CTAs per SM exist
+      // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: the pixel
+      // range is split.  A split costs the last CTA of the tile one more partial tile to add
+      // (measured about 1.1 us for a 128-wide tile, half that for 64), a k-block about 0.33 us, so
+      // the time kb/s * 0.33 + s * 1.1 is least near s = sqrt(0.3 kb) (0.6 kb for 64-wide tiles);
+      // never more splits than fill two CTAs per SM.  Swept on the small VGG (2 .. 148 splits):
+      // the measured optimum of every layer is the power of two next to this value.
       const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
       const int num_kb = y.in_rows / GEMM_BK;
-      // (the patch layer has a single tile: one CTA per SM, each a long run of small k-blocks)
-      y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), num_kb / 8), y.patch ? 148 : 64));
+      const int s_opt = int(std::lround(std::sqrt(double(num_kb) * (y.bn_g <= 64 ? 0.6 : 0.3))));
+      y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), s_opt), y.patch ? 148 : 64));
       const int per = (num_kb + y.split_g - 1) / y.split_g;
       y.split_g = (num_kb + per - 1) / per;
     } else {
