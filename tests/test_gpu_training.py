@@ -223,6 +223,39 @@ def test_serial_tasks_agree_and_timeline_is_consistent():
     tr.close()
 
 
+def test_fewer_hardware_queues_fold_the_stages_and_change_nothing():
+    """With CUDA_DEVICE_MAX_CONNECTIONS = 8 (the CUDA default) lp_create folds the stages onto two
+    stream triples; the tensors must be bit-identical to the unfolded run.  The variable is read
+    when the CUDA context is created, so the folded run is a child process."""
+    import json
+    import os
+    import subprocess
+    import sys
+    import tempfile
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 136, 40], "gelu")
+    a, _, _ = free_run(layers, 56, 4, [3, 2, 1, 0], 0.02, 0.9, 8, lpb.LP_SCHED_LAYERPIPE)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child = (
+        "import sys, json, numpy as np\n"
+        "sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+        "import test_gpu_training as T\n"
+        "from paper_2108_06629_b200 import binding as lpb, inputs as I\n"
+        "layers = I.mlp([264, 192, 320, 136, 40], 'gelu')\n"
+        "a, _, _ = T.free_run(layers, 56, 4, [3, 2, 1, 0], 0.02, 0.9, 8, lpb.LP_SCHED_LAYERPIPE)\n"
+        "np.savez(sys.argv[1], loss=np.array(a['loss']), **{'W%%d' %% l: a['W'][l][0] for l in range(len(layers))})\n"
+    ) % (root, os.path.join(root, "tests"))
+    with tempfile.TemporaryDirectory() as d:
+        out = os.path.join(d, "folded.npz")
+        env = dict(os.environ, CUDA_DEVICE_MAX_CONNECTIONS="8")
+        subprocess.run([sys.executable, "-c", child, out], check=True, env=env, timeout=600)
+        z = np.load(out)
+        for l in range(len(layers)):
+            assert np.array_equal(z["W%d" % l], a["W"][l][0])
+        assert np.array_equal(z["loss"], np.array(a["loss"]))
+
+
 def test_patch_matrix_of_the_first_convolution_layer():
     """A first convolution layer with three input channels keeps its input as the matrix of 3x3
     patches.  After one step the first layer's output (the second layer's stashed input) must be
