@@ -92,6 +92,11 @@ struct GemmArgs {
   int persistent;           // CTAs loop over tiles (grid sized to the machine) instead of one tile each
   int l2_ahead;             // plain GEMM: k-blocks of the B operand to pull into L2 ahead of the pipeline (0 = off)
   int upd_tma;              // EPI_WGRAD_UPDATE: master / momentum / ring tiles move by TMA through the stage ring
+  // EPI_WGRAD_UPDATE with the TMA update: the bias gradient (column sums of delta^l over the batch)
+  // and the bias update of Eq. 6, done by the CTAs of the first column tile (bdelta null = off)
+  const __nv_bfloat16* bdelta;   // delta^l [brows][bld]
+  int bld, brows;
+  float *bb, *bmb, *bdb, *bbring;   // bias master, momentum (may be null), gradient, destination ring slot
   int* status;              // device status word: set non-zero if a bounded wait expires
 };
 
@@ -719,6 +724,33 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t smem0 = smem_u32(smem), full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
           const uint32_t ringbuf = full0 + 1024u;
           const int trow = q * 32 + lane;            // row of the tile this lane owns (tensor-memory lane)
+          if (p.bdelta != nullptr && tm.n0 == 0 && tm.m0 + trow < p.M) {
+            // Bias of output feature m = column sum of delta over the batch, then Eq. 6 -- while
+            // the tile's main loop runs.  Same order of additions as the stand-alone update
+            // kernel (four interleaved partial sums, combined in order), so both give the same bits.
+            const int m = tm.m0 + trow;
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
+            const __nv_bfloat16* src = p.bdelta + m;
+            int r = 0;
+#pragma unroll 4
+            for (; r + 4 <= p.brows; r += 4) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) part[i] += __bfloat162float(src[size_t(r + i) * p.bld]);
+            }
+            for (int i = 0; r + i < p.brows; ++i) part[i] += __bfloat162float(src[size_t(r + i) * p.bld]);
+            float g = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) g += part[i];
+            p.bdb[m] = g;
+            float mm = g;
+            if (p.bmb != nullptr) {
+              mm = p.mu * p.bmb[m] + g;
+              p.bmb[m] = mm;
+            }
+            const float b = p.bb[m] - p.lr * mm;
+            p.bb[m] = b;
+            p.bbring[m] = b;
+          }
           if (good) {
             good = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
             good = __all_sync(0xffffffffu, good);

@@ -689,6 +689,11 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
 }
 
 static inline bool fused_update(const lp_ctx* c) { return (c->cfg.flags & LP_UNFUSED_UPDATE) == 0; }
+// The G kernel with the TMA update also does the bias gradient and bias update of a fully connected
+// layer (one launch less per layer); convolution layers and the other G forms keep the bias kernel.
+static inline bool fused_bias(const lp_ctx* c, const Layer& y) {
+  return fused_update(c) && y.upd_maps && y.d.has_bias && y.col_chunks == 0 && !y.conv;
+}
 
 static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
@@ -714,6 +719,12 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   }
   ++c->launches;
   TimedScope ts(c, LP_TASK_G, st);
+  if (fused_bias(c, y)) {
+    a.bdelta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
+    a.bld = y.ld_out; a.brows = y.out_rows;
+    a.bb = y.b; a.bmb = y.mb; a.bdb = y.db;
+    a.bbring = y.bring + size_t((n + 1) % y.slots) * y.ld_out;
+  }
   if (y.upd_maps && a.mode == EPI_WGRAD_UPDATE) {
     UpdMaps um;
     um.W = y.tm_u_W;
@@ -732,6 +743,7 @@ static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st)
   u.ring = y.ring + size_t(dst_slot) * y.w_elems;
   u.n_elems = fused_update(c) ? 0 : (long long)y.w_elems;   // fused: W was updated by the G kernel
   if (u.n_elems == 0 && !y.d.has_bias) return cudaSuccess;  // nothing left to do
+  if (fused_bias(c, y)) return cudaSuccess;                 // the G kernel did the bias as well
   if (y.d.has_bias) {
     u.delta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
     u.rows = y.out_rows; u.ldd = y.ld_out; u.n_out = y.n_out;

@@ -212,7 +212,10 @@ def test_serial_tasks_agree_and_timeline_is_consistent():
     for kind, count in expect.items():
         st, en = tr.task_timeline(kind)
         n, tot = tr.task_time(kind)
-        assert len(st) == count == n
+        if kind == "update":        # fully connected layers do the bias update inside the G kernel
+            assert len(st) == n and n in (0, count)
+        else:
+            assert len(st) == count == n
         assert np.all(en >= st) and np.all(np.diff(st) > 0)
         assert abs(float(np.sum(en - st)) - tot) <= 1e-3 * max(tot, 1e-3) + 1e-3
         spans += list(zip(st.tolist(), en.tolist()))
