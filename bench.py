@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
 # ncu capture summarised under profiles/ (None until a capture exists for that pair).
 NCU_TRAFFIC_BYTES = {
-    # profiles/gemm_G_fused_update_mlp8_4096.md: 139.57 MB read + 111.45 MB written inside the kernel window
+    # capture of the fused G + update kernel: 139.57 MB read + 111.45 MB written inside the kernel window
     ("mlp8_4096", "G"): 251.02e6,
 }
 
