@@ -221,13 +221,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);
           cur = nxt;
         } else {
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + sub_row;
-            const int row = row0 + rr;
-            const float4 acc = *reinterpret_cast<const float4*>(tile + rr * EPI_PITCH + sub_col);
-            if (row < p.M) epilogue_store4<MODE>(p, row, n, tm.nlim, acc);
-          }
+          epilogue_rows8<MODE>(p, tm, tile, q, sub_row, sub_col, n);
         }
       }
     }
