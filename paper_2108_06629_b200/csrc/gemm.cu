@@ -266,6 +266,7 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   while (s > 2 && size_t(s) * stage_bytes + 1280 > 227 * 1024) --s;
   a.num_stages = s;
   cudaLaunchConfig_t cfg = {};
+  // (convolution geometry: M is a whole number of 128-pixel boxes, and an even one -- the caller checks)
   cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N + GEMM2_BN - 1) / GEMM2_BN, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = size_t(s) * stage_bytes + 1024 + 256;
@@ -288,6 +289,7 @@ static cudaError_t configure_pair() {
   X(false, false, EPI_FPROP)          \
   X(false, false, EPI_STORE_F32)      \
   X(false, true, EPI_DGRAD)           \
+  X(false, true, EPI_DGRAD_UNPOOL)    \
   X(false, true, EPI_STORE_F32)       \
   X(true, true, EPI_STORE_F32)        \
   X(true, true, EPI_WGRAD_UPDATE)
@@ -339,7 +341,7 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
                         cudaStream_t st, const UpdMaps* um) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
   if (bn == GEMM_BN_PAIR) {
-    if (args.g.kind != GEOM_PLAIN) return cudaErrorInvalidValue;
+    if (args.g.kind == GEOM_PIX_K) return cudaErrorInvalidValue;
 #define LP_TRYP(A, B, M) \
   if (a_mn == A && b_mn == B && args.mode == M) return launch_pair<A, B, M>(tmA, tmB, args, st);
     LP_FOR_EACH_PAIR_VARIANT(LP_TRYP)

@@ -11,7 +11,9 @@
 // Hand-offs: TMA loads of both CTAs complete on the leader's "full" barrier (the leader arms it
 // with the byte count of both); tcgen05.commit multicasts the "empty" and "accumulator ready"
 // arrivals to the same barrier in both CTAs.  No TMA load uses cluster multicast.
-// Plain matrices only (no convolution geometry, no split-K); epilogues as in gemm.cuh.
+// Plain matrices, and the forward / delta contractions of 3x3 convolutions (GEOM_PIX_M: each
+// CTA's 128 rows are a box of 128 pixels fetched through the 4-D NHWC map, shifted by the
+// filter tap; one k-block = one tap x 64 channels); no split-K; epilogues as in gemm.cuh.
 #pragma once
 #include "gemm.cuh"
 
@@ -52,6 +54,14 @@ __device__ __forceinline__ void tma2_load_2d_addr(uint32_t smem_dst, const CUten
       "l"(reinterpret_cast<uint64_t>(m)), "r"(leader_bar), "r"(x), "r"(y)
       : "memory");
 }
+__device__ __forceinline__ void tma2_load_4d_addr(uint32_t smem_dst, const CUtensorMap* m, uint32_t leader_bar, int c0, int c1,
+                                                  int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+      "%4, %5, %6}], [%2];" ::"r"(smem_dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
 __device__ __forceinline__ void umma2_f16_lohi(uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
                                                uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -89,12 +99,20 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int num_kb = (p.K + GEMM_BK - 1) / GEMM_BK;
+  const bool pix = (p.g.kind == GEOM_PIX_M);
 
   TileMap tm;
   tm.m0 = (blockIdx.x >> 1) * 256 + int(rank) * 128;    // this CTA's 128 rows
   tm.n0 = blockIdx.y * GEMM2_BN;                        // the pair's 256 columns
   tm.nlim = p.N;
   tm.pn0 = tm.ph0 = tm.pw0 = 0;
+  if (pix) {                                            // this CTA's box of 128 pixels
+    const int bx = (blockIdx.x >> 1) * 2 + int(rank);
+    const int tw = bx % p.g.tiles_w, th = (bx / p.g.tiles_w) % p.g.tiles_h, tn = bx / (p.g.tiles_w * p.g.tiles_h);
+    tm.pw0 = tw << p.g.lw;
+    tm.ph0 = th << p.g.lh;
+    tm.pn0 = tn * (GEMM_BM >> (p.g.lw + p.g.lh));
+  }
   const int nb0 = tm.n0 + int(rank) * 128;              // the half of B this CTA stages
 
   if (threadIdx.x == 0) {
@@ -126,6 +144,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
       uint32_t s = 0, ph = 0;
       int k0 = 0;
+      int c_tap = 0, c_chunk = 0;                      // convolution: filter tap and 64-channel chunk of this k-block
       for (int kb = 0; kb < num_kb; ++kb, k0 += GEMM_BK) {
         ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
         if (!ok) break;
@@ -133,13 +152,27 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t sb = sa + GEMM_A_BYTES;
         const uint32_t fb = map_to_cta(full0 + 8u * s, 0);          // the leader's barrier
         if (rank == 0) mbar_arrive_expect_tx_addr(full0 + 8u * s, 2 * STAGE_BYTES);
-        if (A_MN) {
+        if (pix) {
+          const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
+          const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
+          const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;
+          tma2_load_4d_addr(sa, &tmA, fb, c_chunk * 64, tm.pw0 + sw, tm.ph0 + sh, tm.pn0);
+          if (B_MN) {   // delta: B[k = (tap, co)][n = ci]
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tma2_load_2d_addr(sb + c * 8192, &tmB, fb, c_tap * p.g.tap_pitch + nb0 + c * 64, c_chunk * 64);
+          } else {      // forward: B[n = co][k = (tap, ci)]
+            tma2_load_2d_addr(sb, &tmB, fb, c_tap * p.g.tap_pitch + c_chunk * 64, nb0);
+          }
+          if (++c_chunk == p.g.chunks_per_tap) { c_chunk = 0; ++c_tap; }
+        } else if (A_MN) {
 #pragma unroll
           for (int c = 0; c < 2; ++c) tma2_load_2d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, k0);
         } else {
           tma2_load_2d_addr(sa, &tmA, fb, k0, tm.m0);
         }
-        if (B_MN) {
+        if (pix) {
+          // (B was loaded with the tap's coordinates above)
+        } else if (B_MN) {
 #pragma unroll
           for (int c = 0; c < 2; ++c) tma2_load_2d_addr(sb + c * 8192, &tmB, fb, nb0 + c * 64, k0);
         } else {

@@ -337,6 +337,14 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.bn_f = y.n_out <= 64 ? 64 : 128;
       y.bn_d = y.ld_in <= 64 ? 64 : 128;
       y.bn_g = y.ld_in <= 64 ? 64 : 128;
+      // Wide layers (at least 256 channels on both sides) on an even number of pixel boxes:
+      // 256-pixel x 256-column tiles on SM pairs.  Measured on the VGG-16 layers at batch 64,
+      // pair against single CTA: 512 -> 512 at 28^2 forward 180 / 245 us, delta 189 / 253 us;
+      // 256 -> 256 at 56^2 216 / 240 and 230 / 249 us; 512 -> 512 at 14^2 66 / 79 and 67 / 84 us;
+      // 128 -> 256 forward (18 k-blocks) is slower as a pair (149 / 131 us) and stays single.
+      const bool even_boxes = ((y.in_rows / GEMM_BM) % 2) == 0;
+      if (even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
+      if (even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
       y.split_f = y.split_d = 1;
       const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
@@ -463,7 +471,8 @@ static int build_tensor_maps(lp_ctx* c) {
                                         HALO_H, 1, &err)) != LP_OK) return fail(c, rc, err);
       }
       for (int s = 0; s < y.slots; ++s) {
-        if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64, y.bn_f, &err)) != LP_OK)
+        if ((rc = make_tmap_bf16_2d(&y.tm_f_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64,
+                                    y.bn_f == GEMM_BN_PAIR ? 128 : y.bn_f, &err)) != LP_OK)   // a pair CTA stages half of the 256 columns
           return fail(c, rc, err);
         if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.w_ld, y.n_out, y.w_ld, 64, 64, &err)) != LP_OK)
           return fail(c, rc, err);
