@@ -126,12 +126,16 @@ void gemm_set_tuning(int bn, int stages, int splits) {
 // Split-K factor.  Measured on B200 (M = 256, N = K = 4096): the split main loop is shorter
 // but writing and re-reading the fp32 partial tiles costs more than it saves (25 us unsplit,
 // 28 / 35 / 52 us at 2 / 4 / 8 splits), and under the stage scheduler other kernels fill the
-// idle SMs anyway.  So the automatic choice is "off"; the path stays for experiments and is
-// covered by the tests through lp_set_tuning.
+// idle SMs anyway.  So the automatic choice is "off" for such shapes; the path is covered by the
+// tests through lp_set_tuning.
 int gemm_pick_splits(int M, int N, int K, int bn) {
-  (void)M; (void)N; (void)bn;
   const int num_kb = (K + GEMM_BK - 1) / GEMM_BK;
-  int s = g_force_splits > 0 ? g_force_splits : 1;
+  // The exception: a handful of tiles with a very long contraction (64 x 4096 x 25088: 32 tiles of
+  // 392 k-blocks, one CTA streaming 6.4 MB of weights each): 145 us unsplit, 95 / 74 / 89 us at
+  // 2 / 4 / 8 splits.
+  const long long tiles = (long long)((M + GEMM_BM - 1) / GEMM_BM) * ((N + bn - 1) / bn);
+  const int automatic = (tiles <= 48 && num_kb >= 256) ? 4 : 1;
+  int s = g_force_splits > 0 ? g_force_splits : automatic;
   s = std::max(1, std::min(s, num_kb));
   const int per = (num_kb + s - 1) / s;
   return (num_kb + per - 1) / per;      // no empty split
