@@ -46,6 +46,11 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
 // call is a forward GEMM with K <= 64 and N <= 64: tmA and tmO are 2-D maps with 64 x 128 boxes.
 cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
                              const GemmArgs& args, cudaStream_t stream);
+struct ConvGeom;
+struct HaloGUpdate;
+// G (+ fused update) of a halo-tile layer: tmX = the activations with the 64 x 10 x 18 x 1 halo box,
+// tmD = delta with a 64 x 8 x 16 x 1 box; partial: conv_halo_g_max_ctas() x 5 x 128 x 64 floats.
+int conv_halo_g_max_ctas();
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory; call once per process
 void gemm_set_tuning(int bn, int stages, int splits);   // 0 = automatic
 int gemm_pick_splits(int M, int N, int K, int bn);

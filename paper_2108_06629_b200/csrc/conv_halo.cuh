@@ -289,4 +289,193 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// G (Eq. 5) of the same layers: G[co][tap][ci] = sum over pixels of delta[px][co] a[px + tap][ci].
+//
+// The general kernel gives every (tap, 64-pixel k-block) its own pair of TMA loads, so the nine
+// taps re-read delta and the activations nine times through L2, and with 64 output channels
+// only half of each 128-row MMA is used.  Here the contraction runs over 8 x 16 pixel tiles:
+// per tile one delta box (128 pixels x 64 channels, 16 KiB) and one activation halo box
+// (22.5 KiB) are fetched, and the TRANSPOSED gradient is accumulated,
+//   D[m = (tap pair half, ci)][n = co] += sum_px  A[px][m] B[px][n],
+// with A = two shifted views of the halo box side by side (the descriptor's leading-dimension
+// stride, the distance between the two 64-wide halves of M, is the distance between the two
+// taps: one pixel = 128 bytes, or 1024 bytes from tap (r, 2) to tap (r + 1, 0)) and B = the delta
+// box.  Nine taps = four pairs and a single: five accumulators of 64 columns stay in tensor
+// memory over ALL tiles of the CTA; at the end each CTA writes its 5 x 128 x 64 partial sums and
+// a second small kernel adds the CTAs' partials in CTA order and applies Eq. 6.
+constexpr int HALOG_STAGES = 4;
+constexpr int HALOG_D_OFF = 24576;                              // delta box behind the halo box (1 KiB aligned)
+constexpr int HALOG_STAGE_BYTES = HALOG_D_OFF + GEMM_A_BYTES;   // 40 KiB
+constexpr int HALOG_SMEM_BYTES = HALOG_STAGES * HALOG_STAGE_BYTES + 256 + 1024;
+constexpr int HALOG_GROUPS = 5;
+constexpr int HALOG_PART_FLOATS = HALOG_GROUPS * GEMM_BM * 64;  // partial sums of one CTA
+
+template <int kInstance = 0>   // (a template only so that the header may be included by several translation units)
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD, const ConvGeom g,
+                   const int tiles_total, float* __restrict__ partial, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HALOG_STAGES * HALOG_STAGE_BYTES);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + HALOG_STAGES;
+  uint64_t* accf = empty + HALOG_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accf + 1);
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmX);
+    tma_prefetch_desc(&tmD);
+    for (int b = 0; b < HALOG_STAGES; ++b) {
+      mbar_init(&full[b], 1);
+      mbar_init(&empty[b], 1);
+    }
+    mbar_init(accf, 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int per_cta = (tiles_total + int(gridDim.x) - 1) / int(gridDim.x);
+  const int t_begin = min(int(blockIdx.x) * per_cta, tiles_total);
+  const int t_end = min(t_begin + per_cta, tiles_total);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int issued = 0;
+      uint32_t st = 0, sph = 0;
+      int tw = t_begin % g.tiles_w, th = (t_begin / g.tiles_w) % g.tiles_h, n = t_begin / (g.tiles_w * g.tiles_h);
+      for (int t = t_begin; t < t_end; ++t) {
+        ok = mbar_wait(&empty[st], sph ^ 1u);
+        if (!ok) break;
+        uint8_t* base = smem + st * HALOG_STAGE_BYTES;
+        mbar_arrive_expect_tx(&full[st], HALO_BYTES + GEMM_A_BYTES);
+        tma_load_4d(base, &tmX, &full[st], 0, tw * 8 - 1, th * 16 - 1, n);
+        tma_load_4d(base + HALOG_D_OFF, &tmD, &full[st], 0, tw * 8, th * 16, n);
+        ++issued;
+        if (++st == uint32_t(HALOG_STAGES)) { st = 0; sph ^= 1u; }
+        if (++tw == g.tiles_w) { tw = 0; if (++th == g.tiles_h) { th = 0; ++n; } }
+      }
+      if (!ok) {
+        atomicExch(status, 21);
+        for (int i = (issued > HALOG_STAGES ? issued - HALOG_STAGES : 0); i < issued; ++i)
+          mbar_wait(&full[i % HALOG_STAGES], uint32_t(i / HALOG_STAGES) & 1u);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(GEMM_BM, 64, true, true);
+      // tap groups: first tap of the group as a halo row offset, and the distance to its partner
+      const uint32_t first_row[HALOG_GROUPS] = {0u, 2u, uint32_t(HALO_W + 1), uint32_t(2 * HALO_W), uint32_t(2 * HALO_W + 2)};
+      const uint32_t lbo[HALOG_GROUPS] = {128u, uint32_t((HALO_W - 2) * 128), 128u, 128u, 0u};
+      uint32_t dA_lo[HALOG_GROUPS], dA_hi[HALOG_GROUPS];
+#pragma unroll
+      for (int q = 0; q < HALOG_GROUPS; ++q) {
+        const uint64_t d = make_smem_desc(smem_u32(smem) + first_row[q] * 128u, lbo[q], HALO_W * 128);
+        dA_lo[q] = uint32_t(d);
+        dA_hi[q] = uint32_t(d >> 32);
+      }
+      const uint64_t dB = make_smem_desc(smem_u32(smem) + HALOG_D_OFF, 8192, 1024);
+      const uint32_t dB_lo0 = uint32_t(dB), dB_hi = uint32_t(dB >> 32);
+      bool ok = true;
+      uint32_t st = 0, sph = 0, acc = 0;
+      for (int t = t_begin; t < t_end; ++t) {
+        ok = mbar_wait(&full[st], sph);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t soff = st * uint32_t(HALOG_STAGE_BYTES >> 4);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {            // 16 pixels per MMA: two image rows of the tile
+#pragma unroll
+          for (int q = 0; q < HALOG_GROUPS; ++q)
+            umma_f16_lohi(tmem_base + uint32_t(q * 64), dA_lo[q] + soff + uint32_t(k) * uint32_t((2 * HALO_W * 128) >> 4), dA_hi[q],
+                          dB_lo0 + soff + uint32_t(k) * (2048u >> 4), dB_hi, idesc, acc);
+          acc = 1;
+        }
+        umma_commit(&empty[st]);
+        if (++st == uint32_t(HALOG_STAGES)) { st = 0; sph ^= 1u; }
+      }
+      if (!ok) atomicExch(status, 22);
+      umma_commit(accf);
+    }
+  } else {
+    const int q = warp & 3;
+    bool ok = mbar_wait(accf, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok && lane == 0) atomicExch(status, 23);
+    tc_fence_after();
+    float* dst = partial + size_t(blockIdx.x) * HALOG_PART_FLOATS;
+    const bool any = t_end > t_begin;          // a CTA without tiles contributes zeros
+    for (int grp = 0; grp < HALOG_GROUPS; ++grp) {
+#pragma unroll 1
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        if (ok && any) {
+          tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(grp * 64 + c * 32), r);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = 0u;
+        }
+        float4* o = reinterpret_cast<float4*>(dst + (size_t(grp) * GEMM_BM + q * 32 + lane) * 64 + c * 32);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          o[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Adds the CTAs' partial sums in CTA order and applies Eq. 6 (or only stores G when W is null).
+// One thread per element of the transposed accumulators, n (= output channel) fastest, so the
+// partial sums are read coalesced; the 64 x 9 x 64 weight elements themselves are scattered.
+struct HaloGUpdate {
+  const float* partial;
+  int n_ctas;
+  int n_out, n_in, ld_w;          // weight matrix [n_out][9 * tap_pitch], pitch ld_w
+  int tap_pitch;
+  float* G;                       // may be null
+  float* W;                       // null: store G only
+  float* mW;                      // may be null
+  __nv_bfloat16* ring;
+  float lr, mu;
+};
+template <int kInstance = 0>
+__global__ void __launch_bounds__(256) conv_halo_g_update_kernel(const HaloGUpdate a) {
+  const int e = blockIdx.x * 256 + threadIdx.x;
+  if (e >= HALOG_PART_FLOATS) return;
+  const int co = e & 63, m = (e >> 6) & 127, grp = e >> 13;
+  const int half = m >> 6, ci = m & 63;
+  const int tap = (grp < 4) ? 2 * grp + half : (half == 0 ? 8 : -1);
+  if (tap < 0 || ci >= a.n_in || co >= a.n_out) return;
+  float g = 0.f;
+  const float* src = a.partial + e;
+#pragma unroll 8
+  for (int c = 0; c < a.n_ctas; ++c) g += __ldcg(src + size_t(c) * HALOG_PART_FLOATS);
+  const size_t off = size_t(co) * a.ld_w + size_t(tap) * a.tap_pitch + ci;
+  if (a.G != nullptr) a.G[off] = g;
+  if (a.W == nullptr) return;
+  float mm = g;
+  if (a.mW != nullptr) {
+    mm = a.mu * a.mW[off] + g;
+    a.mW[off] = mm;
+  }
+  const float w = a.W[off] - a.lr * mm;
+  a.W[off] = w;
+  a.ring[off] = __float2bfloat16_rn(w);
+}
+
 }  // namespace lp

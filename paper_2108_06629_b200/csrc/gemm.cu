@@ -320,8 +320,26 @@ cudaError_t conv_halo_launch(int which, const CUtensorMap& tmA, const CUtensorMa
   return cudaErrorInvalidValue;
 }
 
+// G of a halo-tile layer: accumulate over 8 x 16 pixel tiles, then add the CTAs' partial sums and
+// apply the update (upd.W null: store G only).
+cudaError_t conv_halo_g_launch(const CUtensorMap& tmX, const CUtensorMap& tmD, const ConvGeom& g, int batch, float* partial,
+                               HaloGUpdate upd, int* status, cudaStream_t st) {
+  const int tiles = g.tiles_w * g.tiles_h * batch;
+  const int grid = std::min(tiles, sm_count());
+  conv_halo_g_kernel<0><<<grid, GEMM_THREADS, HALOG_SMEM_BYTES, st>>>(tmX, tmD, g, tiles, partial, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  upd.partial = partial;
+  upd.n_ctas = grid;
+  conv_halo_g_update_kernel<0><<<(HALOG_PART_FLOATS + 255) / 256, 256, 0, st>>>(upd);
+  return cudaGetLastError();
+}
+int conv_halo_g_max_ctas() { return sm_count(); }
+
 cudaError_t gemm_configure() {
   cudaError_t e;
+  if ((e = cudaFuncSetAttribute(conv_halo_g_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, HALOG_SMEM_BYTES)) != cudaSuccess)
+    return e;
 #define LP_CFGH(B, M)                                                                                          \
   if ((e = cudaFuncSetAttribute(conv_halo_kernel<B, M>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
                                 HALO_SMEM_BYTES)) != cudaSuccess)                                              \

@@ -26,6 +26,9 @@
 
 namespace lp {
 
+cudaError_t conv_halo_g_launch(const CUtensorMap& tmX, const CUtensorMap& tmD, const ConvGeom& g, int batch, float* partial,
+                               HaloGUpdate upd, int* status, cudaStream_t st);
+
 constexpr int kDeltaSlots = 4;
 constexpr int kLossRing = 256;
 constexpr int kLogRing = 4096;
@@ -89,7 +92,8 @@ struct Layer {
   std::vector<CUtensorMap> tm_f_A, tm_f_B, tm_d_A, tm_d_B, tm_g_A, tm_g_B;
   // 3x3 layers with at most 64 channels on both sides and images tiled by 8 x 16 pixels: the
   // activation / delta box is fetched once per tile with its halo (see conv_halo.cuh)
-  bool halo_f = false, halo_d = false;
+  bool halo_f = false, halo_d = false, halo_g = false;
+  std::vector<CUtensorMap> tm_hg_D;             // delta as 8 x 16 pixel boxes (the halo-tile G kernel)
   bool lean_f = false;                          // patch-matrix layer with at most 64 output channels: forward through the same kernel
   std::vector<CUtensorMap> tm_hf_A, tm_hd_A;    // halo boxes over the stash slots / the delta slots
   std::vector<CUtensorMap> tm_hf_O;             // forward output (next layer's stash slots, or the pre-pool buffer) as 8 x 16 pixel boxes
@@ -292,7 +296,9 @@ static size_t carve(lp_ctx* c, char* base) {
       y.part_d = reinterpret_cast<float*>(take(t * y.split_d * GEMM_BM * y.bn_d * 4));
       y.cnt_d = reinterpret_cast<unsigned*>(take(t * 4));
     }
-    if (y.split_g > 1) {
+    if (y.halo_g) {
+      y.part_g = reinterpret_cast<float*>(take(size_t(conv_halo_g_max_ctas()) * HALOG_PART_FLOATS * 4));
+    } else if (y.split_g > 1) {
       const size_t t = size_t((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
       y.part_g = reinterpret_cast<float*>(take(t * y.split_g * GEMM_BM * y.bn_g * 4));
       y.cnt_g = reinterpret_cast<unsigned*>(take(t * 4));
@@ -349,6 +355,7 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
       y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
+      y.halo_g = y.halo_f;
       y.lean_f = y.patch && y.n_out <= 64 && y.ld_in <= 64 && l + 1 < n;
       // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: the pixel
       // range is split.  A split costs the last CTA of the tile one more partial tile to add
@@ -463,6 +470,12 @@ static int build_tensor_maps(lp_ctx* c) {
           if ((rc = make_tmap_bf16_nhwc(&y.tm_hf_O[s], dst, y.ld_out, y.imW, y.imH, B, y.ld_out, 8, 16, 1, &err)) != LP_OK)
             return fail(c, rc, err);
         }
+      }
+      if (y.halo_g) {
+        y.tm_hg_D.resize(kDeltaSlots);
+        for (int s = 0; s < kDeltaSlots; ++s)
+          if ((rc = make_tmap_bf16_nhwc(&y.tm_hg_D[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out, 8, 16, 1,
+                                        &err)) != LP_OK) return fail(c, rc, err);
       }
       if (y.halo_d) {
         y.tm_hd_A.resize(kDeltaSlots);
@@ -706,6 +719,22 @@ static inline bool fused_bias(const lp_ctx* c, const Layer& y) {
 
 static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
+  if (y.halo_g) {
+    // 3x3 layer with at most 64 channels: G over 8 x 16 pixel tiles, then the CTAs' partial sums
+    // are added in order and Eq. 6 applied (two launches)
+    HaloGUpdate u{};
+    u.n_out = y.n_out; u.n_in = y.n_in; u.ld_w = y.w_ld; u.tap_pitch = y.ld_in;
+    u.G = y.dW;                                   // kept only with LP_CAPTURE_GRADS / LP_UNFUSED_UPDATE
+    if (fused_update(c)) {
+      u.W = y.W; u.mW = y.mW;
+      u.ring = y.ring + size_t((n + 1) % y.slots) * y.w_elems;
+      u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
+    }
+    c->launches += 2;
+    TimedScope ts(c, LP_TASK_G, st);
+    return conv_halo_g_launch(y.tm_hf_A[n % y.x_slots], y.tm_hg_D[n % kDeltaSlots], halo_geom(y, 0), c->cfg.batch, y.part_g,
+                              u, c->status, st);
+  }
   GemmArgs a{};
   a.M = y.n_out; a.N = y.w_ld; a.K = y.in_rows;
   if (!y.conv || y.patch) a.N = y.n_in;
