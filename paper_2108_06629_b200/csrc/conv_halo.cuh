@@ -303,7 +303,8 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // taps: one pixel = 128 bytes, or 1024 bytes from tap (r, 2) to tap (r + 1, 0)) and B = the delta
 // box.  Nine taps = four pairs and a single: five accumulators of 64 columns stay in tensor
 // memory over ALL tiles of the CTA; at the end each CTA writes its 5 x 128 x 64 partial sums and
-// a second small kernel adds the CTAs' partials in CTA order and applies Eq. 6.
+// a second small kernel adds the CTAs' partials in CTA order and applies Eq. 6.  A layer with
+// 128 output channels takes two such passes (64 channels each).
 constexpr int HALOG_STAGES = 4;
 constexpr int HALOG_D_OFF = 24576;                              // delta box behind the halo box (1 KiB aligned)
 constexpr int HALOG_STAGE_BYTES = HALOG_D_OFF + GEMM_A_BYTES;   // 40 KiB
@@ -314,7 +315,7 @@ constexpr int HALOG_PART_FLOATS = HALOG_GROUPS * GEMM_BM * 64;  // partial sums 
 template <int kInstance = 0>   // (a template only so that the header may be included by several translation units)
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD, const ConvGeom g,
-                   const int tiles_total, float* __restrict__ partial, int* __restrict__ status) {
+                   const int tiles_total, const int co0, float* __restrict__ partial, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HALOG_STAGES * HALOG_STAGE_BYTES);
@@ -358,7 +359,7 @@ conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         uint8_t* base = smem + st * HALOG_STAGE_BYTES;
         mbar_arrive_expect_tx(&full[st], HALO_BYTES + GEMM_A_BYTES);
         tma_load_4d(base, &tmX, &full[st], 0, tw * 8 - 1, th * 16 - 1, n);
-        tma_load_4d(base + HALOG_D_OFF, &tmD, &full[st], 0, tw * 8, th * 16, n);
+        tma_load_4d(base + HALOG_D_OFF, &tmD, &full[st], co0, tw * 8, th * 16, n);   // 64 output channels from co0
         ++issued;
         if (++st == uint32_t(HALOG_STAGES)) { st = 0; sph ^= 1u; }
         if (++tw == g.tiles_w) { tw = 0; if (++th == g.tiles_h) { th = 0; ++n; } }
@@ -445,6 +446,7 @@ conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 struct HaloGUpdate {
   const float* partial;
   int n_ctas;
+  int co0;                        // first output channel of this pass (layers with more than 64 take several)
   int n_out, n_in, ld_w;          // weight matrix [n_out][9 * tap_pitch], pitch ld_w
   int tap_pitch;
   float* G;                       // may be null
@@ -457,7 +459,7 @@ template <int kInstance = 0>
 __global__ void __launch_bounds__(256) conv_halo_g_update_kernel(const HaloGUpdate a) {
   const int e = blockIdx.x * 256 + threadIdx.x;
   if (e >= HALOG_PART_FLOATS) return;
-  const int co = e & 63, m = (e >> 6) & 127, grp = e >> 13;
+  const int co = a.co0 + (e & 63), m = (e >> 6) & 127, grp = e >> 13;
   const int half = m >> 6, ci = m & 63;
   const int tap = (grp < 4) ? 2 * grp + half : (half == 0 ? 8 : -1);
   if (tap < 0 || ci >= a.n_in || co >= a.n_out) return;

@@ -326,13 +326,18 @@ cudaError_t conv_halo_g_launch(const CUtensorMap& tmX, const CUtensorMap& tmD, c
                                HaloGUpdate upd, int* status, cudaStream_t st) {
   const int tiles = g.tiles_w * g.tiles_h * batch;
   const int grid = std::min(tiles, sm_count());
-  conv_halo_g_kernel<0><<<grid, GEMM_THREADS, HALOG_SMEM_BYTES, st>>>(tmX, tmD, g, tiles, partial, status);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
   upd.partial = partial;
   upd.n_ctas = grid;
-  conv_halo_g_update_kernel<0><<<(HALOG_PART_FLOATS + 255) / 256, 256, 0, st>>>(upd);
-  return cudaGetLastError();
+  for (int co0 = 0; co0 < upd.n_out; co0 += 64) {      // one pass per 64 output channels; the stream orders the reuse of `partial`
+    conv_halo_g_kernel<0><<<grid, GEMM_THREADS, HALOG_SMEM_BYTES, st>>>(tmX, tmD, g, tiles, co0, partial, status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    upd.co0 = co0;
+    conv_halo_g_update_kernel<0><<<(HALOG_PART_FLOATS + 255) / 256, 256, 0, st>>>(upd);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 int conv_halo_g_max_ctas() { return sm_count(); }
 

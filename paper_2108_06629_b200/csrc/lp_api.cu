@@ -355,7 +355,7 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
       y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
-      y.halo_g = y.halo_f;
+      y.halo_g = y.halo_f;   // (128 output channels in two passes of the G kernel measured slower than the split-K kernel: 182 / 160 us)
       y.lean_f = y.patch && y.n_out <= 64 && y.ld_in <= 64 && l + 1 < n;
       // G contracts over all B*H*W pixels but has only (Cout/128) x 9 x (Cin/BN) tiles: the pixel
       // range is split.  A split costs the last CTA of the tile one more partial tile to add
@@ -454,7 +454,7 @@ static int build_tensor_maps(lp_ctx* c) {
         if ((rc = make_tmap_bf16_nhwc(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
                                       y.box64.bw, y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
       }
-      if (y.halo_f) {
+      if (y.halo_f || y.halo_g) {      // the halo box over the stashed input (forward and G)
         y.tm_hf_A.resize(y.x_slots);
         for (int s = 0; s < y.x_slots; ++s)
           if ((rc = make_tmap_bf16_nhwc(&y.tm_hf_A[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, HALO_W, HALO_H, 1,
@@ -730,7 +730,7 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
       u.ring = y.ring + size_t((n + 1) % y.slots) * y.w_elems;
       u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
     }
-    c->launches += 2;
+    c->launches += 2 * ((y.n_out + 63) / 64);
     TimedScope ts(c, LP_TASK_G, st);
     return conv_halo_g_launch(y.tm_hf_A[n % y.x_slots], y.tm_hg_D[n % kDeltaSlots], halo_geom(y, 0), c->cfg.batch, y.part_g,
                               u, c->status, st);
