@@ -147,6 +147,8 @@ def test_tasks_unfused_update_path():
     layers = I.mlp([200, 328, 130, 75], "gelu")
     run_teacher_forced(layers, 72, 3, [2, 1, 0], 0.05, 0.9, 5, fused=False)
     run_teacher_forced(I.mlp([96, 160, 24], "relu"), 40, 2, [1, 0], 0.05, 0.0, 4, fused=False)
+    # convolution layers (patch-matrix first layer, halo-tile G, split-K G) with the separate update kernel
+    run_teacher_forced(I.vgg(16, [16, 32, "P", 72], [10]), 8, 2, None, 0.05, 0.9, 3, fused=False)
 
 
 def test_tasks_split_k_forward_and_delta():
