@@ -181,6 +181,14 @@ def test_fused_and_unfused_update_agree():
         for n in a["grads"]:
             assert np.array_equal(a["grads"][n][l][0], b["grads"][n][l][0])
     assert a["loss"] == b["loss"]
+    # the same for convolution layers: patch-matrix first layer, halo-tile G with its reduce-and-update
+    # kernel, split-K G with the update in the last CTA's epilogue -- against G stored + the update kernel
+    layers = I.vgg(16, [16, 32, "P", 72], [10])
+    a, _, _ = free_run(layers, 8, 2, None, 0.02, 0.9, 6, lpb.LP_SCHED_LAYERPIPE)
+    b, _, _ = free_run(layers, 8, 2, None, 0.02, 0.9, 6, lpb.LP_SCHED_LAYERPIPE, extra_flags=lpb.LP_UNFUSED_UPDATE)
+    for l in range(len(layers)):
+        assert np.array_equal(a["W"][l][0], b["W"][l][0]) and np.array_equal(a["W"][l][1], b["W"][l][1])
+    assert a["loss"] == b["loss"]
 
 
 def test_serial_tasks_agree_and_timeline_is_consistent():
