@@ -89,6 +89,9 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(lpb.LayerPipeError) as e:
         lpb.lp_workspace_size(wl["layers"], 4, None, [3, 2, 1, -1], wl["batch"])
     assert e.value.code == lpb.LP_ERR_INVALID_ARG
+    with pytest.raises(lpb.LayerPipeError) as e:      # an empty minibatch is refused, not run
+        lpb.lp_workspace_size(wl["layers"], 4, None, None, 0)
+    assert e.value.code == lpb.LP_ERR_INVALID_ARG
     # pixel rows are indexed with 32 bits: batch x image size beyond that is refused, not wrapped
     big = I.vgg(2048, [64, "P"], [10])
     with pytest.raises(lpb.LayerPipeError) as e:
