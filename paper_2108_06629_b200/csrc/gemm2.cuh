@@ -10,7 +10,7 @@
 //
 // Hand-offs: TMA loads of both CTAs complete on the leader's "full" barrier (the leader arms it
 // with the byte count of both); tcgen05.commit multicasts the "empty" and "accumulator ready"
-// arrivals to the same barrier in both CTAs.  No TMA load uses cluster multicast.
+// arrivals to the same barrier in both CTAs.  Every TMA load has a single destination CTA.
 // Plain matrices, and the forward / delta contractions of 3x3 convolutions (GEOM_PIX_M: each
 // CTA's 128 rows are a box of 128 pixels fetched through the 4-D NHWC map, shifted by the
 // filter tap; one k-block = one tap x 64 channels); no split-K; epilogues as in gemm.cuh.
