@@ -203,8 +203,11 @@ int lp_get_version_log(lp_handle h, long long step, int* v_fwd, int* v_bwd, int*
  * until that step's loss kernel has finished. */
 int lp_get_loss(lp_handle h, long long step, float* loss);
 
-/* 0, or the first non-zero status word written by a kernel whose bounded wait expired
- * (then returns LP_ERR_TIMEOUT and fills *detail). Blocks until the device is idle. */
+/* 0, or the status word written by a kernel: a bounded wait that expired (values 1..23: returns
+ * LP_ERR_TIMEOUT), or a label outside [0, classes) met by the loss kernel (value 64: returns
+ * LP_ERR_INVALID_ARG; that row contributes no one-hot term and the minibatch's loss is NaN --
+ * the label is never used as an address).  *detail receives the word.  Blocks until the device
+ * is idle. */
 int lp_device_status(lp_handle h, int* detail);
 
 /* Needs LP_TIME_TASKS.  For task kind LP_TASK_* (plus LP_TASK_CAST = 5): number of kernel
@@ -245,6 +248,23 @@ int lp_destroy(lp_handle h);
 int lp_gemm_bf16(int which, int M, int N, int K, const void* A_dev, int lda,
                  const void* B_dev, int ldb, float* C_dev, int ldc, void* stream);
 
+/* Status word of the lp_gemm_bf16 launches on the current device since the last call: waits for
+ * the device, returns LP_OK (word 0) or LP_ERR_TIMEOUT (a bounded wait inside a kernel ran out;
+ * *detail, may be NULL, receives the word: 1 producer, 2 MMA issuer, 3 / 4 epilogue, 11..13 the
+ * same roles of the SM-pair kernel), and clears the word. */
+int lp_gemm_status(int* detail);
+
+/* Verification of the bounded waits (Eq. 1 contraction as lp_gemm_bf16 with which = 0, K > 64).
+ * Every wait on a barrier inside the kernels gives up after a cycle limit, records a status
+ * word and lets the kernel drain and return, so that a broken hand-off can never hang the GPU.
+ * This call makes one such wait run out ON PURPOSE, in the only harmless way: the TMA producer
+ * is told to skip the last k-block of every tile, so the MMA issuer waits for a fill that never
+ * comes, for `limit_cycles` SM cycles (1e3 .. 2e9) instead of the default of about two seconds.
+ * Nothing faults and nothing spins unbounded; C receives partial sums.  Afterwards
+ * lp_gemm_status must report LP_ERR_TIMEOUT and the next ordinary launch must be correct. */
+int lp_debug_gemm_starved(int M, int N, int K, const void* A_dev, int lda, const void* B_dev, int ldb,
+                          float* C_dev, int ldc, long long limit_cycles, void* stream);
+
 /*
  * Softmax cross-entropy without a handle, a workspace or any allocation.  (The paper has
  * no counterpart: it is the loss kernel of lp_step offered to callers that cannot give the
@@ -262,7 +282,8 @@ int lp_gemm_bf16(int which, int M, int N, int K, const void* A_dev, int lda,
  *   delta_dev[r][c] = bf16( (softmax(logits_dev[r])[c] - [c == labels_dev[r]]) / batch )
  *   *loss_dev       = mean over rows of -log softmax(logits_dev[r])[labels_dev[r]]
  * logits_dev: device fp32 [batch][ld_logits]; labels_dev: device int32 [batch], values in
- * [0, classes); delta_dev: device bf16 [batch][ld_delta], ld_delta >= classes rounded up to
+ * [0, classes) -- a label outside that range is never used as an address: its row gets no
+ * one-hot term and *loss_dev becomes NaN; delta_dev: device bf16 [batch][ld_delta], ld_delta >= classes rounded up to
  * a multiple of 8 (the lanes up to that multiple are written as zeros); loss_dev: device
  * fp32 [1].  All caller-owned.  `stream` is a cudaStream_t (may be 0); the call is
  * asynchronous.
@@ -271,7 +292,7 @@ int lp_gemm_bf16(int which, int M, int N, int K, const void* A_dev, int lda,
  * LP_XENT_STATIC_MAX_BATCH rows, about 64 KiB, resident on every GPU that loads the
  * library for as long as the process lives.  Consequences the caller must know:
  *   - batch > LP_XENT_STATIC_MAX_BATCH (or batch < 1, classes < 1, bad pitches, null
- *     pointers) -> LP_ERR_INVALID_ARG, nothing is launched.
+ *     pointers) -> LP_ERR_INVALID_ARG, nothing is launched; lp_last_error(NULL) says which.
  *   - all calls on one GPU share that array.  The call clears the part that must start
  *     at zero, so leftovers of an earlier call are harmless, but two calls that overlap
  *     on the device (different streams, no ordering between them) race on it and give

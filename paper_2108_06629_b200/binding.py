@@ -80,6 +80,8 @@ def lib():
         "lp_destroy": [vp],
         "lp_gemm_bf16": [C.c_int, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, vp],
         "lp_softmax_xent_static": [vp, C.c_int, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp],
+        "lp_gemm_status": [ip],
+        "lp_debug_gemm_starved": [C.c_int, C.c_int, C.c_int, vp, C.c_int, vp, C.c_int, vp, C.c_int, C.c_longlong, vp],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -96,7 +98,7 @@ def lib():
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
            "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
            "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
-           "lp_gemm_bf16", "lp_softmax_xent_static"]
+           "lp_gemm_bf16", "lp_gemm_status", "lp_debug_gemm_starved", "lp_softmax_xent_static"]
 
 
 def _check(rc, h=None):
@@ -329,6 +331,21 @@ def lp_gemm_bf16(which, M, N, K, A, lda, B, ldb, Cout, ldc, stream=None):
     s = torch.cuda.current_stream().cuda_stream if stream is None else stream
     _check(lib().lp_gemm_bf16(which, M, N, K, C.c_void_p(A.data_ptr()), lda, C.c_void_p(B.data_ptr()), ldb,
                               C.c_void_p(Cout.data_ptr()), ldc, C.c_void_p(s)))
+
+
+def lp_gemm_status():
+    """(return code, status word) of the lp_gemm_bf16 launches since the last call; clears the word."""
+    d = C.c_int()
+    rc = lib().lp_gemm_status(C.byref(d))
+    return rc, d.value
+
+
+def lp_debug_gemm_starved(M, N, K, A, lda, B, ldb, Cout, ldc, limit_cycles, stream=None):
+    """Forward contraction whose producer skips the last k-block: a bounded wait must run out."""
+    import torch
+    s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    _check(lib().lp_debug_gemm_starved(M, N, K, C.c_void_p(A.data_ptr()), lda, C.c_void_p(B.data_ptr()), ldb,
+                                       C.c_void_p(Cout.data_ptr()), ldc, limit_cycles, C.c_void_p(s)))
 
 
 LP_XENT_STATIC_MAX_BATCH = 16384

@@ -13,6 +13,10 @@
 
 namespace lp {
 
+// ---- lp_api.cu --------------------------------------------------------------
+// Error text of calls that have no handle: what lp_last_error(NULL) returns on this thread.
+void set_global_error(const std::string& msg);
+
 // ---- gemm.cu ---------------------------------------------------------------
 // Encode a 2-D bf16 tensor map (128-byte swizzle, zero fill out of bounds).
 // inner/outer are the logical extents in elements, pitch_elems the row pitch.
@@ -74,7 +78,9 @@ cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int
                                  int* labels_copy, int B, int H, int W, int C, int ld, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
-                                cudaStream_t stream);
+                                int* status, cudaStream_t stream);
+// Value of a device status word that does not come from a bounded wait (those are 1..23).
+constexpr int LP_STATUS_BAD_LABEL = 64;   // a label outside [0, classes) reached the loss kernel
 struct UpdateArgs {
   const float* dW;      // [out][ldw] fp32 (pad lanes zero)
   float* W;             // master [out][ldw]

@@ -1,6 +1,8 @@
 // HBM-bound kernels of the training step: input cast + stash, softmax cross-entropy with
 // delta^L, and the fused SGD update (Eq. 6) that also refreshes the bf16 weight-ring slot.
+#include <atomic>
 #include <cstdio>
+#include <mutex>
 
 #include "common.h"
 
@@ -150,7 +152,8 @@ __device__ __forceinline__ float block_reduce(float v, float* sh, bool is_max) {
 
 __global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const int* __restrict__ labels,
                                     __nv_bfloat16* __restrict__ delta, int ldd, float* __restrict__ row_loss,
-                                    unsigned* __restrict__ ticket, float* __restrict__ loss_out, int B, int C) {
+                                    unsigned* __restrict__ ticket, float* __restrict__ loss_out, int B, int C,
+                                    int* __restrict__ status) {
   __shared__ float sh[32];
   __shared__ bool last;
   const int row = blockIdx.x;
@@ -161,7 +164,11 @@ __global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const
   float s = 0.f;
   for (int c = threadIdx.x; c < C; c += blockDim.x) s += expf(z[c] - mx);
   s = block_reduce(s, sh, false);
+  // A label outside [0, C) comes from caller memory: it must not become an address.  Such a row
+  // gets no one-hot term, its loss is NaN (so the minibatch loss is NaN) and the status word, where
+  // there is one, records it.
   const int y = labels[row];
+  const bool y_ok = unsigned(y) < unsigned(C);
   const float invB = 1.0f / float(B);
   const float inv_s = 1.0f / s;
   __nv_bfloat16* d = delta + (long long)row * ldd;
@@ -172,7 +179,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const
     d[c] = __float2bfloat16_rn(v);
   }
   if (threadIdx.x == 0) {
-    row_loss[row] = -((z[y] - mx) - logf(s));
+    row_loss[row] = y_ok ? -((z[y] - mx) - logf(s)) : __int_as_float(0x7fc00000);
+    if (!y_ok && status != nullptr) atomicCAS(status, 0, LP_STATUS_BAD_LABEL);
     __threadfence();
     const unsigned t = atomicAdd(ticket, 1u);
     last = (t == unsigned(B) - 1u);
@@ -198,8 +206,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ zL, int ldz, const
 
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
-                                cudaStream_t stream) {
-  softmax_xent_kernel<<<B, 256, 0, stream>>>(zL, ldz, labels, delta, ldd, row_loss, ticket, loss_out, B, C);
+                                int* status, cudaStream_t stream) {
+  softmax_xent_kernel<<<B, 256, 0, stream>>>(zL, ldz, labels, delta, ldd, row_loss, ticket, loss_out, B, C, status);
   return cudaGetLastError();
 }
 
@@ -407,34 +415,45 @@ static __device__ __align__(256) unsigned char g_xent_scratch[sizeof(XentScratch
 
 namespace {
 constexpr int kMaxDevices = 64;
-XentScratch* g_xent_scratch_addr[kMaxDevices] = {};   // device address of the array, per device
-thread_local char g_xent_err[160];
+// device address of the array, per device; written once per device under the mutex, read with acquire
+std::atomic<XentScratch*> g_xent_scratch_addr[kMaxDevices];
+std::mutex g_xent_setup_mutex;
+int xent_fail(int code, const std::string& why) {
+  lp::set_global_error("lp_softmax_xent_static: " + why);     // readable through lp_last_error(NULL)
+  return code;
+}
 }  // namespace
 
 extern "C" int lp_softmax_xent_static(const float* logits_dev, int ld_logits, const int* labels_dev,
                                       void* delta_dev, int ld_delta, float* loss_dev, int batch, int classes,
                                       void* stream) {
-  if (!logits_dev || !labels_dev || !delta_dev || !loss_dev) return LP_ERR_INVALID_ARG;
-  if (batch < 1 || classes < 1) return LP_ERR_INVALID_ARG;
-  if (batch > LP_XENT_STATIC_MAX_BATCH) return LP_ERR_INVALID_ARG;   // the fixed scratch holds no more rows
-  if (ld_logits < classes || ld_delta < ((classes + 7) & ~7)) return LP_ERR_INVALID_ARG;
+  if (!logits_dev || !labels_dev || !delta_dev || !loss_dev) return xent_fail(LP_ERR_INVALID_ARG, "null pointer");
+  if (batch < 1 || classes < 1) return xent_fail(LP_ERR_INVALID_ARG, "batch and classes must be positive");
+  if (batch > LP_XENT_STATIC_MAX_BATCH)     // the fixed scratch holds no more rows
+    return xent_fail(LP_ERR_INVALID_ARG, "batch exceeds LP_XENT_STATIC_MAX_BATCH (" + std::to_string(LP_XENT_STATIC_MAX_BATCH) + " rows of built-in scratch)");
+  if (ld_logits < classes || ld_delta < ((classes + 7) & ~7))
+    return xent_fail(LP_ERR_INVALID_ARG, "row pitch smaller than the (padded) number of classes");
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LP_ERR_CUDA;
-  if (g_xent_scratch_addr[dev] == nullptr) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return xent_fail(LP_ERR_CUDA, "no current CUDA device");
+  XentScratch* s = g_xent_scratch_addr[dev].load(std::memory_order_acquire);
+  if (s == nullptr) {
     // set-up, once per device, with that device current: ask the runtime where the array lives
-    void* p = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&p, g_xent_scratch);
-    if (e != cudaSuccess || p == nullptr) {
-      snprintf(g_xent_err, sizeof(g_xent_err), "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
-      return LP_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_xent_setup_mutex);
+    s = g_xent_scratch_addr[dev].load(std::memory_order_relaxed);
+    if (s == nullptr) {
+      void* p = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&p, g_xent_scratch);
+      if (e != cudaSuccess || p == nullptr) return xent_fail(LP_ERR_CUDA, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+      s = static_cast<XentScratch*>(p);
+      g_xent_scratch_addr[dev].store(s, std::memory_order_release);
     }
-    g_xent_scratch_addr[dev] = static_cast<XentScratch*>(p);
   }
-  XentScratch* s = g_xent_scratch_addr[dev];
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the counter must start at zero whatever an earlier (possibly failed) call left behind
-  if (cudaMemsetAsync(&s->ticket, 0, sizeof(unsigned), st) != cudaSuccess) return LP_ERR_CUDA;
-  cudaError_t e = lp::launch_softmax_xent(logits_dev, ld_logits, labels_dev, static_cast<__nv_bfloat16*>(delta_dev),
-                                          ld_delta, s->row_loss, &s->ticket, loss_dev, batch, classes, st);
-  return e == cudaSuccess ? LP_OK : LP_ERR_CUDA;
+  cudaError_t e = cudaMemsetAsync(&s->ticket, 0, sizeof(unsigned), st);
+  if (e != cudaSuccess) return xent_fail(LP_ERR_CUDA, std::string("cudaMemsetAsync: ") + cudaGetErrorString(e));
+  e = lp::launch_softmax_xent(logits_dev, ld_logits, labels_dev, static_cast<__nv_bfloat16*>(delta_dev), ld_delta,
+                              s->row_loss, &s->ticket, loss_dev, batch, classes, nullptr, st);
+  if (e != cudaSuccess) return xent_fail(LP_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e));
+  return LP_OK;
 }

@@ -4,6 +4,7 @@
 #include "conv_halo.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <mutex>
 
@@ -179,6 +180,7 @@ template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st,
                               const UpdMaps* um) {
   if (a.splits < 1 || a.partial == nullptr) a.splits = 1;
+  if (a.wait_limit <= 0) a.wait_limit = LP_WAIT_LIMIT_CYCLES;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
   const int tiles_m = (a.M + GEMM_BM - 1) / GEMM_BM;
@@ -196,6 +198,7 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   const long long slots = (long long)sm_count() * per_sm;
   a.persistent = (work >= 4 * slots && a.kb_per_split <= 96) ? 1 : 0;
   if (g_force_persistent >= 0) a.persistent = g_force_persistent;
+  if (a.starve_kb > 0) a.persistent = 0;      // (the starved producer only keeps its ring position for one tile)
   // fused update streamed by TMA: plain geometry, no split-K, tiles at least 128 columns wide
   static const UpdMaps no_maps{};
   a.upd_tma = (MODE == EPI_WGRAD_UPDATE && um != nullptr && a.splits == 1 && BN >= 128 && a.g.kind == GEOM_PLAIN) ? 1 : 0;
@@ -263,6 +266,7 @@ static cudaError_t configure_one() {
 template <bool A_MN, bool B_MN, int MODE>
 static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
   a.splits = 1;
+  if (a.wait_limit <= 0) a.wait_limit = LP_WAIT_LIMIT_CYCLES;
   const int stage_bytes = 32 * 1024;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   int s = g_force_stages > 0 ? g_force_stages : 3;               // 3 x 32 KiB: two CTAs per SM
@@ -389,37 +393,100 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
 // status word for the stand-alone entry point (handles keep theirs in the workspace)
 __device__ int g_gemm_status = 0;
 
-// ---------------------------------------------------------------------------
-extern "C" int lp_gemm_bf16(int which, int M, int N, int K, const void* A, int lda, const void* B, int ldb,
-                            float* C, int ldc, void* stream) {
+namespace {
+// Per device: the address of g_gemm_status there, and whether the kernels' shared-memory attributes
+// have been set on it.  Written once per device under the mutex.
+constexpr int kMaxGemmDevices = 64;
+std::atomic<int*> g_gemm_status_addr[kMaxGemmDevices];
+std::mutex g_gemm_setup_mutex;
+
+int gemm_device_setup(int** status_dev) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxGemmDevices) {
+    lp::set_global_error("lp_gemm_bf16: no current CUDA device");
+    return LP_ERR_CUDA;
+  }
+  int* p = g_gemm_status_addr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
+    std::lock_guard<std::mutex> lock(g_gemm_setup_mutex);
+    p = g_gemm_status_addr[dev].load(std::memory_order_relaxed);
+    if (p == nullptr) {
+      void* q = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&q, g_gemm_status);
+      if (e == cudaSuccess) e = lp::gemm_configure();
+      if (e != cudaSuccess || q == nullptr) {
+        lp::set_global_error(std::string("lp_gemm_bf16 set-up: ") + cudaGetErrorString(e));
+        return LP_ERR_CUDA;
+      }
+      p = static_cast<int*>(q);
+      g_gemm_status_addr[dev].store(p, std::memory_order_release);
+    }
+  }
+  *status_dev = p;
+  return LP_OK;
+}
+
+int gemm_standalone(int which, int M, int N, int K, const void* A, int lda, const void* B, int ldb, float* C, int ldc,
+                    void* stream, long long wait_limit, int starve_kb) {
   using namespace lp;
   if (which < 0 || which > 2 || M < 1 || N < 1 || K < 1 || !A || !B || !C) return LP_ERR_INVALID_ARG;
   if ((lda & 7) || (ldb & 7) || (ldc & 3)) return LP_ERR_INVALID_ARG;
-  static int* status_dev = nullptr;   // address of g_gemm_status on the device first used
-  if (!status_dev) {
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status_dev), g_gemm_status) != cudaSuccess) return LP_ERR_CUDA;
-    if (gemm_configure() != cudaSuccess) return LP_ERR_CUDA;
-  }
+  int* status_dev = nullptr;
+  int rc = gemm_device_setup(&status_dev);
+  if (rc != LP_OK) return rc;
   const int bn = gemm_pick_bn(which, M, N, K);
   uint32_t boxA[2], boxB[2];
   gemm_box_dims(which, bn, boxA, boxB);
   CUtensorMap tmA, tmB;
   std::string err;
-  int rc;
   // A: forward/delta K-major -> rows = M, inner = K; G: stored [K][M] -> inner = M, rows = K
   if (which == 2) rc = make_tmap_bf16_2d(&tmA, A, M, K, lda, boxA[0], boxA[1], &err);
   else            rc = make_tmap_bf16_2d(&tmA, A, K, M, lda, boxA[0], boxA[1], &err);
-  if (rc != LP_OK) return rc;
+  if (rc != LP_OK) { set_global_error(err); return rc; }
   // B: forward stored [N][K]; delta and G stored [K][N]
   if (which == 0) rc = make_tmap_bf16_2d(&tmB, B, K, N, ldb, boxB[0], boxB[1], &err);
   else            rc = make_tmap_bf16_2d(&tmB, B, N, K, ldb, boxB[0], boxB[1], &err);
-  if (rc != LP_OK) return rc;
+  if (rc != LP_OK) { set_global_error(err); return rc; }
   GemmArgs a{};
   a.M = M; a.N = N; a.K = K;
   a.mode = EPI_STORE_F32;
   a.out = C; a.ld_out = ldc;
   a.status = status_dev;
+  a.wait_limit = wait_limit;
+  a.starve_kb = starve_kb;
   cudaError_t e = gemm_launch(which, bn, tmA, tmB, a, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return LP_ERR_CUDA;
+  if (e != cudaSuccess) { set_global_error(std::string("lp_gemm_bf16 launch: ") + cudaGetErrorString(e)); return LP_ERR_CUDA; }
   return LP_OK;
+}
+}  // namespace
+
+// ---------------------------------------------------------------------------
+extern "C" int lp_gemm_bf16(int which, int M, int N, int K, const void* A, int lda, const void* B, int ldb,
+                            float* C, int ldc, void* stream) {
+  return gemm_standalone(which, M, N, K, A, lda, B, ldb, C, ldc, stream, 0, 0);
+}
+
+extern "C" int lp_gemm_status(int* detail) {
+  int* status_dev = nullptr;
+  int rc = gemm_device_setup(&status_dev);
+  if (rc != LP_OK) return rc;
+  int st = 0;
+  const int zero = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(&st, status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(status_dev, &zero, 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+    lp::set_global_error("lp_gemm_status: a CUDA call failed");
+    return LP_ERR_CUDA;
+  }
+  if (detail) *detail = st;
+  if (st != 0) {
+    lp::set_global_error("lp_gemm_bf16: a bounded device-side wait expired (status " + std::to_string(st) + ")");
+    return LP_ERR_TIMEOUT;
+  }
+  return LP_OK;
+}
+
+extern "C" int lp_debug_gemm_starved(int M, int N, int K, const void* A, int lda, const void* B, int ldb, float* C,
+                                     int ldc, long long limit_cycles, void* stream) {
+  if (limit_cycles < 1000 || limit_cycles > 2000000000ll || K <= lp::GEMM_BK) return LP_ERR_INVALID_ARG;
+  return gemm_standalone(0, M, N, K, A, lda, B, ldb, C, ldc, stream, limit_cycles, 1);
 }

@@ -98,6 +98,9 @@ struct GemmArgs {
   int bld, brows;
   float *bb, *bmb, *bdb, *bbring;   // bias master, momentum (may be null), gradient, destination ring slot
   int* status;              // device status word: set non-zero if a bounded wait expires
+  long long wait_limit;     // SM cycles after which a wait on a barrier gives up (0 at the call = the default, about 2 s)
+  int starve_kb;            // verification of the bounded waits only: the TMA producer skips the last starve_kb k-blocks of
+                            // every tile, so the MMA issuer's wait for them must run out (plain GEMM, one tile per CTA)
 };
 
 __device__ __forceinline__ float gelu_fwd(float z) {
@@ -537,7 +540,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             tma_prefetch_l2_2d(&tmB, kk, tm.n0);
           }
         }
-        for (int kb = 0; kb < tc.num_kb; ++kb) {
+        for (int kb = 0; kb < tc.num_kb - p.starve_kb; ++kb) {
           if (ahead > 0 && kb + ahead < tc.num_kb) {
             const int kk = k0 + ahead * GEMM_BK;
             if (B_MN) {
@@ -547,7 +550,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               tma_prefetch_l2_2d(&tmB, kk, tm.n0);
             }
           }
-          ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+          ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u, p.wait_limit);
           if (!ok) break;
           const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
           const uint32_t sb = sa + GEMM_A_BYTES;
@@ -601,7 +604,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (upd_tma && ok) {
             const uint32_t bytes = p.mW != nullptr ? 2u * UPD_CHUNK_BYTES : uint32_t(UPD_CHUNK_BYTES);
             for (int c = 0; c < kChunks; ++c) {
-              ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+              ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u, p.wait_limit);
               if (!ok) break;
               const uint32_t sa = smem0 + s * uint32_t(SM::STAGE_BYTES);
               const uint32_t fb = full0 + 8u * s;
@@ -617,7 +620,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (!ok) {
         atomicExch(p.status, 1);
         // let copies already in flight land before the CTA's shared memory is released
-        for (long long i = (issued > S ? issued - S : 0); i < issued; ++i) mbar_wait(&full_bar[i % S], uint32_t(i / S) & 1u);
+        for (long long i = (issued > S ? issued - S : 0); i < issued; ++i) mbar_wait(&full_bar[i % S], uint32_t(i / S) & 1u, p.wait_limit);
       }
     }
   } else if (warp == 1) {
@@ -642,14 +645,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t buf = PERSIST ? (it & 1u) : 0u;
         if (PERSIST) {
           // the epilogue must have drained this accumulator buffer (tile it - 2)
-          ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u);
+          ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u, p.wait_limit);
           if (!ok) break;
           tc_fence_after();
         }
         const uint32_t tacc = tmem_base + buf * uint32_t(BN);
         uint32_t acc = 0;
         for (int kb = 0; kb < tc.num_kb; ++kb) {
-          ok = mbar_wait_addr(full0 + 8u * s, ph);
+          ok = mbar_wait_addr(full0 + 8u * s, ph, p.wait_limit);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -675,7 +678,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // adjacent phases apart, and a stage may not run two phases ahead of a waiter.
             for (int c = 0; c < kChunks; ++c) {
               if (PERSIST) {
-                ok = mbar_wait_addr(full0 + 8u * s, ph);
+                ok = mbar_wait_addr(full0 + 8u * s, ph, p.wait_limit);
                 if (!ok) break;
               }
               dA_lo += uint32_t(SM::STAGE_BYTES >> 4);
@@ -752,7 +755,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             p.bbring[m] = b;
           }
           if (good) {
-            good = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
+            good = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u, p.wait_limit);
             good = __all_sync(0xffffffffu, good);
             if (!good && lane == 0) atomicExch(p.status, 3);
           }
@@ -764,7 +767,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t sW = smem0 + us * uint32_t(SM::STAGE_BYTES);
             const uint32_t sM = sW + UPD_CHUNK_BYTES;
             if (good) {
-              good = mbar_wait_addr(full0 + 8u * us, uph);
+              good = mbar_wait_addr(full0 + 8u * us, uph, p.wait_limit);
               good = __all_sync(0xffffffffu, good);
               if (!good && lane == 0) atomicExch(p.status, 4);
             }
@@ -877,7 +880,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);   // in flight while the main loop runs
       }
-      ok = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u);
+      ok = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u, p.wait_limit);
       ok = __all_sync(0xffffffffu, ok);      // warp-uniform: tcgen05.ld below is warp-collective
       if (!ok) {
         if (lane == 0) atomicExch(p.status, 3);

@@ -143,6 +143,7 @@ struct lp_ctx {
 namespace lp {
 
 static thread_local std::string g_err;   // for calls without a handle
+void set_global_error(const std::string& msg) { g_err = msg; }
 
 static int fail(lp_ctx* h, int code, const std::string& msg) {
   if (h) {
@@ -1059,7 +1060,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     TimedScope ts(c, LP_TASK_LOSS, st);
     LP_CUDA(c, launch_softmax_xent(c->zL + size_t(ds) * B * c->ld_cls, c->ld_cls, c->labels + size_t(ds) * B,
                                    yl.delta + size_t(ds) * yl.delta_elems, yl.ld_out, c->row_loss + size_t(ds) * B,
-                                   c->ticket + ds, c->loss + (n % kLossRing), B, c->classes, st));
+                                   c->ticket + ds, c->loss + (n % kLossRing), B, c->classes, c->status, st));
     LP_CUDA(c, task_end(c, st, {&c->rZL[ds], &c->rLabels[ds]}, {rd}, &c->loss_ev[n % kLossRing]));
   }
   // ---- backward: delta and G are independent tasks; update follows G -----------
@@ -1349,7 +1350,7 @@ extern "C" int lp_debug_run_task(lp_handle h, int task, int layer, long long ste
       ++h->launches;
       LP_CUDA(h, launch_softmax_xent(h->zL + size_t(ds) * B * h->ld_cls, h->ld_cls, h->labels + size_t(ds) * B,
                                      yl.delta + size_t(ds) * yl.delta_elems, yl.ld_out, h->row_loss + size_t(ds) * B,
-                                     h->ticket + ds, h->loss + (step % kLossRing), B, h->classes, st));
+                                     h->ticket + ds, h->loss + (step % kLossRing), B, h->classes, h->status, st));
       break;
     }
     case LP_TASK_DELTA:
@@ -1404,6 +1405,8 @@ extern "C" int lp_device_status(lp_handle h, int* detail) {
   int st = 0;
   LP_CUDA(h, cudaMemcpy(&st, h->status, 4, cudaMemcpyDeviceToHost));
   if (detail) *detail = st;
+  if (st == LP_STATUS_BAD_LABEL)
+    return fail(h, LP_ERR_INVALID_ARG, "a label outside [0, classes) reached the loss kernel (that minibatch's loss is NaN)");
   if (st != 0) return fail(h, LP_ERR_TIMEOUT, "a bounded device-side wait expired (status " + std::to_string(st) + ")");
   return LP_OK;
 }

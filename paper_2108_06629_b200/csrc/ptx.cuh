@@ -50,11 +50,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 #ifndef LP_WAIT_LIMIT_CYCLES
 #define LP_WAIT_LIMIT_CYCLES 4000000000ll
 #endif
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = LP_WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > LP_WAIT_LIMIT_CYCLES) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
 }
@@ -71,11 +71,11 @@ __device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar, uint32_t parity
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar, uint32_t parity, long long limit = LP_WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait_addr(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait_addr(bar, parity)) {
-    if (clock64() - t0 > LP_WAIT_LIMIT_CYCLES) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
 }

@@ -1,11 +1,24 @@
 """Helpers shared by the GPU parity tests."""
 import numpy as np
 
+_CHUNK = 1 << 24      # elements compared at a time (keeps the float64 temporaries of huge tensors small)
+
+
+def _chunks(a, b):
+    a = np.asarray(a).reshape(-1)
+    b = np.asarray(b).reshape(-1)
+    assert a.size == b.size, (a.size, b.size)
+    for i in range(0, max(a.size, 1), _CHUNK):
+        yield a[i:i + _CHUNK].astype(np.float64), b[i:i + _CHUNK].astype(np.float64)
+
 
 def rel_l2(a, b):
-    a = np.asarray(a, dtype=np.float64).ravel()
-    b = np.asarray(b, dtype=np.float64).ravel()
-    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+    num = den = 0.0
+    for x, y in _chunks(a, b):
+        d = x - y
+        num += float(d @ d)
+        den += float(y @ y)
+    return float(np.sqrt(num) / max(np.sqrt(den), 1e-300))
 
 
 def bf16_ulp(x):
@@ -17,16 +30,20 @@ def bf16_ulp(x):
 def assert_bf16_close(got, want, what, tol_rel=2e-3, min_equal=0.98):
     """Same operands on both sides: the two bf16 results may differ only where the fp32
     value sat next to a rounding boundary, i.e. by at most one bf16 spacing, rarely."""
-    got = np.asarray(got, dtype=np.float64)
-    want = np.asarray(want, dtype=np.float64).reshape(got.shape)
+    got = np.asarray(got)
+    want = np.asarray(want).reshape(got.shape)
     r = rel_l2(got, want)
     assert r <= tol_rel, "%s: relative L2 error %.3e > %.1e" % (what, r, tol_rel)
     # absolute part: fp32 accumulation error of the contraction (a few 1e-6 of a typical
     # element) also moves elements whose own magnitude, hence bf16 spacing, is tiny
-    rms = float(np.sqrt(np.mean(want * want))) if want.size else 0.0
-    slack = bf16_ulp(want) * 1.01 + 3e-5 * rms
-    bad = np.abs(got - want) > slack
-    assert not bad.any(), "%s: %d elements differ by more than one bf16 spacing" % (what, int(bad.sum()))
-    eq = float((got == want).mean()) if want.size else 1.0
+    sq = sum(float(y @ y) for _, y in _chunks(got, want))
+    rms = float(np.sqrt(sq / want.size)) if want.size else 0.0
+    n_bad = n_eq = 0
+    for x, y in _chunks(got, want):
+        slack = bf16_ulp(y) * 1.01 + 3e-5 * rms
+        n_bad += int((np.abs(x - y) > slack).sum())
+        n_eq += int((x == y).sum())
+    assert n_bad == 0, "%s: %d elements differ by more than one bf16 spacing" % (what, n_bad)
+    eq = n_eq / want.size if want.size else 1.0
     assert eq >= min_equal, "%s: only %.4f of the elements are bit-equal" % (what, eq)
     return r

@@ -75,3 +75,49 @@ def test_deep_pipeline_and_two_stage_pipeline_agree():
     lpb.lp_set_tuning(0, 0)
     assert np.array_equal(outs[0], outs[1])
     assert rel_l2(outs[0], _reference(0, M, N, K, A, B)) < 1e-6 + 2e-7 * np.sqrt(K)
+
+
+def test_status_word_is_clear_after_ordinary_launches():
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    A, B = _operands(0, 256, 384, 512, 3)
+    Cd = torch.empty((256, 384), device="cuda")
+    lpb.lp_gemm_bf16(0, 256, 384, 512, A.cuda(), 512, B.cuda(), 512, Cd, 384)
+    rc, word = lpb.lp_gemm_status()
+    assert (rc, word) == (lpb.LP_OK, 0)
+
+
+def test_bounded_wait_runs_out_reports_and_leaves_the_device_usable():
+    """Every barrier wait in the kernels is bounded.  Here one is made to run out in the harmless
+    way the library offers for it: the producer skips the last k-block, the MMA issuer waits for it
+    for 2e6 cycles (about a millisecond) and gives up.  The kernel must return by itself, the
+    status word must say so, and the next ordinary launch must be exact and leave the word clear."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    M, N, K = 256, 384, 512
+    A, B = _operands(0, M, N, K, 11)
+    Ad, Bd = A.cuda(), B.cuda()
+    Cd = torch.zeros((M, N), device="cuda")
+    assert lpb.lp_gemm_status() == (lpb.LP_OK, 0)
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    lpb.lp_debug_gemm_starved(M, N, K, Ad, K, Bd, K, Cd, N, 2_000_000)
+    t1.record()
+    rc, word = lpb.lp_gemm_status()            # waits for the device
+    assert rc == lpb.LP_ERR_TIMEOUT and word in (2, 3), (rc, word)
+    assert b"bounded" in lpb.lib().lp_last_error(None)
+    assert t0.elapsed_time(t1) < 500.0         # gave up after the short limit, not after seconds
+    # what did arrive was contracted: the result is the product over the first K - 64 columns (if the
+    # epilogue's own wait had not run out first, in which case C was left alone)
+    if word == 2:
+        ref = A.double().numpy()[:, :K - 64] @ B.double().numpy()[:, :K - 64].T
+        assert rel_l2(Cd.cpu().numpy(), ref) < 1e-5
+    assert lpb.lp_gemm_status() == (lpb.LP_OK, 0)          # reading the word cleared it
+    lpb.lp_gemm_bf16(0, M, N, K, Ad, K, Bd, K, Cd, N)
+    assert lpb.lp_gemm_status() == (lpb.LP_OK, 0)
+    assert rel_l2(Cd.cpu().numpy(), _reference(0, M, N, K, A, B)) < 1e-6 + 2e-7 * np.sqrt(K)
+    # argument checks of the verification call
+    lib = lpb.lib()
+    assert lib.lp_debug_gemm_starved(M, N, 64, None, K, None, K, None, N, 2_000_000, None) == lpb.LP_ERR_INVALID_ARG
+    assert lib.lp_debug_gemm_starved(M, N, K, Ad.data_ptr(), K, Bd.data_ptr(), K, Cd.data_ptr(), N, 5, None) == lpb.LP_ERR_INVALID_ARG

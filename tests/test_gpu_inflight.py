@@ -1,0 +1,175 @@
+"""Parity with several minibatches in flight (Section III-C, Fig. 6).
+
+Overlapping the forward pass of new minibatches with delta and G of older ones is the
+schedule the method is about, and it is the mode the benchmark times.  Here every
+``lp_step`` is enqueued without any host call in between -- no gradient read, no loss
+read, no synchronisation -- so that the stage scheduler's cross-minibatch edges carry the
+whole burden: write-after-read on the ring slot of version n - d_l, on the d_l + 2
+activation-stash slots, on the four delta slots, on the pre-pool buffer and the argmax
+slots.  Losses, the version log and the weights are read only after ``lp_flush``.
+
+Two launch patterns: "natural" (the host enqueues as fast as it can) and "gated" (a
+bounded spin kernel holds the caller's stream while ALL steps are enqueued, so that even a
+network whose step is shorter than its enqueue time runs with the deepest overlap the
+delays allow).
+
+Asserted:
+  (i)   weights after the flush within 5e-3 per tensor of the oracle's, losses and the
+        weight change within the free-running bounds of test_gpu_training.py, version log
+        bit-exact;
+  (ii)  weights and losses BIT-IDENTICAL to a run of the same handle configuration that
+        waits for the device after every step -- the kernels are deterministic, so any
+        difference is a missed hazard;
+  (iii) LayerPipe and fused-B schedules bit-identical.
+"""
+import functools
+
+import numpy as np
+import pytest
+
+from gpu_common import rel_l2
+
+pytestmark = pytest.mark.gpu
+
+GATE_CYCLES = 300_000_000     # about 0.15 s of spinning on the caller's stream (bounded)
+
+
+def run(layers, batch, stages, delays, lr, mu, steps, schedule, mode, flags=0):
+    """mode: 'sync' (device idle after every step), 'natural', 'gated'."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    W0, b0 = I.initial_weights(layers, 0)
+    tr = lpb.Trainer(layers, batch, stages, delays=delays, lr=lr, momentum=mu, schedule=schedule, flags=flags,
+                     W0=W0, b0=b0)
+    xs, ys = [], []
+    for n in range(steps):
+        x, y = I.minibatch(layers, batch, n)
+        xs.append(torch.from_numpy(x).cuda())
+        ys.append(torch.from_numpy(y).cuda())
+    torch.cuda.synchronize()
+    if mode == "gated":
+        torch.cuda._sleep(GATE_CYCLES)
+    for n in range(steps):
+        tr.step(xs[n], ys[n])
+        if mode == "sync":
+            torch.cuda.synchronize()
+    tr.flush()
+    torch.cuda.synchronize()
+    out = dict(schedule=tr.get_schedule())
+    out["loss"] = [tr.get_loss(n) for n in range(steps)]
+    out["vlog"] = [tr.get_version_log(n) for n in range(steps)]
+    out["W"] = [tr.get_weights(l) for l in range(len(layers))]
+    rc, detail = tr.device_status()
+    assert rc == 0, detail
+    tr.close()
+    return out, W0, b0
+
+
+@functools.lru_cache(maxsize=None)
+def _oracle(key, steps):
+    """One oracle trajectory per configuration (shared by the cases that use it)."""
+    from oracle import layerpipe_oracle as O
+    from paper_2108_06629_b200 import inputs as I
+    layers, batch, delays, lr, mu = CONFIGS[key]()
+    W0, b0 = I.initial_weights(layers, 0)
+    orc = O.DelayedGradientTrainer(layers, list(delays), lr, mu, W0, b0, mirror=True, dtype=np.float32)
+    recs = []
+    for n in range(steps):
+        x, y = I.minibatch(layers, batch, n)
+        r = orc.step(x, y)
+        recs.append(dict(loss=r["loss"], v=r["v"], slot=r["slot"]))
+    Wf, bf = orc.weights()
+    return recs, Wf, bf
+
+
+CONFIGS = {}
+
+
+def same_bits(a, b, what):
+    assert a["loss"] == b["loss"], (what, "loss")
+    for l, (x, y) in enumerate(zip(a["W"], b["W"])):
+        assert np.array_equal(x[0], y[0]) and np.array_equal(x[1], y[1]), (what, "layer", l)
+        assert x[2] == y[2]
+
+
+def check(key, layers, batch, stages, delays, lr, mu, steps, loss_bound=5e-3, dw_bound=5e-2, modes=("natural", "gated")):
+    from paper_2108_06629_b200 import binding as lpb
+    ref, W0, b0 = run(layers, batch, stages, delays, lr, mu, steps, lpb.LP_SCHED_LAYERPIPE, "sync")
+    stage, delay, slots = ref["schedule"]
+    CONFIGS[key] = lambda: (layers, batch, tuple(delay), lr, mu)
+    recs, Wf, bf = _oracle(key, steps)
+    # (i) against the oracle
+    for n in range(steps):
+        vf, vb, sl = ref["vlog"][n]
+        assert vf == recs[n]["v"] and vb == recs[n]["v"] and sl == recs[n]["slot"]
+        assert abs(ref["loss"][n] - recs[n]["loss"]) <= loss_bound * abs(recs[n]["loss"]), (key, "loss", n)
+    worst = 0.0
+    for l in range(len(layers)):
+        W, bb, ver = ref["W"][l]
+        assert ver == steps
+        rw = rel_l2(W, Wf[l])
+        worst = max(worst, rw)
+        assert rw <= 5e-3, (key, "W", l, rw)
+        assert rel_l2(W - W0[l], Wf[l] - W0[l]) <= dw_bound, (key, "W - W0", l)
+    # (ii) in flight == synchronised, (iii) fused-B == LayerPipe, all bit for bit
+    for mode in modes:
+        for sched in (lpb.LP_SCHED_LAYERPIPE, lpb.LP_SCHED_FUSED_B):
+            got, _, _ = run(layers, batch, stages, delays, lr, mu, steps, sched, mode)
+            assert got["vlog"] == ref["vlog"]
+            same_bits(got, ref, (key, mode, "fused_b" if sched else "layerpipe"))
+    print("%s: %d minibatches in flight-capable run, worst weight error %.2e vs oracle, delays %s" % (key, steps, worst, delay))
+
+
+def test_inflight_mlp4_784():
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp4_784"]
+    check("mlp4_784", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], wl["steps"])
+
+
+def test_inflight_mlp8_4096_full_size_every_ring_wraps():
+    """Delays 7..0 -> rings of 8..1 slots and stashes of 9..2 slots; 20 minibatches wrap each of
+    them at least twice, and the delay of 7 exceeds the four delta slots."""
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp8_4096"]
+    check("mlp8_4096", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 20)
+
+
+def test_inflight_vgg_small_32_full_config():
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["vgg_small_32"]
+    check("vgg_small_32", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], wl["steps"],
+          loss_bound=3e-2, dw_bound=0.25)
+
+
+def test_inflight_convnet_with_planned_delays_of_four_and_more():
+    """Six planned stages on a small conv net: pooled layers (pre-pool buffer, argmax slots),
+    halo-tile and split-K G kernels, delays up to 5."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(32, [32, 32, "P", 64, 64, "P", 128, "P"], [96, 10])
+    check("cnn32", layers, 16, 6, None, 0.01, 0.9, 14, loss_bound=3e-2, dw_bound=0.25)
+
+
+def test_inflight_delays_longer_than_the_delta_slots_and_out_of_order():
+    """Explicit delays {9, 2, 6, 0, 5, 0}: longer than the four delta slots, not monotone, with
+    momentum; the paper's 2 x convention {4, 2, 0} on a second net."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 136, 200, 72, 40], "gelu")
+    check("odd_delays", layers, 56, 6, [9, 2, 6, 0, 5, 0], 0.02, 0.9, 24)
+    layers = I.mlp([96, 160, 64, 24], "relu")
+    check("double_delays", layers, 40, 3, [4, 2, 0], 0.05, 0.0, 12, dw_bound=0.1)
+
+
+def test_inflight_unfused_update_and_captured_gradients():
+    """The separate update kernel (its own task between G and the ring slot) and the gradient
+    capture buffer (rewritten every step: a WAW/WAR edge of its own) in flight."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 40], "gelu")
+    args = (layers, 56, 3, [2, 1, 0], 0.02, 0.9, 12)
+    ref, _, _ = run(*args, lpb.LP_SCHED_LAYERPIPE, "sync")
+    for flags in (lpb.LP_UNFUSED_UPDATE, lpb.LP_CAPTURE_GRADS):
+        for mode in ("natural", "gated"):
+            for sched in (lpb.LP_SCHED_LAYERPIPE, lpb.LP_SCHED_FUSED_B):
+                got, _, _ = run(*args, sched, mode, flags=flags)
+                same_bits(got, ref, ("flags", flags, mode, sched))

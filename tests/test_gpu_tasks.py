@@ -242,3 +242,63 @@ def test_tasks_mlp8_4096_full_size():
     w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 10,
                            check_steps={0, 4, 9})
     print("worst per-task errors", w)
+
+
+def test_tasks_mlp16_8192_full_size_one_minibatch():
+    """The tensor-bound workload at full size (2048 x 8192 x 8192, sixteen layers): every task of
+    one minibatch on the oracle's operands -- 256 x 256 SM-pair tiles with 64 tiles per dimension
+    for all three contractions, the update of 67 M weights per layer in the G kernel."""
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp16_8192"]
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 1)
+    print("mlp16_8192 worst per-task errors", w)
+
+
+def test_tasks_vgg16_224_full_size_one_minibatch():
+    """VGG-16 shapes at 224 x 224, batch 64, planned stages: pixel boxes with seven tiles per row
+    (224 / 112 / 56 / 28 pixels), the 2 x 2 x 32 box at 14 x 14, split-K G over 3.2 M pixel rows,
+    SM-pair convolution tiles, the patch-matrix first layer, the halo-tile 64 -> 64 layer, the
+    automatic split-K and the persistent streamed update of the 25088 -> 4096 layer."""
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["vgg16_224"]
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 1)
+    print("vgg16_224 worst per-task errors", w)
+
+
+def test_tasks_pixel_boxes_with_seven_tiles_per_row():
+    """56 / 28 / 14 pixel images: boxes of 8 x 8 x 2, 4 x 4 x 8 and 2 x 2 x 32 pixels, seven boxes
+    per image row, none of them served by the halo-tile kernels (56 is not a multiple of 16)."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(56, [16, 16, "P", 32, 32, "P", 64], [10])
+    run_teacher_forced(layers, 32, 4, None, 0.05, 0.9, 3)
+
+
+def test_tasks_sm_pair_convolution_tiles_at_28_and_14_pixels():
+    """256 -> 256 channels at 28 x 28 and (behind a pool) at 14 x 14, batch 64: an even number of
+    128-pixel boxes, so forward and delta run as 256-pixel x 256-column tiles on SM pairs."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(28, [256, 256, "P", 256], [10])
+    run_teacher_forced(layers, 64, 3, None, 0.02, 0.0, 2)
+
+
+def test_tasks_single_image_224_patch_layer_and_automatic_split_k():
+    """One 224 x 224 RGB image: the patch-matrix first layer (forward through the halo pipeline, G as
+    one tile split 148 ways over 50 k pixel rows) and a fully connected layer with 3136 k-blocks and
+    a single tile, which takes the automatic four-way split-K."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.vgg(224, [16, "P"], [10])
+    run_teacher_forced(layers, 1, 2, None, 0.05, 0.9, 3)
+    run_teacher_forced(layers, 2, 2, None, 0.05, 0.0, 2)
+
+
+def test_tasks_persistent_update_walk_of_three_tiles_per_cta():
+    """G of a 4500 -> 3000 layer: 24 x 36 = 864 tiles on 296 CTA slots, forced persistent, so every
+    CTA streams the update of about three tiles back to back through its stage ring."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([4500, 3000, 75], "gelu")
+    lpb.lp_set_tuning(0, 0, 512)
+    try:
+        run_teacher_forced(layers, 72, 2, [1, 0], 0.05, 0.9, 2)
+    finally:
+        lpb.lp_set_tuning(0, 0, 0)

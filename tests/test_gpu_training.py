@@ -316,3 +316,34 @@ def test_step_rejects_bad_arguments_without_side_effects():
     tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
     assert tr.get_version_log(0)[0] == [0, 0]
     tr.close()
+
+
+def test_label_out_of_range_is_reported_not_dereferenced():
+    """A label outside [0, classes) must never become an address: the loss of that minibatch is NaN,
+    the status word reports it as an argument error, nothing faults, and a new handle works."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([64, 32, 16], "relu")
+    W0, b0 = I.initial_weights(layers, 0)
+    tr = lpb.Trainer(layers, 8, 2, W0=W0, b0=b0)
+    x, y = I.minibatch(layers, 8, 0)
+    tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    assert np.isfinite(tr.get_loss(0))
+    assert tr.device_status() == (lpb.LP_OK, 0)
+    for bad in (16, -1, 2 ** 31 - 1, -2 ** 31):
+        yb = y.copy()
+        yb[3] = bad
+        tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(yb).cuda())
+    tr.flush()
+    torch.cuda.synchronize()
+    assert all(np.isnan(tr.get_loss(n)) for n in range(1, 5))
+    rc, word = tr.device_status()
+    assert rc == lpb.LP_ERR_INVALID_ARG and word == 64
+    assert b"label" in lpb.lib().lp_last_error(tr.h)
+    tr.close()
+    tr = lpb.Trainer(layers, 8, 2, W0=W0, b0=b0)
+    tr.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    tr.flush()
+    assert np.isfinite(tr.get_loss(0)) and tr.device_status() == (lpb.LP_OK, 0)
+    tr.close()

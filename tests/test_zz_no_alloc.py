@@ -75,3 +75,29 @@ def test_static_scratch_loss_refuses_what_does_not_fit():
     torch.cuda.synchronize()
     # all-zero logits: uniform softmax, loss = log 8 (16384 row losses added in fp32)
     assert abs(float(loss.item()) - np.log(8.0)) < 1e-3 * np.log(8.0)
+    # the refusals say why
+    assert lpb.lp_softmax_xent_static(lg, lb, delta, loss, 8) == lpb.LP_ERR_INVALID_ARG
+    assert b"LP_XENT_STATIC_MAX_BATCH" in lpb.lib().lp_last_error(None)
+
+
+def test_static_scratch_loss_never_uses_a_bad_label_as_an_address():
+    """This entry point has no status word to report through, so a label outside [0, classes)
+    shows up as a NaN loss; the rows with valid labels are unaffected and nothing faults."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    batch, classes = 16, 8
+    lg = torch.zeros((batch, classes), dtype=torch.float32, device="cuda")
+    delta = torch.zeros((batch, classes), dtype=torch.bfloat16, device="cuda")
+    loss = torch.zeros((1,), dtype=torch.float32, device="cuda")
+    for bad in (8, -1, 2 ** 31 - 1):
+        lb = torch.zeros((batch,), dtype=torch.int32, device="cuda")
+        lb[5] = bad
+        assert lpb.lp_softmax_xent_static(lg, lb, delta, loss, classes) == lpb.LP_OK
+        torch.cuda.synchronize()
+        assert np.isnan(float(loss.item()))
+        d = delta.float().cpu().numpy()
+        assert abs(d[0, 0] - (1.0 / 8 - 1.0) / batch) < 1e-3 and abs(d[5, 0] - (1.0 / 8) / batch) < 1e-3
+    lb = torch.zeros((batch,), dtype=torch.int32, device="cuda")
+    assert lpb.lp_softmax_xent_static(lg, lb, delta, loss, classes) == lpb.LP_OK
+    torch.cuda.synchronize()
+    assert abs(float(loss.item()) - np.log(8.0)) < 1e-5
