@@ -29,12 +29,6 @@ from paper_2108_06629_b200 import replicas  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the
-# ncu capture summarised under profiles/ (None until a capture exists for that pair).
-NCU_TRAFFIC_BYTES = {
-    # capture of the fused G + update kernel: 139.57 MB read + 111.45 MB written inside the kernel window
-    ("mlp8_4096", "G"): 251.02e6,
-}
 
 
 def load_peaks():
@@ -198,9 +192,14 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------- our arm
-def timed_loop(torch, tr, xs, ys, steps, stream):
+MIN_TIMED_SECONDS = 1.5     # the timed region is repeated until this much device time has been measured
+
+
+def timed_block(torch, tr, xs, ys, steps, stream):
+    """EXACTLY `steps` lp_step calls + lp_flush between two events on the caller's stream."""
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
     e0.record(stream)
     P = len(xs)
     for k in range(steps):
@@ -211,7 +210,7 @@ def timed_loop(torch, tr, xs, ys, steps, stream):
     return e0.elapsed_time(e1)
 
 
-def e2e_loop(torch, tr, hx, hy, xd, yd, steps, stream, lag, first_step):
+def e2e_block(torch, tr, hx, hy, xd, yd, steps, stream, lag, first_step):
     """Every step: pinned host -> device copy of that step's minibatch and labels, lp_step,
     and a device -> host read of one finished step's loss (the step `lag` calls back, so
     that the read does not drain the pipeline; the last `lag` losses are read at the end)."""
@@ -219,11 +218,12 @@ def e2e_loop(torch, tr, hx, hy, xd, yd, steps, stream, lag, first_step):
     e1 = torch.cuda.Event(enable_timing=True)
     P = len(hx)
     losses = []
+    torch.cuda.synchronize()
     e0.record(stream)
     for k in range(steps):
-        xd.copy_(hx[k % P], non_blocking=True)
-        yd.copy_(hy[k % P], non_blocking=True)
-        tr.step(xd, yd)
+        xd[k % 2].copy_(hx[k % P], non_blocking=True)
+        yd[k % 2].copy_(hy[k % P], non_blocking=True)
+        tr.step(xd[k % 2], yd[k % 2])
         if k >= lag:
             losses.append(tr.get_loss(first_step + k - lag))
     for k in range(max(steps - lag, 0), steps):
@@ -235,7 +235,176 @@ def e2e_loop(torch, tr, hx, hy, xd, yd, steps, stream, lag, first_step):
     return e0.elapsed_time(e1)
 
 
-def run_ours(args, wl):
+def repeat_blocks(block, min_seconds, max_blocks=400):
+    """Run `block()` (returns milliseconds) at least 3 times and until min_seconds of device time
+    have been measured.  Returns the list of block times."""
+    ts = []
+    while len(ts) < 3 or (sum(ts) < 1e3 * min_seconds and len(ts) < max_blocks):
+        ts.append(block())
+    return ts
+
+
+def summarize(ts, steps):
+    med = statistics.median(ts)
+    return {"ms_per_step": med / steps, "ms_per_step_min": min(ts) / steps, "ms_per_step_max": max(ts) / steps,
+            "blocks": len(ts), "timed_seconds": sum(ts) * 1e-3}
+
+
+class Workload:
+    """Host and device copies of a workload's synthetic inputs, shared by every handle of the run."""
+
+    def __init__(self, torch, name, dev):
+        self.name = name
+        self.wl = I.WORKLOADS[name]
+        self.layers, self.B = self.wl["layers"], self.wl["batch"]
+        self.W0, self.b0 = I.initial_weights(self.layers, 0)
+        self.P = 8
+        self.hx, self.hy = [], []
+        for n in range(self.P):
+            x, y = I.minibatch(self.layers, self.B, n)
+            self.hx.append(torch.from_numpy(x).pin_memory())
+            self.hy.append(torch.from_numpy(y).pin_memory())
+        self.xs = [t.to(dev) for t in self.hx]
+        self.ys = [t.to(dev) for t in self.hy]
+        self.dev = dev
+
+    def trainer(self, lpb, schedule, flags=0):
+        wl = self.wl
+        return lpb.Trainer(self.layers, self.B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                           schedule=schedule, flags=flags, W0=self.W0, b0=self.b0, device=self.dev)
+
+
+def throughput(torch, lpb, w, schedule, steps, warmup, min_seconds, stream, flags=0):
+    """samples/s of one handle: warm-up (fills every ring), then repeated blocks of `steps` steps."""
+    tr = w.trainer(lpb, schedule, flags)
+    stage, delays, slots = tr.get_schedule()
+    prewarm = max(delays) + 3 + max(warmup, 3)
+    for k in range(prewarm):
+        tr.step(w.xs[k % w.P], w.ys[k % w.P])
+    tr.flush()
+    torch.cuda.synchronize()
+    l0 = tr.kernel_launches()
+    ts = repeat_blocks(lambda: timed_block(torch, tr, w.xs, w.ys, steps, stream), min_seconds)
+    launches = (tr.kernel_launches() - l0) // len(ts)
+    rc, detail = tr.device_status()
+    if rc != 0:
+        raise SystemExit("device status %d (%d)" % (rc, detail))
+    return tr, ts, launches, prewarm, (stage, delays, slots)
+
+
+def kernel_times(torch, lpb, w, sched, flags, steps, stream):
+    """Per task kind: launches, total and average event-timed duration over `steps` minibatches."""
+    trp = w.trainer(lpb, sched, flags)
+    _, delays, _ = trp.get_schedule()
+    for k in range(max(delays) + 6):
+        trp.step(w.xs[k % w.P], w.ys[k % w.P])
+    trp.flush()
+    torch.cuda.synchronize()
+    trp.reset_task_times()
+    nprof = max(1, min(steps, 32768 // (6 * len(w.layers))))
+    timed_block(torch, trp, w.xs, w.ys, nprof, stream)
+    out = {}
+    for kind in ("forward", "delta", "G", "update", "loss", "cast"):
+        n, tot = trp.task_time(kind)
+        out[kind] = dict(launches=n, total_ms=tot, avg_us=1e3 * tot / max(n, 1))
+    trp.close()
+    del trp
+    torch.cuda.empty_cache()
+    return out
+
+
+KERNEL_NAMES = {"forward": "gemm (forward contraction, Eqs. 1-2)", "delta": "gemm (delta contraction, Eqs. 3-4)",
+                "G": "gemm (G contraction with the update of Eq. 6 in its epilogue)", "update": "sgd_update_kernel"}
+
+
+def ncu_traffic(workload, kind):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the table
+    in profiles/ncu_traffic.md (rows `| workload | task | bytes per launch | source |`); None if there
+    is no capture for that pair."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.md")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        cells = [c.strip() for c in line.strip().strip("|").split("|")]
+        if len(cells) >= 3 and cells[0] == workload and cells[1] == kind:
+            try:
+                return float(cells[2])
+            except ValueError:
+                return None
+    return None
+
+
+def roofline(workload, wl, kinds, peaks):
+    wm = work_model(wl["layers"], wl["batch"], wl["momentum"])
+    dom = max(("forward", "delta", "G", "update"), key=lambda k: kinds[k]["total_ms"])
+    per = wm[dom]
+    avg_bytes = sum(p["bytes"] for p in per) / len(per)
+    avg_flops = sum(p["flops"] for p in per) / len(per)
+    avg_s = kinds[dom]["avg_us"] * 1e-6
+    ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if avg_flops / max(avg_bytes, 1.0) > ridge:
+        roof = {"bound": "tensor", "achieved": avg_flops / avg_s / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "peak_kind": "sustained (kernel timed inside a seconds-long step loop)",
+                "frac_of_burst_peak": avg_flops / avg_s / 1e12 / peaks["bf16_tflops"]}
+    else:
+        roof = {"bound": "hbm", "achieved": avg_bytes / avg_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = ncu_traffic(workload, dom)
+    roof["kernel"] = KERNEL_NAMES[dom]
+    roof["task"] = dom
+    roof["peak_source"] = "of " + peaks["_source"]
+    roof["avg_launch_us"] = kinds[dom]["avg_us"]
+    roof["avg_launch_us_overlapped"] = kinds[dom].get("avg_us_overlapped")
+    roof["timing"] = ("CUDA events around every launch of the kernel, on the stream it runs on, in a pass of the same "
+                      "steps with all tasks on one stream; avg_launch_us_overlapped is the same measurement under the "
+                      "concurrent schedule")
+    roof["algorithmic_per_launch"] = {"bytes": avg_bytes, "flops": avg_flops}
+    # every contraction kind against the tensor roof (the metric's "tensor-pipe utilisation vs peak")
+    roof["contractions"] = {}
+    for k in ("forward", "delta", "G"):
+        if kinds[k]["launches"]:
+            fl = sum(p["flops"] for p in wm[k]) / len(wm[k])
+            t = fl / (kinds[k]["avg_us"] * 1e-6) / 1e12
+            roof["contractions"][k] = {"tflops": t, "frac_of_sustained": t / peaks["bf16_tflops_sustained"],
+                                       "frac_of_burst": t / peaks["bf16_tflops"], "avg_us": kinds[k]["avg_us"]}
+    return roof, wm
+
+
+def step_figures(wm, ms_per_step, peaks):
+    step_flops = sum(p["flops"] for k in ("forward", "delta", "G") for p in wm[k])
+    step_bytes = sum(p["bytes"] for k in wm for p in wm[k])
+    s = ms_per_step * 1e-3
+    return {"tflops": step_flops / s / 1e12, "gbs_algorithmic": step_bytes / s / 1e9,
+            "frac_of_bf16_sustained": step_flops / s / 1e12 / peaks["bf16_tflops_sustained"],
+            "frac_of_bf16_burst": step_flops / s / 1e12 / peaks["bf16_tflops"],
+            "frac_of_hbm": step_bytes / s / 1e9 / peaks["hbm_gbs"]}
+
+
+def short_measure(torch, lpb, name, dev, stream, peaks, seconds=0.6):
+    """samples/s of one workload under both schedules, a fraction of a second each (the
+    per_workload object of the JSON line)."""
+    w = Workload(torch, name, dev)
+    steps = {"mlp4_784": 200, "mlp8_4096": 50, "vgg_small_32": 50, "vgg16_224": 10, "mlp16_8192": 10}.get(name, 20)
+    out = {"batch": w.B}
+    for sched, key in ((lpb.LP_SCHED_LAYERPIPE, "layerpipe"), (lpb.LP_SCHED_FUSED_B, "fused_b")):
+        tr, ts, launches, _, (stage, delays, _) = throughput(torch, lpb, w, sched, steps, 3, seconds, stream)
+        tr.close()
+        del tr
+        torch.cuda.empty_cache()
+        sm = summarize(ts, steps)
+        out[key] = {"samples_per_s": w.B / (sm["ms_per_step"] * 1e-3), "ms_per_step": sm["ms_per_step"],
+                    "blocks": sm["blocks"], "steps_per_block": steps}
+        out["delays"] = delays
+        out["launches_per_step"] = launches // steps
+    out["speedup_vs_fused_b"] = out["layerpipe"]["samples_per_s"] / out["fused_b"]["samples_per_s"]
+    wm = work_model(w.layers, w.B, w.wl["momentum"])
+    out["step"] = step_figures(wm, out["layerpipe"]["ms_per_step"], peaks)
+    del w
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args):
     import torch
     from paper_2108_06629_b200 import binding as lpb
 
@@ -248,25 +417,14 @@ def run_ours(args, wl):
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        backend = os.environ.get("LP_BENCH_BACKEND", "nccl")
+        dist.init_process_group(backend, device_id=torch.device("cuda", local) if backend == "nccl" else None)
     lpb.lib()   # fails loudly if the CUDA library is missing
-
-    layers, B = wl["layers"], wl["batch"]
-    W0, b0 = I.initial_weights(layers, 0)
-    sched = lpb.LP_SCHED_FUSED_B if args.schedule == "fused_b" else lpb.LP_SCHED_LAYERPIPE
     dev = "cuda:%d" % local
-    tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
-                     schedule=sched, W0=W0, b0=b0, device=dev)
-    stage, delays, slots = tr.get_schedule()
-    P = 8
-    hx, hy = [], []
-    for n in range(P):
-        x, y = I.minibatch(layers, B, n)
-        hx.append(torch.from_numpy(x).pin_memory())
-        hy.append(torch.from_numpy(y).pin_memory())
-    xs = [t.to(dev) for t in hx]
-    ys = [t.to(dev) for t in hy]
     stream = torch.cuda.current_stream()
+    sched = lpb.LP_SCHED_FUSED_B if args.schedule == "fused_b" else lpb.LP_SCHED_LAYERPIPE
+    w = Workload(torch, args.workload, dev)
+    wl, layers, B = w.wl, w.layers, w.B
 
     def barrier():
         torch.cuda.synchronize()
@@ -275,118 +433,68 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        return replicas.max_over_ranks(ms, dist, dev)
+        return replicas.max_over_ranks(ms, dist, dev if (dist is None or dist.get_backend() == "nccl") else "cpu")
 
-    # warm-up: fill every ring (max delay + 3 minibatches) plus the requested W
-    prewarm = max(delays) + 3 + max(args.warmup, 3)
-    for k in range(prewarm):
-        tr.step(xs[k % P], ys[k % P])
-    tr.flush()
+    # ---- device-resident throughput: blocks of exactly K steps, repeated for >= 1.5 s ------------
     barrier()
-    # ---- device-resident throughput ---------------------------------------------------
     clocks = ClockSampler(local)
     time.sleep(0.25)
-    l0 = tr.kernel_launches()
-    ms = timed_loop(torch, tr, xs, ys, args.steps, stream)
-    launches = tr.kernel_launches() - l0
+    tr, ts, launches, prewarm, (stage, delays, slots) = throughput(torch, lpb, w, sched, args.steps, args.warmup,
+                                                                    args.min_seconds, stream)
     barrier()
-    ms = max_over_ranks(ms)
-    # ---- end to end: host buffers, copies inside the timed region --------------------------
-    xd = torch.empty_like(xs[0])
-    yd = torch.empty_like(ys[0])
-    first = prewarm + args.steps
+    dev_sum = summarize(ts, args.steps)
+    ms = max_over_ranks(dev_sum["ms_per_step"] * args.steps)
+    # ---- end to end: host buffers, copies inside the timed region --------------------------------
+    xd = [torch.empty_like(w.xs[0]) for _ in range(2)]
+    yd = [torch.empty_like(w.ys[0]) for _ in range(2)]
     lag = max(delays) + 1
-    ms_e2e = e2e_loop(torch, tr, hx, hy, xd, yd, args.steps, stream, lag, first)
+    state = {"first": prewarm + args.steps * len(ts)}
+
+    def e2e_once():
+        t = e2e_block(torch, tr, w.hx, w.hy, xd, yd, args.steps, stream, lag, state["first"])
+        state["first"] += args.steps
+        return t
+    ts_e2e = repeat_blocks(e2e_once, min(args.min_seconds, 1.0))
     barrier()
-    ms_e2e = max_over_ranks(ms_e2e)
+    e2e_sum = summarize(ts_e2e, args.steps)
+    ms_e2e = max_over_ranks(e2e_sum["ms_per_step"] * args.steps)
     clk = clocks.stop()
-    rc, detail = tr.device_status()
-    if rc != 0:
-        raise SystemExit("device status %d (%d): a bounded wait expired" % (rc, detail))
     tr.close()
     del tr
     torch.cuda.empty_cache()
 
-    # ---- same GPU, same kernels, backward as ONE task per layer (PipeDream-style) -------------
-    other = None
+    line = None
     if rank == 0:
+        peaks = load_peaks()
+        # ---- same GPU, same kernels, backward as ONE task per layer (PipeDream-style) -------------
         osched = lpb.LP_SCHED_LAYERPIPE if sched == lpb.LP_SCHED_FUSED_B else lpb.LP_SCHED_FUSED_B
-        tro = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
-                          schedule=osched, W0=W0, b0=b0, device=dev)
-        for k in range(prewarm):
-            tro.step(xs[k % P], ys[k % P])
-        tro.flush()
-        torch.cuda.synchronize()
-        ms_o = timed_loop(torch, tro, xs, ys, args.steps, stream)
+        tro, ts_o, _, _, _ = throughput(torch, lpb, w, osched, args.steps, args.warmup, min(args.min_seconds, 1.0), stream)
         tro.close()
         del tro
         torch.cuda.empty_cache()
+        o_sum = summarize(ts_o, args.steps)
         other = {"schedule": "layerpipe" if osched == lpb.LP_SCHED_LAYERPIPE else "fused_b",
-                 "value": args.steps * B / (ms_o * 1e-3), "unit": "samples/s (1 GPU)", "ms_per_step": ms_o / args.steps}
-
-    line = None
-    if rank == 0:
-        # ---- per-kernel times for the roofline (separate handles with timing events) ----------
-        # In the real schedule up to a dozen kernels share the GPU, so a kernel's event-timed
-        # duration there is the time it spent sharing, not its own cost.  The roofline therefore
-        # uses a second pass of the same steps with every task on one stream (LP_SERIAL_TASKS: the
-        # same kernels, launches and operands, none overlapping); the overlapped averages are
-        # reported beside it.
-        def kernel_times(flags):
-            trp = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
-                              schedule=sched, flags=flags, W0=W0, b0=b0, device=dev)
-            for k in range(prewarm):
-                trp.step(xs[k % P], ys[k % P])
-            trp.flush()
-            torch.cuda.synchronize()
-            trp.reset_task_times()
-            nprof = min(args.steps, 32768 // (6 * len(layers)))
-            timed_loop(torch, trp, xs, ys, nprof, stream)
-            out = {}
-            for kind in ("forward", "delta", "G", "update", "loss", "cast"):
-                n, tot = trp.task_time(kind)
-                out[kind] = dict(launches=n, total_ms=tot, avg_us=1e3 * tot / max(n, 1))
-            trp.close()
-            del trp
-            torch.cuda.empty_cache()
-            return out
-
-        kinds_live = kernel_times(lpb.LP_TIME_TASKS)
-        kinds = kernel_times(lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS)
+                 "value": B / (o_sum["ms_per_step"] * 1e-3), "unit": "samples/s (1 GPU)", **o_sum}
+        # ---- per-kernel times for the roofline ---------------------------------------------------
+        # Under the real schedule up to a dozen kernels share the GPU, so a kernel's event-timed
+        # duration there is the time it spent sharing, not its own cost.  The roofline uses a second
+        # pass of the same steps with every task on one stream (LP_SERIAL_TASKS: the same kernels,
+        # launches and operands, none overlapping); the overlapped averages are reported beside it.
+        kinds_live = kernel_times(torch, lpb, w, sched, lpb.LP_TIME_TASKS, args.steps, stream)
+        kinds = kernel_times(torch, lpb, w, sched, lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS, args.steps, stream)
         for kind in kinds:
             kinds[kind]["avg_us_overlapped"] = kinds_live[kind]["avg_us"]
-        peaks = load_peaks()
-        wm = work_model(layers, B, wl["momentum"])
-        dom = max(("forward", "delta", "G", "update"), key=lambda k: kinds[k]["total_ms"])
-        per = wm[dom]
-        avg_bytes = sum(p["bytes"] for p in per) / len(per)
-        avg_flops = sum(p["flops"] for p in per) / len(per)
-        avg_s = kinds[dom]["avg_us"] * 1e-6
-        ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-        if avg_flops / max(avg_bytes, 1.0) > ridge:
-            roof = {"bound": "tensor", "achieved": avg_flops / avg_s / 1e12, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s"}
-        else:
-            roof = {"bound": "hbm", "achieved": avg_bytes / avg_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-        roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.workload, dom))
-        roof["kernel"] = {"forward": "gemm_tcgen05_kernel<forward>", "delta": "gemm_tcgen05_kernel<delta>",
-                          "G": "gemm_tcgen05_kernel<G>", "update": "sgd_update_kernel"}[dom]
-        roof["peak_source"] = "of " + peaks["_source"]
-        roof["avg_launch_us"] = kinds[dom]["avg_us"]
-        roof["avg_launch_us_overlapped"] = kinds[dom]["avg_us_overlapped"]
-        roof["timing"] = ("CUDA events around every launch of the kernel in a pass of the same steps with all tasks on "
-                          "one stream; avg_launch_us_overlapped is the same measurement under the concurrent schedule")
-        roof["algorithmic_per_launch"] = {"bytes": avg_bytes, "flops": avg_flops}
-        # whole-step figures against both roofs
-        step_flops = sum(p["flops"] for k in ("forward", "delta", "G") for p in wm[k])
-        step_bytes = sum(p["bytes"] for k in wm for p in wm[k])
-        step_s = ms * 1e-3 / args.steps
-        # ---- the oracle on the host cores, bounded sample ---------------------------------------
+        roof, wm = roofline(args.workload, wl, kinds, peaks)
+        del w
+        torch.cuda.empty_cache()
+        per_workload = {}
+        if not args.no_per_workload and world == 1:
+            for name in I.WORKLOADS:
+                per_workload[name] = short_measure(torch, lpb, name, dev, stream, peaks)
         cpu = cpu_baseline(wl)
         value = world * args.steps * B / (ms * 1e-3)
         e2e_value = world * args.steps * B / (ms_e2e * 1e-3)
-        in_bytes = xs[0].numel() * xs[0].element_size() + ys[0].numel() * ys[0].element_size()
+        in_bytes = xd[0].numel() * xd[0].element_size() + yd[0].numel() * yd[0].element_size()
         line = {
             "metric": "training samples/sec", "value": value, "unit": "samples/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -394,19 +502,21 @@ def run_ours(args, wl):
             "config": {"workload": args.workload, "batch": B, "stages_used": max(stage) + 1, "delays": delays,
                        "ring_slots": slots, "schedule": args.schedule, "parallelism": "replicas only",
                        "l2": "working set per step exceeds L2 (weights + update streams), no flush",
-                       "prewarm_steps": prewarm},
+                       "prewarm_steps": prewarm,
+                       "timed_region": "blocks of exactly `steps` lp_step calls + lp_flush between CUDA events, device idle on both "
+                                       "sides; repeated until >= %.1f s were measured; value = median block" % args.min_seconds},
+            "timing": dev_sum,
             "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": 4,
-                    "ms_per_step": ms_e2e / args.steps},
+                    **e2e_sum},
             "gpu_launches": int(launches),
             "clocks": clk,
             "roofline": roof,
-            "step": {"tflops": step_flops / step_s / 1e12, "gbs_algorithmic": step_bytes / step_s / 1e9,
-                     "frac_of_bf16_sustained": step_flops / step_s / 1e12 / peaks["bf16_tflops_sustained"],
-                     "frac_of_hbm": step_bytes / step_s / 1e9 / peaks["hbm_gbs"]},
+            "step": step_figures(wm, ms / args.steps, peaks),
             "kernels": kinds,
             "other_schedule": other,
             "speedup_vs_fused_b": ((value / world) / other["value"] if other["schedule"] == "fused_b"
                                    else other["value"] / (value / world)),
+            "per_workload": per_workload,
             "cpu_baseline": cpu,
         }
     if dist is not None:
@@ -443,18 +553,26 @@ def cpu_baseline(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mlp8_4096", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--workload", default="mlp16_8192", choices=sorted(I.WORKLOADS))
     ap.add_argument("--schedule", default="layerpipe", choices=["layerpipe", "fused_b"])
+    ap.add_argument("--min-seconds", dest="min_seconds", type=float, default=MIN_TIMED_SECONDS)
+    ap.add_argument("--no-per-workload", dest="no_per_workload", action="store_true")
     args = ap.parse_args()
-    wl = I.WORKLOADS[args.workload]
+    if args.steps < 1 or args.gpus < 1:
+        raise SystemExit("--steps and --gpus must be positive")
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:
-            run_reference(args, wl)
+            run_reference(args, I.WORKLOADS[args.workload])
         return
-    run_ours(args, wl)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: run the N replicas ourselves, one process per GPU
+        out = replicas.spawn_replicas([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+        sys.stdout.write(out)
+        return
+    run_ours(args)
 
 
 if __name__ == "__main__":

@@ -7,8 +7,9 @@ binary32 number.  Rounding to nearest with ties to even therefore has a closed
 form on the bit pattern: add 0x7FFF plus the lowest kept bit, then clear the
 low 16 bits.  NaNs are passed through quietly (the add could otherwise carry a
 NaN payload into the exponent).  The paper fixes no precision; the rounding
-points at which this function is applied are listed in
-``layerpipe_oracle.train``.
+points at which this function is applied are listed in the module docstring
+of ``layerpipe_oracle`` (mirror mode) and applied by
+``DelayedGradientTrainer._Q``.
 """
 import numpy as np
 

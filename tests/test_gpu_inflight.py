@@ -147,7 +147,7 @@ def test_inflight_convnet_with_planned_delays_of_four_and_more():
     halo-tile and split-K G kernels, delays up to 5."""
     from paper_2108_06629_b200 import inputs as I
     layers = I.vgg(32, [32, 32, "P", 64, 64, "P", 128, "P"], [96, 10])
-    check("cnn32", layers, 16, 6, None, 0.01, 0.9, 14, loss_bound=3e-2, dw_bound=0.25)
+    check("cnn32", layers, 16, 6, None, 0.0005, 0.9, 14, loss_bound=3e-2, dw_bound=0.25)   # (larger steps blow the loss up to 10 within four minibatches)
 
 
 def test_inflight_delays_longer_than_the_delta_slots_and_out_of_order():

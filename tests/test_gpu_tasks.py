@@ -17,7 +17,7 @@ from gpu_common import assert_bf16_close, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None, fused=True, bias=True):
+def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps=None, fused=True, bias=True, check_layers=None):
     from oracle import layerpipe_oracle as O
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
@@ -30,6 +30,12 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
     orc = O.DelayedGradientTrainer(layers, delays, lr, mu, W0, b0, mirror=True, dtype=np.float32)
     L = len(layers)
     worst = {}
+
+    def k_fwd(l):       # terms of layer l's forward contraction (its delta contraction has k_bwd terms)
+        return layers[l]["n_in"] * (layers[l].get("R", 1) * layers[l].get("S", 1))
+
+    def k_bwd(l):
+        return layers[l]["n_out"] * (layers[l].get("R", 1) * layers[l].get("S", 1))
 
     def note(k, v):
         worst[k] = max(worst.get(k, 0.0), v)
@@ -45,26 +51,27 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
         if check_steps is not None and n not in check_steps:
             continue
         slot = rec["slot"]
+        todo = range(L) if check_layers is None else sorted(check_layers)     # layers whose tasks are run and compared
         # weight versions this minibatch reads
-        for l in range(L):
+        for l in todo:
             Wv, bv = stash[l][rec["v"][l]]
             tr.debug_write("ring_w", l, slot[l], Wv)
             if bias:
                 tr.debug_write("ring_b", l, slot[l], bv)
         tr.debug_write("labels", 0, n, y.astype(np.float32))
         # forward tasks
-        for l in range(L):
+        for l in todo:
             tr.debug_write("input", l, n, rec["a"][l])
             tr.debug_run_task("forward", l, n)
             if l < L - 1:
-                note("a", assert_bf16_close(tr.debug_read("input", l + 1, n), rec["a"][l + 1], "a^%d step %d" % (l + 1, n)))
+                note("a", assert_bf16_close(tr.debug_read("input", l + 1, n), rec["a"][l + 1], "a^%d step %d" % (l + 1, n), k_terms=k_fwd(l)))
                 if layers[l].get("pool", 0):
                     # which window element wins may legitimately differ where two candidates are within
                     # a rounding of each other; everywhere else the recorded position must agree
                     same = float((tr.debug_read("pool_idx", l, n) == rec["amax"][l]).mean())
                     assert same > 0.995, ("pool argmax", l, n, same)
                 if layers[l]["act"] == "gelu":
-                    note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n)))
+                    note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n), k_terms=k_fwd(l)))
             else:
                 r = rel_l2(tr.debug_read("logits", 0, n), rec["zL"])
                 assert r < 1e-5, ("logits", n, r)
@@ -76,7 +83,7 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
         loss = float(tr.debug_read("loss", 0, n)[0])
         assert abs(loss - rec["loss"]) <= 2e-6 * max(1.0, abs(rec["loss"])), (loss, rec["loss"])
         # backward tasks
-        for l in range(L - 1, -1, -1):
+        for l in reversed(todo):
             tr.debug_write("delta", l, n, rec["delta"][l])
             tr.debug_write("input", l, n, rec["a"][l])
             if l > 0:
@@ -86,7 +93,7 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                     tr.debug_write("pool_idx", l - 1, n, rec["amax"][l - 1].astype(np.float32))
                 tr.debug_run_task("delta", l, n)
                 note("delta", assert_bf16_close(tr.debug_read("delta", l - 1, n), rec["delta"][l - 1],
-                                                "delta^%d step %d" % (l - 1, n)))
+                                                "delta^%d step %d" % (l - 1, n), k_terms=k_bwd(l)))
             # pre-update state of the oracle; with the fused update the G kernel itself applies Eq. 6
             tr.debug_write("master_w", l, 0, pre_W[l])
             if bias:
@@ -97,7 +104,8 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                     tr.debug_write("mom_b", l, 0, pre_mb[l])
             tr.debug_run_task("G", l, n)
             r = rel_l2(tr.debug_read("grad_w", l, 0), rec["dW"][l])
-            assert r < 2e-5, ("G", l, n, r)
+            k_g = int(np.prod(rec["delta"][l].shape[:-1]))        # terms of the G contraction: samples (x pixels)
+            assert r < 2e-5 + 1e-7 * np.sqrt(k_g), ("G", l, n, r)   # fp32 accumulation over k_g terms on both sides
             note("G", r)
             if not fused:
                 tr.debug_write("grad_w", l, 0, rec["dW"][l])      # Eq. 6 from the oracle's gradient
@@ -250,7 +258,9 @@ def test_tasks_mlp16_8192_full_size_one_minibatch():
     for all three contractions, the update of 67 M weights per layer in the G kernel."""
     from paper_2108_06629_b200 import inputs as I
     wl = I.WORKLOADS["mlp16_8192"]
-    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 1)
+    # (the sixteen layers have one shape: first, second, one in the middle and the last are run)
+    w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 1,
+                           check_layers={0, 1, 9, 15})
     print("mlp16_8192 worst per-task errors", w)
 
 

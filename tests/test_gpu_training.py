@@ -13,7 +13,8 @@ between the two sides in its last bits, a different rounding of one element pert
 next layer, and after a few layers the two trajectories differ by bf16 rounding noise
 (and, with ReLU at small batch, by a few flipped gates).  That bound is asserted where
 it applies -- task by task on identical operands, in test_gpu_tasks.py -- and here the
-free-running gradients are held to the noise level derived in the design notes."""
+free-running quantities are held to a small multiple of what separates two correct CPU
+executions of the same recursion (the oracle in float32 and in float64; see chaos_level)."""
 import numpy as np
 import pytest
 
@@ -59,15 +60,32 @@ def oracle_run(layers, batch, delays, lr, mu, steps, W0, b0):
     return orc, recs
 
 
-def rounding_noise(n_layers):
-    """Free-running disagreement caused by independent bf16 roundings: one rounding has
-    relative error up to 2^-9; a gradient of the first layer sits behind about 2 L of them
-    (L forward stores, L backward stores), which add in quadrature."""
-    return 2.0 ** -9 * np.sqrt(2.0 * n_layers)
+def chaos_level(key):
+    """How far two CORRECT executions of the same recursion drift apart when only their
+    accumulation arithmetic differs (the oracle in float32 against the oracle in float64, both
+    rounding to bf16 at the same points): tests/golden/chaos_levels.json, written by
+    tests/golden/make_chaos_levels.py from the oracle alone.  No GPU value enters it."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "chaos_levels.json")) as f:
+        return json.load(f)[key]
 
 
-def compare(name, layers, batch, stages, delays, lr, mu, steps, grad_bound, step0_bound, loss_bound=5e-3, dw_bound=5e-2):
+CHAOS_FACTOR = 2.5     # a GPU run may sit this many times further from the fp32 oracle than the fp64 oracle does
+
+
+def compare(name, layers, batch, stages, delays, lr, mu, steps, floors=(2e-3, 2e-3, 1e-3, 5e-3)):
+    """Bounds = CHAOS_FACTOR x the oracle-vs-oracle separation of this very configuration (never below
+    `floors` = (first-step gradient, later gradients, loss, weight change): where the oracle pair
+    happens to agree to 1e-8, e.g. a first step without a single flipped ReLU gate, the GPU is
+    still allowed its summation-order noise)."""
     from paper_2108_06629_b200 import binding as lpb
+    lvl = chaos_level(name)
+    assert lvl["steps"] == steps
+    step0_bound = max(floors[0], CHAOS_FACTOR * lvl["grad_step0"])
+    grad_bound = max(floors[1], CHAOS_FACTOR * lvl["grad_later"])
+    loss_bound = max(floors[2], CHAOS_FACTOR * lvl["loss"])
+    dw_bound = max(floors[3], CHAOS_FACTOR * lvl["weight_change"])
     a, W0, b0 = free_run(layers, batch, stages, delays, lr, mu, steps, lpb.LP_SCHED_LAYERPIPE)
     b, _, _ = free_run(layers, batch, stages, delays, lr, mu, steps, lpb.LP_SCHED_FUSED_B)
     L = len(layers)
@@ -81,67 +99,70 @@ def compare(name, layers, batch, stages, delays, lr, mu, steps, grad_bound, step
     stage, delay, slots = a["schedule"]
     orc, recs = oracle_run(layers, batch, delay, lr, mu, steps, W0, b0)
     assert slots == [d + 1 for d in delay]
-    worst_g = 0.0
+    g0 = g_later = worst_loss = 0.0
     for n in range(steps):
         vf, vb, sl = a["vlog"][n]
         assert vf == recs[n]["v"] and vb == recs[n]["v"] and sl == recs[n]["slot"]      # bit-exact
-        assert abs(a["loss"][n] - recs[n]["loss"]) <= loss_bound * abs(recs[n]["loss"])
-        for l in range(L):
-            g = rel_l2(a["grads"][n][l][0], recs[n]["dW"][l])
-            worst_g = max(worst_g, g)
-            assert g <= (step0_bound if n == 0 else grad_bound), (name, "dW", n, l, g)
+        worst_loss = max(worst_loss, abs(a["loss"][n] - recs[n]["loss"]) / abs(recs[n]["loss"]))
+        g = max(rel_l2(a["grads"][n][l][0], recs[n]["dW"][l]) for l in range(L))
+        if n == 0:
+            g0 = g
+        else:
+            g_later = max(g_later, g)
     Wf, bf = orc.weights()
-    worst_w = worst_dw = 0.0
+    worst_w = worst_dw = worst_b = 0.0
     for l in range(L):
         W, bb, ver = a["W"][l]
         assert ver == steps
-        rw = rel_l2(W, Wf[l])
-        rd = rel_l2(W - W0[l], Wf[l] - W0[l])
-        worst_w, worst_dw = max(worst_w, rw), max(worst_dw, rd)
-        assert rw <= 5e-3, (name, "W", l, rw)
-        assert rd <= dw_bound, (name, "W - W0", l, rd)
-        assert rel_l2(bb, bf[l]) <= max(5e-2, dw_bound), (name, "b", l)
-    print("%s: worst free-running dW error %.2e, weights %.2e, weight change %.2e, launches %d"
-          % (name, worst_g, worst_w, worst_dw, a["launches"]))
+        worst_w = max(worst_w, rel_l2(W, Wf[l]))
+        worst_dw = max(worst_dw, rel_l2(W - W0[l], Wf[l] - W0[l]))
+        worst_b = max(worst_b, rel_l2(bb, bf[l]))
+    print("%s: free-running GPU vs oracle / bound (oracle fp32 vs fp64): dW step 0 %.2e / %.2e (%.2e), later %.2e / %.2e (%.2e), "
+          "loss %.2e / %.2e (%.2e), weight change %.2e / %.2e (%.2e), weights %.2e, launches %d"
+          % (name, g0, step0_bound, lvl["grad_step0"], g_later, grad_bound, lvl["grad_later"], worst_loss, loss_bound,
+             lvl["loss"], worst_dw, dw_bound, lvl["weight_change"], worst_w, a["launches"]))
+    assert g0 <= step0_bound, (name, "dW of the first step", g0, step0_bound)
+    assert g_later <= grad_bound, (name, "dW of later steps", g_later, grad_bound)
+    assert worst_loss <= loss_bound, (name, "loss", worst_loss, loss_bound)
+    assert worst_w <= 5e-3, (name, "W", worst_w)
+    assert worst_dw <= dw_bound, (name, "W - W0", worst_dw, dw_bound)
+    assert worst_b <= max(5e-2, dw_bound), (name, "b", worst_b)
 
 
 def test_free_running_mlp4_784():
     from paper_2108_06629_b200 import inputs as I
     wl = I.WORKLOADS["mlp4_784"]
-    compare("mlp4_784", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], wl["steps"],
-            grad_bound=0.15, step0_bound=2e-3)      # ReLU at batch 32: a flipped gate moves dW by ~1e-2
+    compare("mlp4_784", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], wl["steps"])
 
 
 def test_free_running_gelu_momentum_planned_stages():
     """No explicit delays: stage map and delays come from Algorithm 1."""
     from paper_2108_06629_b200 import inputs as I
     layers = I.mlp([384] * 6 + [100], "gelu")
-    compare("gelu6", layers, 96, 4, None, 0.02, 0.9, 12, grad_bound=5 * rounding_noise(6),
-            step0_bound=1.5 * rounding_noise(6))
+    compare("gelu6", layers, 96, 4, None, 0.02, 0.9, 12)
 
 
 def test_free_running_mlp8_4096_full_size():
     from paper_2108_06629_b200 import inputs as I
     wl = I.WORKLOADS["mlp8_4096"]
-    compare("mlp8_4096", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 12,
-            grad_bound=5 * rounding_noise(8), step0_bound=1.5 * rounding_noise(8))
+    compare("mlp8_4096", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 12)
 
 
 def test_free_running_small_convnet_planned_stages():
     from paper_2108_06629_b200 import inputs as I
     layers = I.vgg(16, [16, 32, "P", 64, "P"], [48, 10])
-    compare("cnn16", layers, 32, 3, None, 0.02, 0.9, 8, grad_bound=0.2, step0_bound=2e-2)
+    compare("cnn16", layers, 32, 3, None, 0.02, 0.9, 8)
 
 
 def test_free_running_vgg_small_32_full_config():
     from paper_2108_06629_b200 import inputs as I
     wl = I.WORKLOADS["vgg_small_32"]
     compare("vgg_small_32", wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"],
-            wl["steps"], grad_bound=0.3, step0_bound=0.1, loss_bound=3e-2, dw_bound=0.25)
+            wl["steps"])
     # (ReLU gates and pooling winners are decisions: behind eight layers, 128 x 32 x 32 pixels, a
-    # few of them fall differently on the two sides and each moves the first layer's gradient by
-    # a visible amount -- measured 5e-2 on the first step.  The same configuration is held to one
-    # bf16 spacing task by task in test_gpu_tasks.py.)
+    # few of them fall differently on any two executions and each moves the first layer's gradient
+    # by a visible amount -- the float32 and float64 oracles already differ by 3e-2 on the first
+    # step.  The same configuration is held to one bf16 spacing task by task in test_gpu_tasks.py.)
 
 
 def test_bf16_input_equals_fp32_input_of_the_same_values():

@@ -282,3 +282,95 @@ def test_mirror_mode_stays_close_to_exact_and_rounds_operands():
         for t in rm["a"][:4] + rm["delta"]:
             assert np.array_equal(rn_bf16(t), t)      # operands really are bf16 values
         assert rm["dW"][0].dtype == np.float32
+
+
+# ----------------------------------------------------------------------------
+# where mirror mode rounds: an independent restatement with torch's own bf16 cast
+# ----------------------------------------------------------------------------
+def _tq(t):
+    """Round a float64 torch tensor to bf16 the way a bf16 store does (via binary32)."""
+    return t.float().bfloat16().double()
+
+
+def test_mirror_mode_rounding_points_are_where_a_bf16_store_happens():
+    """Mirror mode must round the weight VERSION handed to the contractions (not the master), the
+    STORED z (not the z the activation is computed from), each activation, delta^L and each
+    delta^{l-1} once, after the product with f'.  Restated here for a two-layer GELU net with
+    torch's bf16 cast; a dropped or misplaced rounding in the oracle changes thousands of elements
+    by a bf16 spacing (4e-3 relative), the comparison is exact."""
+    rng = np.random.default_rng(3)
+    B, n0, n1, n2, lr = 12, 40, 56, 10, 0.37
+    layers = [O.fc(n0, n1, "gelu"), O.fc(n1, n2, "none")]
+    W = [rng.standard_normal((n1, n0)) * 0.2, rng.standard_normal((n2, n1)) * 0.2]     # not bf16 values
+    b = [rng.standard_normal(n1) * 0.1, rng.standard_normal(n2) * 0.1]
+    orc = O.DelayedGradientTrainer(layers, [0, 0], lr, 0.0, W, b, mirror=True, dtype=np.float64)
+    Wt = [torch.tensor(w) for w in W]
+    bt = [torch.tensor(v) for v in b]
+    assert not np.array_equal(rn_bf16(W[0]), W[0].astype(np.float32))
+    for n in range(2):
+        x = rng.standard_normal((B, n0))
+        y = rng.integers(0, n2, size=B)
+        rec = orc.step(x, y, capture=True)
+        # the version in the stash is the rounded one, the master is not
+        assert np.array_equal(orc.stash[0][n + 1][0], rn_bf16(orc.W[0]).astype(np.float64))
+        assert not np.array_equal(orc.W[0], rn_bf16(orc.W[0]).astype(np.float64))
+        x0 = _tq(torch.tensor(x))
+        W1q, W2q = _tq(Wt[0]), _tq(Wt[1])
+        z1 = x0 @ W1q.T + bt[0]                                   # bias stays fp32/fp64: not rounded
+        zs1 = _tq(z1)
+        a1 = _tq(F.gelu(z1))                                      # f of the UNROUNDED z
+        zL = a1 @ W2q.T + bt[1]
+        p = torch.softmax(zL, dim=1)
+        p[torch.arange(B), torch.tensor(y)] -= 1.0
+        dL = _tq(p / B)
+        Phi = 0.5 * (1 + torch.erf(zs1 / np.sqrt(2.0)))
+        fprime = Phi + zs1 * torch.exp(-0.5 * zs1 * zs1) / np.sqrt(2 * np.pi)   # f' on the STORED z
+        d1 = _tq((dL @ W2q) * fprime)                             # one rounding, after the product
+        G2, G1 = dL.T @ a1, d1.T @ x0
+        assert np.array_equal(rec["a"][0], x0.numpy())
+        assert np.array_equal(rec["zs"][0], zs1.numpy())
+        assert np.array_equal(rec["a"][1], a1.numpy())
+        assert np.array_equal(rec["delta"][1], dL.numpy())
+        assert np.array_equal(rec["delta"][0], d1.numpy())
+        assert np.allclose(rec["zL"], zL.numpy(), rtol=0, atol=1e-12)
+        assert np.allclose(rec["dW"][1], G2.numpy(), rtol=0, atol=1e-12)
+        assert np.allclose(rec["dW"][0], G1.numpy(), rtol=0, atol=1e-12)
+        # sensitivity of this very test: each alternative placement is visibly different
+        assert not np.array_equal(_tq(F.gelu(zs1)).numpy(), a1.numpy())            # f of the rounded z
+        assert not np.array_equal(_tq(x0 @ Wt[0].T + bt[0]).numpy(), zs1.numpy())  # unrounded weights
+        assert not np.array_equal(_tq(_tq(dL @ W2q) * fprime).numpy(), d1.numpy())  # two roundings
+        Wt = [Wt[0] - lr * G1, Wt[1] - lr * G2]                   # Eq. 6 on the master
+        bt = [bt[0] - lr * d1.sum(0), bt[1] - lr * dL.sum(0)]
+        assert np.allclose(orc.W[0], Wt[0].numpy(), rtol=0, atol=1e-12)
+
+
+def test_mac_costs_count_the_multiply_accumulates_of_the_direct_loops():
+    """The planner's cost model says a layer costs B*Ho*Wo*Cout*R*S*Cin multiply-accumulates (FC:
+    B*in*out).  Counted here by running the direct loops of Eq. 1 over the zero-padded input, one
+    increment per multiply-accumulate; the loops' result is also the oracle's forward."""
+    from oracle import partition_oracle as P
+    rng = np.random.default_rng(4)
+    B = 2
+    lay = O.conv(3, 4, 7, 6, act="none", R=5, S=3, pad=2, stride=2)
+    x = rng.standard_normal((B, 7, 6, 3))
+    W = rng.standard_normal(O.weight_shape(lay))
+    Ho, Wo = O.conv_out_hw(lay)
+    xp = np.pad(x, ((0, 0), (2, 2), (2, 2), (0, 0)))
+    z = np.zeros((B, Ho, Wo, 4))
+    macs = 0
+    for n in range(B):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                for co in range(4):
+                    for r in range(5):
+                        for s in range(3):
+                            for ci in range(3):
+                                z[n, ho, wo, co] += xp[n, 2 * ho + r, 2 * wo + s, ci] * W[co, r, s, ci]
+                                macs += 1
+    assert np.allclose(z, O.linear_forward(lay, x, W), atol=1e-12)
+    fcl = O.fc(11, 5, "none")
+    fix, flex = P.mac_costs([lay, fcl], B)
+    assert fix[0] == 2 * macs and flex[0] == 0              # forward + G; the first layer has no delta
+    assert fix[1] == 2 * (B * 11 * 5) and flex[1] == B * 11 * 5
+    fix, flex = P.mac_costs([fcl, lay], B)
+    assert flex[1] == macs                                  # delta costs one contraction
