@@ -264,20 +264,24 @@ static cudaError_t configure_one() {
 
 // ---- two-CTA (SM pair) kernel ---------------------------------------------------------------
 template <bool A_MN, bool B_MN, int MODE>
-static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st) {
+static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st, const UpdMaps* um) {
   a.splits = 1;
   if (a.wait_limit <= 0) a.wait_limit = LP_WAIT_LIMIT_CYCLES;
+  static const UpdMaps no_maps{};
+  a.upd_tma = (MODE == EPI_WGRAD_UPDATE && um != nullptr && a.g.kind == GEOM_PLAIN) ? 1 : 0;
+  if (!a.upd_tma) um = &no_maps;
   const int stage_bytes = 32 * 1024;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   int s = g_force_stages > 0 ? g_force_stages : 3;               // 3 x 32 KiB: two CTAs per SM
-  s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb, 2)));
-  while (s > 2 && size_t(s) * stage_bytes + 1280 > 227 * 1024) --s;
+  s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb + (a.upd_tma ? GEMM2_BN / 32 : 0), 2)));
+  const size_t tail = 1024 + 256 + (a.upd_tma ? 1024 + UPD_RING_BYTES : 0);   // alignment slack, barriers, bf16 staging tile
+  while (s > 2 && size_t(s) * stage_bytes + tail > 227 * 1024) --s;
   a.num_stages = s;
   cudaLaunchConfig_t cfg = {};
   // (convolution geometry: M is a whole number of 128-pixel boxes, and an even one -- the caller checks)
   cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N + GEMM2_BN - 1) / GEMM2_BN, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = size_t(s) * stage_bytes + 1024 + 256;
+  cfg.dynamicSmemBytes = size_t(s) * stage_bytes + tail;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -286,12 +290,20 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE>, tmA, tmB, a);
+  if constexpr (MODE == EPI_WGRAD_UPDATE) {
+    if (a.upd_tma) return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, tmA, tmB, *um, a);
+  }
+  return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false>, tmA, tmB, *um, a);
 }
 template <bool A_MN, bool B_MN, int MODE>
 static cudaError_t configure_pair() {
-  return cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              227 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       227 * 1024);
+  if constexpr (MODE == EPI_WGRAD_UPDATE) {
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  }
+  return e;
 }
 #define LP_FOR_EACH_PAIR_VARIANT(X)   \
   X(false, false, EPI_FPROP)          \
@@ -374,7 +386,7 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
   if (bn == GEMM_BN_PAIR) {
     if (args.g.kind == GEOM_PIX_K) return cudaErrorInvalidValue;
 #define LP_TRYP(A, B, M) \
-  if (a_mn == A && b_mn == B && args.mode == M) return launch_pair<A, B, M>(tmA, tmB, args, st);
+  if (a_mn == A && b_mn == B && args.mode == M) return launch_pair<A, B, M>(tmA, tmB, args, st, um);
     LP_FOR_EACH_PAIR_VARIANT(LP_TRYP)
 #undef LP_TRYP
     return cudaErrorInvalidValue;

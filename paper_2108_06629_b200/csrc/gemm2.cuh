@@ -81,18 +81,28 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
       : "memory");
 }
 
-template <bool A_MN, bool B_MN, int MODE>
+// UTMA (EPI_WGRAD_UPDATE only): Eq. 6 on the accumulator tile with the fp32 master / momentum tile
+// streamed by TMA through the operand ring once the tile's k-blocks have passed -- each CTA fills
+// "chunks" of its own 128 rows x 32 columns (16 KiB + 16 KiB, one stage), its epilogue updates them in
+// place in shared memory and TMA stores write master, momentum and the bf16 ring image back.  A
+// chunk fill completes on the CTA's own barrier ufull[stage] (the operand fills of both CTAs
+// complete on the leader's full[stage]); both kinds of use release the stage through empty[stage],
+// so the ring position, and with it the phase of empty[], stays uniform in both CTAs.
+template <bool A_MN, bool B_MN, int MODE, bool UTMA = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                     const GemmArgs p) {
+                     const __grid_constant__ UpdMaps um, const GemmArgs p) {
+  static_assert(!UTMA || MODE == EPI_WGRAD_UPDATE, "the streamed update belongs to the G contraction");
   constexpr int STAGE_BYTES = GEMM_A_BYTES + 128 * GEMM_BK * 2;      // A rows + half of the B tile: 32 KiB
+  constexpr int kChunks = GEMM2_BN / 32;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int S = p.num_stages;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + size_t(S) * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
   uint64_t* acc_bar = empty_bar + GEMM_MAX_STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+  uint64_t* ufull_bar = acc_bar + 1;                                   // [GEMM_MAX_STAGES] chunk fills (UTMA)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ufull_bar + GEMM_MAX_STAGES);
   float* epi_tile = reinterpret_cast<float*>(smem);
 
   const int warp = threadIdx.x >> 5;
@@ -118,9 +128,15 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if (UTMA) {
+      tma_prefetch_desc(&um.W);
+      if (p.mW != nullptr) tma_prefetch_desc(&um.M);
+      tma_prefetch_desc(&um.R);
+    }
     for (int s = 0; s < S; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
+      mbar_init(&ufull_bar[s], 1);
     }
     mbar_init(acc_bar, 1);
     fence_barrier_init();
@@ -145,8 +161,8 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       uint32_t s = 0, ph = 0;
       int k0 = 0;
       int c_tap = 0, c_chunk = 0;                      // convolution: filter tap and 64-channel chunk of this k-block
-      for (int kb = 0; kb < num_kb; ++kb, k0 += GEMM_BK) {
-        ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u);
+      for (int kb = 0; kb < num_kb - p.starve_kb; ++kb, k0 += GEMM_BK) {
+        ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u, p.wait_limit);
         if (!ok) break;
         const uint32_t sa = smem0 + s * uint32_t(STAGE_BYTES);
         const uint32_t sb = sa + GEMM_A_BYTES;
@@ -181,10 +197,31 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         issued = kb + 1;
         if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
       }
+      int chunks_issued = 0;
+      if constexpr (UTMA) {
+        if (ok) {
+          const uint32_t bytes = p.mW != nullptr ? 2u * UPD_CHUNK_BYTES : uint32_t(UPD_CHUNK_BYTES);
+          const uint32_t ufull0 = smem_u32(ufull_bar);
+          for (int c = 0; c < kChunks; ++c) {
+            ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u, p.wait_limit);
+            if (!ok) break;
+            const uint32_t sa = smem0 + s * uint32_t(STAGE_BYTES);
+            const uint32_t ub = ufull0 + 8u * s;
+            mbar_arrive_expect_tx_addr(ub, bytes);
+            tma_load_2d_addr(sa, &um.W, ub, tm.n0 + c * 32, tm.m0);
+            if (p.mW != nullptr) tma_load_2d_addr(sa + UPD_CHUNK_BYTES, &um.M, ub, tm.n0 + c * 32, tm.m0);
+            chunks_issued = c + 1;
+            if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
       if (!ok) {
         atomicExch(p.status, 11);
+        // let copies already in flight land before the CTA's shared memory is released
         if (rank == 0)
-          for (int kb = max(0, issued - S); kb < issued; ++kb) mbar_wait(&full_bar[kb % S], (kb / S) & 1);
+          for (int kb = max(0, issued - S); kb < issued; ++kb) mbar_wait(&full_bar[kb % S], (kb / S) & 1, p.wait_limit);
+        for (int c = max(0, chunks_issued - S); c < chunks_issued; ++c)
+          mbar_wait(&ufull_bar[(num_kb + c) % S], uint32_t(c / S) & 1u, p.wait_limit);
       }
     }
   } else if (warp == 1) {
@@ -201,7 +238,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       uint32_t dA_lo = uint32_t(dA), dB_lo = uint32_t(dB);
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
-        ok = mbar_wait_addr(full0 + 8u * s, ph);
+        ok = mbar_wait_addr(full0 + 8u * s, ph, p.wait_limit);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
@@ -230,9 +267,104 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int sub_col = (lane & 7) * 4;
     const int row0 = tm.m0 + q * 32;
     constexpr bool upd = (MODE == EPI_WGRAD_UPDATE);
+    if constexpr (UTMA) {
+      // Every one of the 128 epilogue threads runs the same number of named barriers whatever
+      // happens: after a wait that ran out, the remaining chunks only keep the barrier count.
+      const uint32_t smem0 = smem_u32(smem), empty0 = smem_u32(empty_bar), ufull0 = smem_u32(ufull_bar);
+      const uint32_t ringbuf = smem_u32(full_bar) + 1024u;      // bf16 image of the chunk (8 KiB, 64-byte swizzle)
+      const int trow = q * 32 + lane;                           // row of this CTA's half tile = tensor-memory lane
+      bool good = mbar_wait(acc_bar, 0, p.wait_limit);
+      good = __all_sync(0xffffffffu, good);
+      if (!good && lane == 0) atomicExch(p.status, 13);
+      tc_fence_after();
+      uint32_t us = uint32_t(num_kb % S), pending_stage = 0;
+      bool pending = false;
+#pragma unroll 1
+      for (int c = 0; c < kChunks; ++c) {
+        const uint32_t sW = smem0 + us * uint32_t(STAGE_BYTES);
+        const uint32_t sM = sW + UPD_CHUNK_BYTES;
+        if (good) {
+          good = mbar_wait_addr(ufull0 + 8u * us, uint32_t(c / S) & 1u, p.wait_limit);
+          good = __all_sync(0xffffffffu, good);
+          if (!good && lane == 0) atomicExch(p.status, 14);
+        }
+        uint32_t packed[16];
+        if (good) {
+          uint32_t r[32];
+          tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+          tmem_ld_wait();
+          const uint32_t rowoff = uint32_t(trow) * 128u;
+          const uint32_t swz = uint32_t(trow & 7);
+          const int grow = tm.m0 + trow;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t off = rowoff + ((uint32_t(j) ^ swz) << 4);
+            float g[4] = {__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                          __uint_as_float(r[4 * j + 3])};
+            const int n = tm.n0 + c * 32 + 4 * j;
+            if (p.out != nullptr && grow < p.M && n < tm.nlim) {
+              float* dst = reinterpret_cast<float*>(p.out) + size_t(grow) * p.ld_out + n;
+              if (n + 3 < tm.nlim) {
+                __stcs(reinterpret_cast<float4*>(dst), make_float4(g[0], g[1], g[2], g[3]));
+              } else {
+                for (int e = 0; e < 4; ++e) if (n + e < tm.nlim) dst[e] = g[e];
+              }
+            }
+            float m[4] = {g[0], g[1], g[2], g[3]};
+            if (p.mW != nullptr) {
+              float4 mm;
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(mm.x), "=f"(mm.y), "=f"(mm.z), "=f"(mm.w) : "r"(sM + off));
+              m[0] = p.mu * mm.x + g[0]; m[1] = p.mu * mm.y + g[1];
+              m[2] = p.mu * mm.z + g[2]; m[3] = p.mu * mm.w + g[3];
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sM + off), "f"(m[0]), "f"(m[1]), "f"(m[2]), "f"(m[3]) : "memory");
+            }
+            float4 w;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w) : "r"(sW + off));
+            w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sW + off), "f"(w.x), "f"(w.y), "f"(w.z), "f"(w.w) : "memory");
+            packed[2 * j] = pack_bf16x2(w.x, w.y);
+            packed[2 * j + 1] = pack_bf16x2(w.z, w.w);
+          }
+        }
+        // the bf16 staging tile is free once the previous chunk's stores have read it; the same
+        // wait releases that chunk's stage to the producer
+        if (threadIdx.x == 64 && pending) {
+          tma_store_wait_read0();
+          mbar_arrive_addr(empty0 + 8u * pending_stage);
+          pending = false;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (good) {
+          const uint32_t roff = ringbuf + uint32_t(trow) * 64u;
+          const uint32_t rs = uint32_t(trow >> 1) & 3u;
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(roff + ((uint32_t(u) ^ rs) << 4)), "r"(packed[4 * u]),
+                         "r"(packed[4 * u + 1]), "r"(packed[4 * u + 2]), "r"(packed[4 * u + 3])
+                         : "memory");
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64) {
+          if (good) {
+            const int n = tm.n0 + c * 32;
+            tma_store_2d_addr(&um.W, sW, n, tm.m0);
+            if (p.mW != nullptr) tma_store_2d_addr(&um.M, sM, n, tm.m0);
+            tma_store_2d_addr(&um.R, ringbuf, n, tm.m0);
+            tma_store_commit();
+            pending = true;
+            pending_stage = us;
+          } else {
+            mbar_arrive_addr(empty0 + 8u * us);      // keep the producer's bounded waits short
+          }
+        }
+        if (++us == uint32_t(S)) us = 0;
+      }
+      if (pending) tma_store_wait_read0();           // (thread 64 only) shared memory must outlive the last stores' reads
+    } else {
     WmRegs cur;
     if constexpr (upd) load_wm(p, row0, tm.n0 + sub_col, tm.nlim, sub_row, cur);
-    bool ok = mbar_wait(acc_bar, 0);
+    bool ok = mbar_wait(acc_bar, 0, p.wait_limit);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok && lane == 0) atomicExch(p.status, 13);
     tc_fence_after();
@@ -257,6 +389,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           epilogue_rows8<MODE>(p, tm, tile, q, sub_row, sub_col, n);
         }
       }
+    }
     }
   }
   // neither CTA may release shared or tensor memory while its partner can still touch it

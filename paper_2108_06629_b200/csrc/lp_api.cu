@@ -521,7 +521,7 @@ static int build_tensor_maps(lp_ctx* c) {
       if ((rc = make_tmap_bf16_2d(&y.tm_d_B[s], y.ring + s * y.w_elems, y.n_in, y.n_out, y.ld_in, bB[0], bB[1], &err)) != LP_OK)
         return fail(c, rc, err);
     // G: A = delta^l stored [B][out] -> MN-major (M = out contiguous); B = a^{l-1} stored [B][in] -> MN-major
-    y.upd_maps = (y.bn_g == 128 || y.bn_g == 256) && y.split_g == 1;
+    y.upd_maps = (y.bn_g == 128 || y.bn_g == 256 || y.bn_g == GEMM_BN_PAIR) && y.split_g == 1;
     if (y.upd_maps) {
       if ((rc = make_tmap_rows32(&y.tm_u_W, y.W, 4, y.n_in, y.n_out, y.w_ld, GEMM_BM, &err)) != LP_OK) return fail(c, rc, err);
       if (y.mW && (rc = make_tmap_rows32(&y.tm_u_M, y.mW, 4, y.n_in, y.n_out, y.w_ld, GEMM_BM, &err)) != LP_OK) return fail(c, rc, err);
@@ -715,7 +715,7 @@ static inline bool fused_update(const lp_ctx* c) { return (c->cfg.flags & LP_UNF
 // The G kernel with the TMA update also does the bias gradient and bias update of a fully connected
 // layer (one launch less per layer); convolution layers and the other G forms keep the bias kernel.
 static inline bool fused_bias(const lp_ctx* c, const Layer& y) {
-  return fused_update(c) && y.upd_maps && y.d.has_bias && y.col_chunks == 0 && !y.conv;
+  return fused_update(c) && y.upd_maps && y.bn_g != GEMM_BN_PAIR && y.d.has_bias && y.col_chunks == 0 && !y.conv;
 }
 
 static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {

@@ -74,7 +74,7 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                     note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n), k_terms=k_fwd(l)))
             else:
                 r = rel_l2(tr.debug_read("logits", 0, n), rec["zL"])
-                assert r < 1e-5, ("logits", n, r)
+                assert r < 1e-5 + 1e-7 * np.sqrt(k_fwd(l)), ("logits", n, r)      # fp32 accumulation over k_fwd terms on both sides
                 note("logits", r)
         # loss task
         tr.debug_write("logits", 0, n, rec["zL"])
