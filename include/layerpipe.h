@@ -139,6 +139,24 @@ int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, int n_stages
  */
 int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev, void* stream);
 
+/*
+ * Operational parallelism (Section III-B, Fig. 5(c)-(d); Algorithm 1's OP(T_idle, T_flex)): the
+ * delta contraction of layer l is divided BY OUTPUT CHANNELS into delta'' -- borrowed by the
+ * processor that holds layer l+1 -- and delta', which stays with layer l; the two pieces are
+ * independent and run concurrently.  piece_stage / piece_amount: host [2 * n_layers] in the layout
+ * lp_plan / lp_plan_costs write ([2l] = delta'' or the whole, [2l+1] = delta'; amount 0 = no such
+ * piece).  For every layer with two pieces the columns of delta^{l-1} are divided in the ratio of
+ * the amounts, rounded to whole tiles of the contraction kernel (at least one tile each); piece
+ * [2l] is enqueued on the delta stream of stage piece_stage[2l], piece [2l+1] on that of
+ * piece_stage[2l+1], each with the unchanged f' epilogue, and delta^{l-1} counts as written when
+ * both have finished.  Layers whose delta kernel has a single column tile, or runs split-K, keep
+ * one piece.  The numbers do not change: every output element is produced by the same
+ * instructions in the same order as in the unsplit launch.  split_col_out (host [n_layers], may be
+ * NULL) receives the first column of delta' (0 = unsplit).  Must be called before the first
+ * lp_step; LP_SCHED_FUSED_B runs the pieces back to back inside its one backward task.
+ */
+int lp_set_delta_split(lp_handle h, const int* piece_stage, const long long* piece_amount, int* split_col_out);
+
 /* Make `stream` wait for everything enqueued so far (all updates applied: every layer
  * holds version = number of lp_step calls). Does not block the host. */
 int lp_flush(lp_handle h, void* stream);
@@ -217,6 +235,10 @@ int lp_device_status(lp_handle h, int* detail);
 enum { LP_TASK_CAST = 5 };
 int lp_get_task_time(lp_handle h, int task, long long* launches, double* total_ms);
 int lp_reset_task_times(lp_handle h);
+/* The same sums for one layer: Algorithm 1's `profile` step.  With LP_TIME_TASKS | LP_SERIAL_TASKS
+ * these are the costs of the tasks alone on the GPU: T_fix[l] = forward + G (+ update), T_flex[l] =
+ * delta, in any integer unit (e.g. nanoseconds), are what lp_plan_costs takes. */
+int lp_get_layer_task_time(lp_handle h, int task, int layer, long long* launches, double* total_ms);
 /* Needs LP_TIME_TASKS.  The timeline behind lp_get_task_time: for the first min(capacity, launches)
  * timed launches of `task`, in launch order, start_ms[i] and end_ms[i] (host arrays) receive the
  * kernel's begin and end in milliseconds after the first event timed since the last reset (of any

@@ -75,6 +75,8 @@ def lib():
         "lp_device_status": [vp, ip],
         "lp_get_task_time": [vp, C.c_int, llp, _P(C.c_double)],
         "lp_reset_task_times": [vp],
+        "lp_get_layer_task_time": [vp, C.c_int, C.c_int, llp, _P(C.c_double)],
+        "lp_set_delta_split": [vp, ip, llp, ip],
         "lp_get_task_timeline": [vp, C.c_int, C.c_int, _P(C.c_float), _P(C.c_float), _P(C.c_int)],
         "lp_set_tuning": [C.c_int, C.c_int, C.c_int],
         "lp_destroy": [vp],
@@ -97,7 +99,7 @@ def lib():
 
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
            "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
-           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
+           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_get_layer_task_time", "lp_set_delta_split", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
            "lp_gemm_bf16", "lp_gemm_status", "lp_debug_gemm_starved", "lp_softmax_xent_static"]
 
 
@@ -306,6 +308,23 @@ class Trainer:
         _check(lib().lp_get_task_timeline(self.h, k, capacity, st.ctypes.data_as(_P(C.c_float)),
                                           en.ctypes.data_as(_P(C.c_float)), C.byref(n)), self.h)
         return st[:n.value], en[:n.value]
+
+    def layer_task_time(self, task, layer):
+        """(launches, total milliseconds) of one task kind of one layer; needs flags=LP_TIME_TASKS."""
+        k = dict(self.TASK, cast=5)[task]
+        n, ms = C.c_longlong(), C.c_double()
+        _check(lib().lp_get_layer_task_time(self.h, k, layer, C.byref(n), C.byref(ms)), self.h)
+        return n.value, ms.value
+
+    def set_delta_split(self, piece_stage, piece_amount):
+        """Divide the delta contractions by output columns as a plan's pieces say (before the first
+        step).  Returns the first column of delta' per layer (0 = unsplit)."""
+        n = len(self.layers)
+        ps = (C.c_int * (2 * n))(*[int(x) for x in piece_stage])
+        pa = (C.c_longlong * (2 * n))(*[int(x) for x in piece_amount])
+        out = (C.c_int * n)()
+        _check(lib().lp_set_delta_split(self.h, ps, pa, out), self.h)
+        return list(out)
 
     def reset_task_times(self):
         _check(lib().lp_reset_task_times(self.h), self.h)

@@ -184,7 +184,7 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   a.kb_per_split = (num_kb + a.splits - 1) / a.splits;
   const int tiles_m = (a.M + GEMM_BM - 1) / GEMM_BM;
-  int tiles_n = (a.N + BN - 1) / BN;
+  int tiles_n = (a.N - a.n_begin + BN - 1) / BN;
   if (a.g.kind == GEOM_PIX_K) tiles_n = a.g.n_per_tap * (a.N / a.g.tap_pitch);   // (tap, channel block)
   const long long work = (long long)tiles_m * tiles_n * a.splits;
   // BN <= 128: two CTAs per SM (2 x 2 x BN tensor-memory columns); BN = 256: one.
@@ -273,13 +273,13 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   const int stage_bytes = 32 * 1024;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
   int s = g_force_stages > 0 ? g_force_stages : 3;               // 3 x 32 KiB: two CTAs per SM
-  s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb + (a.upd_tma ? GEMM2_BN / 32 : 0), 2)));
+  s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb + (a.upd_tma ? GEMM2_BN / 64 : 0), 2)));
   const size_t tail = 1024 + 256 + (a.upd_tma ? 1024 + UPD_RING_BYTES : 0);   // alignment slack, barriers, bf16 staging tile
   while (s > 2 && size_t(s) * stage_bytes + tail > 227 * 1024) --s;
   a.num_stages = s;
   cudaLaunchConfig_t cfg = {};
   // (convolution geometry: M is a whole number of 128-pixel boxes, and an even one -- the caller checks)
-  cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N + GEMM2_BN - 1) / GEMM2_BN, 1);
+  cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N - a.n_begin + GEMM2_BN - 1) / GEMM2_BN, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = size_t(s) * stage_bytes + tail;
   cfg.stream = st;

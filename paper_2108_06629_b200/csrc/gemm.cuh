@@ -58,6 +58,8 @@ struct ConvGeom {
 
 struct GemmArgs {
   int M, N, K;
+  int n_begin;              // first output column of this launch (a multiple of the tile width; columns [n_begin, N) are
+                            // computed): one piece of a contraction split by output columns (Section III-B, delta' / delta'')
   int num_stages;
   int mode;                 // EPI_*
   int act;                  // ACT_*  (FPROP: f of this layer; DGRAD: f' of the previous layer)
@@ -412,7 +414,7 @@ __device__ __forceinline__ TileCtx decode_tile(const GemmArgs& p, int t, int til
   c.kb_begin = (p.splits > 1) ? c.z * p.kb_per_split : 0;
   c.num_kb = (p.splits > 1) ? max(0, min(num_kb_total, c.kb_begin + p.kb_per_split) - c.kb_begin) : num_kb_total;
   c.tm.m0 = bx * GEMM_BM;
-  c.tm.n0 = by * BN;
+  c.tm.n0 = p.n_begin + by * BN;
   c.tm.nlim = p.N;
   c.tm.pn0 = c.tm.ph0 = c.tm.pw0 = 0;
   c.tap = 0;

@@ -113,7 +113,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
   TileMap tm;
   tm.m0 = (blockIdx.x >> 1) * 256 + int(rank) * 128;    // this CTA's 128 rows
-  tm.n0 = blockIdx.y * GEMM2_BN;                        // the pair's 256 columns
+  tm.n0 = p.n_begin + blockIdx.y * GEMM2_BN;            // the pair's 256 columns
   tm.nlim = p.N;
   tm.pn0 = tm.ph0 = tm.pw0 = 0;
   if (pix) {                                            // this CTA's box of 128 pixels
@@ -200,17 +200,21 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       int chunks_issued = 0;
       if constexpr (UTMA) {
         if (ok) {
-          const uint32_t bytes = p.mW != nullptr ? 2u * UPD_CHUNK_BYTES : uint32_t(UPD_CHUNK_BYTES);
+          // one fill = one stage = 32 KiB: master + momentum of a 32-column chunk, or (no momentum)
+          // the master of two neighbouring chunks -- the epilogue is bound by bytes in flight
+          const int per = p.mW != nullptr ? 1 : 2;
           const uint32_t ufull0 = smem_u32(ufull_bar);
-          for (int c = 0; c < kChunks; ++c) {
+          for (int f = 0; f < kChunks / per; ++f) {
             ok = mbar_wait_addr(empty0 + 8u * s, ph ^ 1u, p.wait_limit);
             if (!ok) break;
             const uint32_t sa = smem0 + s * uint32_t(STAGE_BYTES);
             const uint32_t ub = ufull0 + 8u * s;
-            mbar_arrive_expect_tx_addr(ub, bytes);
-            tma_load_2d_addr(sa, &um.W, ub, tm.n0 + c * 32, tm.m0);
-            if (p.mW != nullptr) tma_load_2d_addr(sa + UPD_CHUNK_BYTES, &um.M, ub, tm.n0 + c * 32, tm.m0);
-            chunks_issued = c + 1;
+            mbar_arrive_expect_tx_addr(ub, 2u * UPD_CHUNK_BYTES);
+            const int n = tm.n0 + f * per * 32;
+            tma_load_2d_addr(sa, &um.W, ub, n, tm.m0);
+            if (p.mW != nullptr) tma_load_2d_addr(sa + UPD_CHUNK_BYTES, &um.M, ub, n, tm.m0);
+            else                 tma_load_2d_addr(sa + UPD_CHUNK_BYTES, &um.W, ub, n + 32, tm.m0);
+            chunks_issued = f + 1;
             if (++s == uint32_t(S)) { s = 0; ph ^= 1u; }
           }
         }
@@ -220,8 +224,8 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         // let copies already in flight land before the CTA's shared memory is released
         if (rank == 0)
           for (int kb = max(0, issued - S); kb < issued; ++kb) mbar_wait(&full_bar[kb % S], (kb / S) & 1, p.wait_limit);
-        for (int c = max(0, chunks_issued - S); c < chunks_issued; ++c)
-          mbar_wait(&ufull_bar[(num_kb + c) % S], uint32_t(c / S) & 1u, p.wait_limit);
+        for (int f = max(0, chunks_issued - S); f < chunks_issued; ++f)
+          mbar_wait(&ufull_bar[(num_kb + f) % S], uint32_t(f / S) & 1u, p.wait_limit);
       }
     }
   } else if (warp == 1) {
@@ -277,14 +281,16 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       good = __all_sync(0xffffffffu, good);
       if (!good && lane == 0) atomicExch(p.status, 13);
       tc_fence_after();
+      const int per = p.mW != nullptr ? 1 : 2;                  // 32-column chunks per stage fill
       uint32_t us = uint32_t(num_kb % S), pending_stage = 0;
-      bool pending = false;
+      bool pending = false, pending_release = false;
 #pragma unroll 1
       for (int c = 0; c < kChunks; ++c) {
-        const uint32_t sW = smem0 + us * uint32_t(STAGE_BYTES);
-        const uint32_t sM = sW + UPD_CHUNK_BYTES;
-        if (good) {
-          good = mbar_wait_addr(ufull0 + 8u * us, uint32_t(c / S) & 1u, p.wait_limit);
+        const int f = c / per, sub = c % per;
+        const uint32_t sW = smem0 + us * uint32_t(STAGE_BYTES) + (per == 2 ? uint32_t(sub) * UPD_CHUNK_BYTES : 0u);
+        const uint32_t sM = sW + UPD_CHUNK_BYTES;                // (momentum form only)
+        if (good && sub == 0) {
+          good = mbar_wait_addr(ufull0 + 8u * us, uint32_t(f / S) & 1u, p.wait_limit);
           good = __all_sync(0xffffffffu, good);
           if (!good && lane == 0) atomicExch(p.status, 14);
         }
@@ -327,10 +333,10 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           }
         }
         // the bf16 staging tile is free once the previous chunk's stores have read it; the same
-        // wait releases that chunk's stage to the producer
+        // wait releases that chunk's stage to the producer when it was the stage's last chunk
         if (threadIdx.x == 64 && pending) {
           tma_store_wait_read0();
-          mbar_arrive_addr(empty0 + 8u * pending_stage);
+          if (pending_release) mbar_arrive_addr(empty0 + 8u * pending_stage);
           pending = false;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -345,6 +351,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         fence_proxy_async_smem();
         asm volatile("bar.sync 1, 128;" ::: "memory");
+        const bool last_of_stage = (sub == per - 1);
         if (threadIdx.x == 64) {
           if (good) {
             const int n = tm.n0 + c * 32;
@@ -353,12 +360,13 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             tma_store_2d_addr(&um.R, ringbuf, n, tm.m0);
             tma_store_commit();
             pending = true;
+            pending_release = last_of_stage;
             pending_stage = us;
-          } else {
+          } else if (last_of_stage) {
             mbar_arrive_addr(empty0 + 8u * us);      // keep the producer's bounded waits short
           }
         }
-        if (++us == uint32_t(S)) us = 0;
+        if (last_of_stage && ++us == uint32_t(S)) us = 0;
       }
       if (pending) tma_store_wait_read0();           // (thread 64 only) shared memory must outlive the last stores' reads
     } else {

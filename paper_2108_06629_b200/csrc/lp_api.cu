@@ -103,6 +103,11 @@ struct Layer {
   std::vector<Res> rX, rZ, rDelta, rRing, rPidx;
   Res rDW;
   Ev last_update;
+  // Section III-B: the delta contraction of this layer split by output columns into delta'' =
+  // columns [0, split_col), run on the streams of piece_stage[0] (the stage holding layer l+1),
+  // and delta' = columns [split_col, n_in), run on piece_stage[1].  split_col = 0: one piece.
+  int split_col = 0;
+  int piece_stage[2] = {0, 0};
 };
 
 }  // namespace lp
@@ -134,6 +139,7 @@ struct lp_ctx {
   std::vector<cudaEvent_t> tpool;              // timing events (LP_TIME_TASKS)
   size_t tpool_next = 0;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed[6];
+  std::vector<int> timed_layer[6];             // layer of each timed launch (-1: none)
   std::string err;
   int latched = 0;
   char* ws = nullptr;
@@ -562,12 +568,13 @@ struct TimedScope {
   cudaStream_t st;
   int kind;
   cudaEvent_t e1 = nullptr;
-  TimedScope(lp_ctx* c_, int kind_, cudaStream_t st_) : c(c_), st(st_), kind(kind_) {
+  TimedScope(lp_ctx* c_, int kind_, cudaStream_t st_, int layer = -1) : c(c_), st(st_), kind(kind_) {
     if ((c->cfg.flags & LP_TIME_TASKS) && c->tpool_next + 2 <= c->tpool.size()) {
       cudaEvent_t e0 = c->tpool[c->tpool_next++];
       e1 = c->tpool[c->tpool_next++];
       cudaEventRecord(e0, st);
       c->timed[kind].push_back({e0, e1});
+      c->timed_layer[kind].push_back(layer);
     }
   }
   ~TimedScope() {
@@ -639,7 +646,7 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   }
   a.splits = y.split_f; a.partial = y.part_f; a.tile_counter = y.cnt_f;
   ++c->launches;
-  TimedScope ts(c, LP_TASK_FORWARD, st);
+  TimedScope ts(c, LP_TASK_FORWARD, st, l);
   if (y.lean_f) {
     const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
     return conv_halo_launch(0, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], tmo, a, st);
@@ -657,16 +664,19 @@ static cudaError_t launch_pool(lp_ctx* c, int l, long long n, cudaStream_t st) {
   Layer& y = c->L[l];
   Layer& nx = c->L[l + 1];
   ++c->launches;
-  TimedScope ts(c, LP_TASK_FORWARD, st);
+  TimedScope ts(c, LP_TASK_FORWARD, st, l);
   return launch_maxpool2(y.a_full, nx.X + size_t(n % nx.x_slots) * nx.x_elems, y.pidx + size_t(n % nx.x_slots) * y.pidx_elems,
                          c->cfg.batch, y.imH, y.imW, y.ld_out, st);
 }
 
-static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
+// piece: -1 = the whole contraction; 0 = delta'' (columns [0, split_col)); 1 = delta' (the rest)
+static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st, int piece = -1) {
   Layer& y = c->L[l];
   Layer& pv = c->L[l - 1];
   GemmArgs a{};
   a.M = y.in_rows; a.N = y.n_in; a.K = y.n_out;
+  if (piece == 0) a.N = y.split_col;
+  if (piece == 1) a.n_begin = y.split_col;
   if (y.conv) {
     const int cpt = (y.ld_out + 63) / 64;
     a.K = y.taps * cpt * GEMM_BK;
@@ -703,7 +713,7 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
   a.status = c->status;
   a.splits = y.split_d; a.partial = y.part_d; a.tile_counter = y.cnt_d;
   ++c->launches;
-  TimedScope ts(c, LP_TASK_DELTA, st);
+  TimedScope ts(c, LP_TASK_DELTA, st, l);
   if (y.halo_d) {
     a.g = halo_geom(y, 1);
     return conv_halo_launch(1, y.tm_hd_A[n % kDeltaSlots], y.tm_d_B[ring_slot], y.tm_hd_A[0], a, st);
@@ -732,7 +742,7 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
       u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
     }
     c->launches += 2 * ((y.n_out + 63) / 64);
-    TimedScope ts(c, LP_TASK_G, st);
+    TimedScope ts(c, LP_TASK_G, st, l);
     return conv_halo_g_launch(y.tm_hf_A[n % y.x_slots], y.tm_hg_D[n % kDeltaSlots], halo_geom(y, 0), c->cfg.batch, y.part_g,
                               u, c->status, st);
   }
@@ -757,7 +767,7 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
     a.out = y.dW;
   }
   ++c->launches;
-  TimedScope ts(c, LP_TASK_G, st);
+  TimedScope ts(c, LP_TASK_G, st, l);
   if (fused_bias(c, y)) {
     a.bdelta = y.delta + size_t(n % kDeltaSlots) * y.delta_elems;
     a.bld = y.ld_out; a.brows = y.out_rows;
@@ -799,7 +809,7 @@ static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st)
   }
   u.lr = c->cfg.lr; u.mu = c->cfg.momentum;
   ++c->launches;
-  TimedScope ts(c, LP_TASK_UPDATE, st);
+  TimedScope ts(c, LP_TASK_UPDATE, st, l);
   return launch_sgd_update(u, st);
 }
 
@@ -985,10 +995,63 @@ extern "C" int lp_get_task_timeline(lp_handle h, int task, int capacity, float* 
   return LP_OK;
 }
 
+extern "C" int lp_get_layer_task_time(lp_handle h, int task, int layer, long long* launches, double* total_ms) {
+  if (!h || task < 0 || task > LP_TASK_CAST) return LP_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= int(h->L.size())) return fail(h, LP_ERR_INVALID_ARG, "layer index out of range");
+  if (!(h->cfg.flags & LP_TIME_TASKS)) return fail(h, LP_ERR_NOT_READY, "handle was created without LP_TIME_TASKS");
+  LP_CUDA(h, cudaDeviceSynchronize());
+  double tot = 0.0;
+  long long cnt = 0;
+  for (size_t i = 0; i < h->timed[task].size(); ++i) {
+    if (h->timed_layer[task][i] != layer) continue;
+    float ms = 0.f;
+    LP_CUDA(h, cudaEventElapsedTime(&ms, h->timed[task][i].first, h->timed[task][i].second));
+    tot += ms;
+    ++cnt;
+  }
+  if (launches) *launches = cnt;
+  if (total_ms) *total_ms = tot;
+  return LP_OK;
+}
+
+extern "C" int lp_set_delta_split(lp_handle h, const int* piece_stage, const long long* piece_amount, int* split_col_out) {
+  if (!h || !piece_stage || !piece_amount) return LP_ERR_INVALID_ARG;
+  if (h->n_steps != 0) return fail(h, LP_ERR_NOT_READY, "the split must be set before the first lp_step");
+  const int nL = int(h->L.size());
+  for (int l = 0; l < nL; ++l) {
+    const long long a0 = piece_amount[2 * l], a1 = piece_amount[2 * l + 1];
+    if (a0 < 0 || a1 < 0) return fail(h, LP_ERR_INVALID_ARG, "negative piece amount");
+    for (int k = 0; k < 2; ++k)
+      if ((k == 0 ? a0 : a1) > 0 && (piece_stage[2 * l + k] < 0 || piece_stage[2 * l + k] >= h->n_stages))
+        return fail(h, LP_ERR_INVALID_ARG, "piece stage outside [0, n_stages)");
+  }
+  for (int l = 0; l < nL; ++l) {
+    Layer& y = h->L[l];
+    y.split_col = 0;
+    const long long a0 = piece_amount[2 * l], a1 = piece_amount[2 * l + 1];
+    if (split_col_out) split_col_out[l] = 0;
+    if (l == 0 || a0 == 0 || a1 == 0) continue;        // no delta task, or placed whole
+    // The pieces are column ranges of whole tiles: kernels with a single column tile (the halo-tile
+    // kernel, narrow layers) and split-K launches (their partial-tile scratch is indexed by the
+    // tile number of the whole contraction) keep the contraction in one piece.
+    const int wd = y.bn_d == GEMM_BN_PAIR ? 256 : y.bn_d;
+    if (y.halo_d || y.split_d > 1 || y.n_in <= wd) continue;
+    const int tiles = (y.n_in + wd - 1) / wd;
+    long long t0 = (tiles * a0 + (a0 + a1) / 2) / (a0 + a1);        // nearest whole number of tiles for delta''
+    t0 = std::max<long long>(1, std::min<long long>(tiles - 1, t0));
+    y.split_col = int(t0) * wd;
+    y.piece_stage[0] = piece_stage[2 * l];
+    y.piece_stage[1] = piece_stage[2 * l + 1];
+    if (split_col_out) split_col_out[l] = y.split_col;
+  }
+  return LP_OK;
+}
+
 extern "C" int lp_reset_task_times(lp_handle h) {
   if (!h) return LP_ERR_INVALID_ARG;
   LP_CUDA(h, cudaDeviceSynchronize());
   for (auto& v : h->timed) v.clear();
+  for (auto& v : h->timed_layer) v.clear();
   h->tpool_next = 0;
   return LP_OK;
 }
@@ -1082,15 +1145,41 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     if (fusedB) {
       cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
       LP_CUDA(c, task_begin(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}));
-      if (l > 0) LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+      if (l > 0 && y.split_col > 0) {      // (one serial task: the pieces follow one another)
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], st, 0));
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], st, 1));
+      } else if (l > 0) {
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+      }
       LP_CUDA(c, launch_G(c, l, n, st));
       LP_CUDA(c, launch_update(c, l, n, st));
       LP_CUDA(c, task_end(c, st, {rdl, rw, rx, raux, ridx}, {rdprev, &y.rDW, rnew}, &y.last_update));
     } else {
-      if (l > 0) {
+      if (l > 0 && y.split_col > 0 && !serial) {
+        // delta'' on the streams of the stage that holds layer l+1, delta' on this layer's own:
+        // two kernels over disjoint column ranges of delta^{l-1}, concurrent; the buffer counts as
+        // written when both are done (the second stream joins the first before the event that
+        // later tasks wait on)
+        cudaStream_t s0 = c->sD[y.piece_stage[0] % c->n_groups], s1 = c->sD[y.piece_stage[1] % c->n_groups];
+        LP_CUDA(c, task_begin(c, s0, {rdl, rw, raux, ridx}, {rdprev}));
+        LP_CUDA(c, task_begin(c, s1, {rdl, rw, raux, ridx}, {rdprev}));
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], s0, 0));
+        LP_CUDA(c, launch_delta(c, l, n, slot[l], s1, 1));
+        if (s0 != s1) {
+          cudaEvent_t e = c->pool[c->pool_next++ % c->pool.size()];
+          LP_CUDA(c, cudaEventRecord(e, s0));
+          LP_CUDA(c, cudaStreamWaitEvent(s1, e, 0));
+        }
+        LP_CUDA(c, task_end(c, s1, {rdl, rw, raux, ridx}, {rdprev}, nullptr));
+      } else if (l > 0) {
         cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
         LP_CUDA(c, task_begin(c, st, {rdl, rw, raux, ridx}, {rdprev}));
-        LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+        if (y.split_col > 0) {
+          LP_CUDA(c, launch_delta(c, l, n, slot[l], st, 0));
+          LP_CUDA(c, launch_delta(c, l, n, slot[l], st, 1));
+        } else {
+          LP_CUDA(c, launch_delta(c, l, n, slot[l], st));
+        }
         LP_CUDA(c, task_end(c, st, {rdl, rw, raux, ridx}, {rdprev}, nullptr));
       }
       cudaStream_t sg = (serial ? user : c->sG[y.stage % c->n_groups]);
@@ -1355,7 +1444,12 @@ extern "C" int lp_debug_run_task(lp_handle h, int task, int layer, long long ste
     }
     case LP_TASK_DELTA:
       if (layer < 1) return fail(h, LP_ERR_INVALID_ARG, "the first layer has no delta task");
-      LP_CUDA(h, launch_delta(h, layer, step, slot, st));
+      if (h->L[layer].split_col > 0) {
+        LP_CUDA(h, launch_delta(h, layer, step, slot, st, 0));
+        LP_CUDA(h, launch_delta(h, layer, step, slot, st, 1));
+      } else {
+        LP_CUDA(h, launch_delta(h, layer, step, slot, st));
+      }
       break;
     case LP_TASK_G: LP_CUDA(h, launch_G(h, layer, step, st)); break;
     case LP_TASK_UPDATE: LP_CUDA(h, launch_update(h, layer, step, st)); break;

@@ -120,7 +120,7 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
             if bias:
                 assert rel_l2(tr.debug_read("master_b", l, 0), orc.b[l]) < 1e-5
             if mu != 0.0:
-                assert rel_l2(tr.debug_read("mom_w", l, 0), orc.mW[l]) < 1e-6
+                assert rel_l2(tr.debug_read("mom_w", l, 0), orc.mW[l]) < 1e-6 + 1e-7 * np.sqrt(k_g)   # m = mu m + G carries G's accumulation error
             new_slot = (n + 1) % (delays[l] + 1)
             Wq, bq = orc.stash[l][n + 1]
             note("ring", assert_bf16_close(tr.debug_read("ring_w", l, new_slot), Wq, "ring W^%d step %d" % (l, n),
