@@ -404,6 +404,57 @@ def short_measure(torch, lpb, name, dev, stream, peaks, seconds=0.6):
     return out
 
 
+def borrowing_report(torch, lpb, w, args, stream):
+    """Section III-B executed and measured.  Algorithm 1's step 2 (`profile`): per-layer task times
+    from a pass with every task alone on the GPU; T_fix = forward + G + update, T_flex = delta, in
+    nanoseconds, go through lp_plan_costs.  Four variants of the LayerPipe schedule are timed: the
+    default plan (integer MAC model) and the plan from measured times, each with the delta
+    contractions in one piece and divided into delta'' / delta' as the plan says."""
+    wl, L = w.wl, len(w.layers)
+    trp = w.trainer(lpb, lpb.LP_SCHED_LAYERPIPE, lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS)
+    _, delays, _ = trp.get_schedule()
+    for k in range(max(delays) + 4):
+        trp.step(w.xs[k % w.P], w.ys[k % w.P])
+    trp.flush()
+    torch.cuda.synchronize()
+    trp.reset_task_times()
+    nprof = max(2, min(8, 32768 // (6 * L)))
+    timed_block(torch, trp, w.xs, w.ys, nprof, stream)
+    fix, flex = [], []
+    for l in range(L):
+        t = {k: trp.layer_task_time(k, l)[1] / nprof for k in ("forward", "G", "update", "delta")}
+        fix.append(max(1, int(1e6 * (t["forward"] + t["G"] + t["update"]))))
+        flex.append(int(1e6 * t["delta"]))
+    trp.close()
+    del trp
+    torch.cuda.empty_cache()
+    plans = {"mac_model": lpb.lp_plan(w.layers, w.B, wl["stages"]), "measured": lpb.lp_plan_costs(fix, flex, wl["stages"])}
+    out = {"profile_ns": {"T_fix": fix, "T_flex": flex}, "variants": {}}
+    steps = args.steps
+    for pname, plan in plans.items():
+        for split in (False, True):
+            tr = lpb.Trainer(w.layers, w.B, wl["stages"], stage=plan["stage"], delays=wl["delays"] if pname == "mac_model" else None,
+                             lr=wl["lr"], momentum=wl["momentum"], schedule=lpb.LP_SCHED_LAYERPIPE, W0=w.W0, b0=w.b0, device=w.dev)
+            cols = tr.set_delta_split(plan["piece_stage"], plan["piece_amount"]) if split else None
+            _, d, _ = tr.get_schedule()
+            for k in range(max(d) + 6):
+                tr.step(w.xs[k % w.P], w.ys[k % w.P])
+            tr.flush()
+            torch.cuda.synchronize()
+            ts = repeat_blocks(lambda: timed_block(torch, tr, w.xs, w.ys, steps, stream), 0.5)
+            rc, detail = tr.device_status()
+            tr.close()
+            del tr
+            torch.cuda.empty_cache()
+            if rc != 0:
+                raise SystemExit("device status %d (%d)" % (rc, detail))
+            sm = summarize(ts, steps)
+            out["variants"]["%s%s" % (pname, "+split" if split else "")] = {
+                "samples_per_s": w.B / (sm["ms_per_step"] * 1e-3), "ms_per_step": sm["ms_per_step"], "stage": plan["stage"],
+                "delays": d, "stages_used": plan["used"], "split_col": cols}
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2108_06629_b200 import binding as lpb
@@ -485,6 +536,7 @@ def run_ours(args):
         for kind in kinds:
             kinds[kind]["avg_us_overlapped"] = kinds_live[kind]["avg_us"]
         roof, wm = roofline(args.workload, wl, kinds, peaks)
+        borrowing = borrowing_report(torch, lpb, w, args, stream) if world == 1 else None
         del w
         torch.cuda.empty_cache()
         per_workload = {}
@@ -516,6 +568,7 @@ def run_ours(args):
             "other_schedule": other,
             "speedup_vs_fused_b": ((value / world) / other["value"] if other["schedule"] == "fused_b"
                                    else other["value"] / (value / world)),
+            "borrowing": borrowing,
             "per_workload": per_workload,
             "cpu_baseline": cpu,
         }

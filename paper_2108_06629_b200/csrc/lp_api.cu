@@ -41,6 +41,8 @@ static inline int pad8(int x) { return (x + 7) & ~7; }
 struct Ev {
   cudaEvent_t e = nullptr;
   cudaStream_t s = nullptr;
+  int si = -1;             // index of the stream it was recorded on (see lp_ctx::stream_index)
+  long long seq = 0;       // position in the handle's sequence of recorded events
 };
 
 struct Res {                 // one buffer (or ring slot) the tracker protects
@@ -129,8 +131,23 @@ struct lp_ctx {
   std::vector<lp::Res> rZL, rLabels;
   // streams / events
   std::vector<cudaStream_t> sF, sD, sG;
+  // Events of the hazard tracker.  A handle stored in a Res must stay valid until that buffer's next
+  // write, at most max(x_slots) minibatches later, so the pool holds more events than that many
+  // minibatches can record; joins that nothing stores (lp_flush, the two pieces of a split delta)
+  // take theirs from a small pool of their own.
   std::vector<cudaEvent_t> pool;
   size_t pool_next = 0;
+  std::vector<cudaEvent_t> jpool;
+  size_t jpool_next = 0;
+  long long ev_seq = 0;
+  // waited[a][b]: the latest event (by sequence number) of stream b that stream a already waits for.
+  // Events of one stream complete in order, so waiting for an earlier one again is redundant.
+  std::vector<cudaStream_t> streams;          // index 0 = the caller's stream of the current lp_step
+  std::vector<std::vector<long long>> waited;
+  int stream_index(cudaStream_t s) const {
+    for (size_t i = 1; i < streams.size(); ++i) if (streams[i] == s) return int(i);
+    return 0;
+  }
   std::vector<lp::Ev> loss_ev;
   // bookkeeping
   long long n_steps = 0;
@@ -394,23 +411,26 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
 
 // ---------------------------------------------------------------------------
 // hazard tracker
-static void wait_on(lp_ctx* c, cudaStream_t s, const Ev& e, std::vector<cudaEvent_t>* seen, cudaError_t* err) {
+static inline void wait_on(lp_ctx* c, cudaStream_t s, int si, const Ev& e, cudaError_t* err) {
   if (!e.e || e.s == s) return;
-  for (cudaEvent_t x : *seen) if (x == e.e) return;
-  seen->push_back(e.e);
+  if (e.si > 0) {                         // (index 0 is whatever stream the caller passes: never pruned)
+    long long& w = c->waited[si][e.si];
+    if (w >= e.seq) return;               // this stream already waits for that event or a later one of its stream
+    w = e.seq;
+  }
   cudaError_t r = cudaStreamWaitEvent(s, e.e, 0);
   if (r != cudaSuccess && *err == cudaSuccess) *err = r;
 }
 
 static cudaError_t task_begin(lp_ctx* c, cudaStream_t s, std::initializer_list<Res*> reads,
                               std::initializer_list<Res*> writes) {
-  std::vector<cudaEvent_t> seen;
   cudaError_t err = cudaSuccess;
-  for (Res* r : reads) if (r) wait_on(c, s, r->last_write, &seen, &err);
+  const int si = c->stream_index(s);
+  for (Res* r : reads) if (r) wait_on(c, s, si, r->last_write, &err);
   for (Res* w : writes) {
     if (!w) continue;
-    wait_on(c, s, w->last_write, &seen, &err);
-    for (const Ev& e : w->readers) wait_on(c, s, e, &seen, &err);
+    wait_on(c, s, si, w->last_write, &err);
+    for (const Ev& e : w->readers) wait_on(c, s, si, e, &err);
   }
   return err;
 }
@@ -419,7 +439,7 @@ static cudaError_t task_end(lp_ctx* c, cudaStream_t s, std::initializer_list<Res
                             std::initializer_list<Res*> writes, Ev* out_ev) {
   cudaEvent_t e = c->pool[c->pool_next++ % c->pool.size()];
   cudaError_t r = cudaEventRecord(e, s);
-  Ev ev{e, s};
+  Ev ev{e, s, c->stream_index(s), ++c->ev_seq};
   for (Res* x : reads) if (x) x->readers.push_back(ev);
   for (Res* w : writes) {
     if (!w) continue;
@@ -558,6 +578,7 @@ static void destroy_ctx(lp_ctx* c) {
   kill(c->sD);
   kill(c->sG);
   for (cudaEvent_t e : c->pool) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->jpool) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->tpool) if (e) cudaEventDestroy(e);
   delete c;
 }
@@ -901,6 +922,7 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   int conn = 8;
   if (const char* e = getenv("CUDA_DEVICE_MAX_CONNECTIONS")) conn = std::max(1, std::min(32, atoi(e)));
   c->n_groups = std::max(1, std::min(used, (conn - 2) / 3));
+  if (const char* e = getenv("LP_STREAM_TRIPLES")) c->n_groups = std::max(1, std::min(c->n_groups, atoi(e)));   // experiments: fewer triples
   c->sF.assign(c->n_groups, nullptr);
   c->sD.assign(c->n_groups, nullptr);
   c->sG.assign(c->n_groups, nullptr);
@@ -909,8 +931,20 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
     LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sD[s], cudaStreamNonBlocking, pD));
     LP_CUDA(nullptr, cudaStreamCreateWithPriority(&c->sG[s], cudaStreamNonBlocking, pG));
   }
-  c->pool.assign(kEventPool, nullptr);
+  {
+    int max_delay = 0;
+    for (int d : dl) max_delay = std::max(max_delay, d);
+    const size_t per_step = size_t(5) * n_layers + 8;                  // tasks of one minibatch, with room to spare
+    const size_t want = std::max<size_t>(kEventPool, (size_t(max_delay) + 4) * per_step);
+    if (want > (size_t(1) << 20)) return fail(nullptr, LP_ERR_UNSUPPORTED, "delays x layers need more than 2^20 scheduler events");
+    c->pool.assign(want, nullptr);
+  }
   for (auto& e : c->pool) LP_CUDA(nullptr, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  c->jpool.assign(64, nullptr);
+  for (auto& e : c->jpool) LP_CUDA(nullptr, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  c->streams.assign(1, nullptr);
+  for (int s = 0; s < c->n_groups; ++s) { c->streams.push_back(c->sF[s]); c->streams.push_back(c->sD[s]); c->streams.push_back(c->sG[s]); }
+  c->waited.assign(c->streams.size(), std::vector<long long>(c->streams.size(), 0));
   if (cfg->flags & LP_TIME_TASKS) {
     c->tpool.assign(2 * 32768, nullptr);
     for (auto& e : c->tpool) LP_CUDA(nullptr, cudaEventCreate(&e));
@@ -1070,6 +1104,10 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   const bool fusedB = (c->cfg.schedule == LP_SCHED_FUSED_B);
   const bool serial = (c->cfg.flags & LP_SERIAL_TASKS) != 0;   // every task on the caller's stream
   const int ds = int(n % kDeltaSlots);
+  if (c->streams[0] != user) {            // what the previous caller's stream waited for says nothing about this one
+    c->streams[0] = user;
+    std::fill(c->waited[0].begin(), c->waited[0].end(), 0ll);
+  }
 
   // version bookkeeping (the integers the parity tests compare bit-exactly)
   std::vector<int> slot(nL);
@@ -1166,7 +1204,7 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
         LP_CUDA(c, launch_delta(c, l, n, slot[l], s0, 0));
         LP_CUDA(c, launch_delta(c, l, n, slot[l], s1, 1));
         if (s0 != s1) {
-          cudaEvent_t e = c->pool[c->pool_next++ % c->pool.size()];
+          cudaEvent_t e = c->jpool[c->jpool_next++ % c->jpool.size()];
           LP_CUDA(c, cudaEventRecord(e, s0));
           LP_CUDA(c, cudaStreamWaitEvent(s1, e, 0));
         }
@@ -1210,7 +1248,7 @@ extern "C" int lp_flush(lp_handle h, void* stream) {
   cudaStream_t user = static_cast<cudaStream_t>(stream);
   auto join = [&](std::vector<cudaStream_t>& v) -> cudaError_t {
     for (cudaStream_t s : v) {
-      cudaEvent_t e = h->pool[h->pool_next++ % h->pool.size()];
+      cudaEvent_t e = h->jpool[h->jpool_next++ % h->jpool.size()];
       cudaError_t r = cudaEventRecord(e, s);
       if (r != cudaSuccess) return r;
       r = cudaStreamWaitEvent(user, e, 0);

@@ -73,8 +73,22 @@ def run_teacher_forced(layers, batch, stages, delays, lr, mu, steps, check_steps
                 if layers[l]["act"] == "gelu":
                     note("z", assert_bf16_close(tr.debug_read("z", l, n), rec["zs"][l], "z^%d step %d" % (l, n), k_terms=k_fwd(l)))
             else:
-                r = rel_l2(tr.debug_read("logits", 0, n), rec["zL"])
-                assert r < 1e-5 + 1e-7 * np.sqrt(k_fwd(l)), ("logits", n, r)      # fp32 accumulation over k_fwd terms on both sides
+                got_zL = tr.debug_read("logits", 0, n)
+                r = rel_l2(got_zL, rec["zL"])
+                if r >= 1e-5 + 1e-7 * np.sqrt(k_fwd(l)):      # fp32 accumulation over k_fwd terms on both sides
+                    # A very long contraction with few outputs (one 224 x 224 image: 200704 terms, 10 logits): the
+                    # outputs are small against the sum of the magnitudes of their terms, and the fp32 oracle's own
+                    # accumulation error shows.  Judge both against float64 on the same operands, with the
+                    # random-walk forward-error bound 4 eps sqrt(K) |a| |W|^T.
+                    a64 = np.asarray(rec["a"][l], dtype=np.float64).reshape(batch, -1)
+                    Wv, bv = stash[l][rec["v"][l]]
+                    W64 = np.asarray(Wv, dtype=np.float64).reshape(layers[l]["n_out"], -1)
+                    ref = a64 @ W64.T + (0.0 if bv is None else np.asarray(bv, dtype=np.float64))
+                    bound = 4.0 * 2.0 ** -24 * np.sqrt(k_fwd(l)) * np.linalg.norm(np.abs(a64) @ np.abs(W64).T)
+                    err_gpu = np.linalg.norm(got_zL.reshape(ref.shape) - ref)
+                    err_orc = np.linalg.norm(np.asarray(rec["zL"], dtype=np.float64).reshape(ref.shape) - ref)
+                    assert err_gpu <= bound, ("logits against float64", n, err_gpu, bound, err_orc)
+                    r = err_gpu / np.linalg.norm(ref)
                 note("logits", r)
         # loss task
         tr.debug_write("logits", 0, n, rec["zL"])
