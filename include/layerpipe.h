@@ -53,8 +53,16 @@ enum { LP_CAPTURE_GRADS = 1u, /* keep G of the latest step readable by lp_get_gr
        LP_UNFUSED_UPDATE = 4u, /* write G to memory and run Eq. 6 as a separate kernel. Default:  */
                                /* the update is fused into the epilogue of the G contraction and  */
                                /* G is only stored when LP_CAPTURE_GRADS is set                    */
-       LP_SERIAL_TASKS = 8u };  /* measurement aid: enqueue every task on the caller's stream, so  */
+       LP_SERIAL_TASKS = 8u,   /* measurement aid: enqueue every task on the caller's stream, so  */
                                /* that no two kernels overlap and LP_TIME_TASKS times each alone  */
+       LP_RECOMPUTE = 16u };   /* activation recomputation instead of stashing, see below         */
+/* LP_RECOMPUTE (Section III-A names both stashing and recomputation as what the delays between a and
+ * the backward pass may stand for): a layer whose input is produced inside its own stage, and whose
+ * delay would need a stash of more than four minibatches, keeps that input (with the stored z and
+ * the pooling positions that go with it) only until the next layer has read it; when the backward
+ * pass of the minibatch reaches the stage, the producing forward task runs again on the stashed
+ * weight version.  One more forward contraction per such layer buys (d_l - 2) x batch x features
+ * x 2 bytes of stash.  The results are bit-identical to the stashing run. */
 
 /* One layer of the chain (Eqs. 1-2: z = W a (+ b), a = f(z)). */
 typedef struct {

@@ -24,6 +24,7 @@ LP_CAPTURE_GRADS = 1
 LP_TIME_TASKS = 2
 LP_UNFUSED_UPDATE = 4
 LP_SERIAL_TASKS = 8
+LP_RECOMPUTE = 16
 
 
 class lp_layer(C.Structure):
@@ -246,9 +247,11 @@ class Trainer:
         B = self.batch
         if l["kind"] == "conv":
             H, W = l["H"], l["W"]
-            Hp, Wp = (H // 2, W // 2) if l.get("pool", 0) else (H, W)
+            Ho = (H + 2 * l["pad"] - l["R"]) // l["stride"] + 1          # delta^l lives on the layer's output grid
+            Wo = (W + 2 * l["pad"] - l["S"]) // l["stride"] + 1
+            Hp, Wp = (Ho // 2, Wo // 2) if l.get("pool", 0) else (Ho, Wo)
             wshape = (l["n_out"], l["R"], l["S"], l["n_in"])
-            shapes = {"input": (B, H, W, l["n_in"]), "delta": (B, H, W, l["n_out"]),
+            shapes = {"input": (B, H, W, l["n_in"]), "delta": (B, Ho, Wo, l["n_out"]),
                       "pool_idx": (B, Hp, Wp, l["n_out"])}
         else:
             wshape = (l["n_out"], l["n_in"])

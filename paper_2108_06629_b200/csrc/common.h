@@ -24,7 +24,7 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64
                       uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer, std::string* err);
 
 int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
-                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err);
+                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err, uint32_t step = 1);
 
 // fp32 (elem_bytes 4) or bf16 (2) row-major tensor moved in boxes of 32 columns x box_outer rows
 // (the streamed tiles of the fused update).

@@ -88,17 +88,19 @@ int make_tmap_rows32(CUtensorMap* out, const void* base, int elem_bytes, uint64_
 // NHWC bf16 tensor [N][H][W][C] with channel pitch `pitch_c` (multiple of 8): dimensions
 // (C, W, H, N), box (64 channels, bw, bh, bn pixels).  Coordinates outside the tensor read zero.
 int make_tmap_bf16_nhwc(CUtensorMap* out, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
-                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err) {
+                        uint64_t pitch_c, uint32_t bw, uint32_t bh, uint32_t bn, std::string* err, uint32_t step) {
   EncodeTiledFn fn = get_encode_fn(err);
   if (!fn) return LP_ERR_CUDA;
-  if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch_c & 7) || bw > 256 || bh > 256 || bn > 256) {
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch_c & 7) || step < 1 || bw * step > 256 || bh * step > 256 || bn > 256) {
     if (err) *err = "tensor map: base must be 16-byte aligned, channel pitch a multiple of 8, box <= 256";
     return LP_ERR_INVALID_ARG;
   }
+  // step > 1: the box takes every step-th pixel in w and h (a strided convolution's input seen from a
+  // box of its output pixels): the traversed extent is bw * step, of which ceil(. / step) = bw are loaded
   cuuint64_t dims[4] = {C, W, H, N};
   cuuint64_t strides[3] = {pitch_c * 2, W * pitch_c * 2, H * W * pitch_c * 2};
-  cuuint32_t box[4] = {64, bw, bh, bn};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
+  cuuint32_t box[4] = {64, bw * step, bh * step, bn};
+  cuuint32_t estr[4] = {1, step, step, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -46,14 +46,24 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
 enum { GEOM_PLAIN = 0, GEOM_PIX_M = 1, GEOM_PIX_K = 2 };
 struct ConvGeom {
   int kind;
-  int H, W;              // image size of the pixel tensor
+  int H, W;              // PIX_M: size of the tensor the tile rows index (the output of the contraction);
+                         // PIX_K: size of the pixel grid the contraction runs over (the layer's output grid)
   int lw, lh;            // log2 of the box width / height; images per box = box pixels >> (lw + lh)
-  int tiles_w, tiles_h;  // boxes per image row / column
-  int S, pad;            // filter width (taps = R*S, tap = r*S + s) and padding
-  int flip;              // 0: pixel shift = tap - pad (forward, G); 1: pad - tap (delta)
+  int tiles_w, tiles_h;  // boxes per row / column of the grid the boxes tile
+  int S, pad;            // filter width (tap = r*S + s) and padding
+  int flip;              // 0: forward / G (input pixel = output pixel * stride + tap - pad); 1: delta
   int chunks_per_tap;    // PIX_M: 64-channel chunks of the A tensor per tap
   int tap_pitch;         // elements between taps inside a row of the weight matrix (padded Cin)
   int n_per_tap;         // PIX_K: column tiles per tap
+  // General filters and strides.  stride: the convolution's stride (forward and G fetch the input
+  // through a tensor map that steps `stride` pixels; start coordinate = box origin * stride + shift).
+  // Delta of a strided layer runs once per residue class (roff_h, roff_w) of the input pixel
+  // modulo the stride: the tile rows are the pixels (h*rs + roff_h, w*rs + roff_w) of the H x W
+  // tensor, rs = stride, and only the taps r = tap_r0 + tap_step*i, s = tap_s0 + tap_step*j
+  // (j < tap_ns) reach such a pixel, from delta pixel (h + (roff_h + pad - r)/stride, ...).
+  int stride;            // >= 1
+  int rs, roff_h, roff_w;
+  int tap_r0, tap_s0, tap_step, tap_ns;   // enumeration of the taps of this launch: k-th tap = (r0 + step*(k / ns), s0 + step*(k % ns))
 };
 
 struct GemmArgs {
@@ -136,11 +146,11 @@ __device__ __forceinline__ int tile_row(const GemmArgs& p, const TileMap& t, int
     const int row = t.m0 + tr;
     return row < p.M ? row : -1;
   }
+  // (pixel boxes tile their grid exactly: every row of a tile exists)
   const int w = t.pw0 + (tr & ((1 << p.g.lw) - 1));
   const int h = t.ph0 + ((tr >> p.g.lw) & ((1 << p.g.lh) - 1));
   const int n = t.pn0 + (tr >> (p.g.lw + p.g.lh));
-  const int row = (n * p.g.H + h) * p.g.W + w;
-  return row < p.M ? row : -1;
+  return (n * p.g.H + h * p.g.rs + p.g.roff_h) * p.g.W + w * p.g.rs + p.g.roff_w;
 }
 
 // Bias of four consecutive output columns (zero where there is none).
@@ -574,16 +584,23 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             k0 += GEMM_BK;
           } else if (p.g.kind == GEOM_PIX_M) {
             // A: 128 pixels x 64 channels of the activation / delta tensor, shifted by the tap
-            const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
-            const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
-            const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;
-            tma_load_4d_addr(sa, &tmA, fb, c_chunk * 64, tm.pw0 + sw, tm.ph0 + sh, tm.pn0);
+            const int r = p.g.tap_r0 + p.g.tap_step * (c_tap / p.g.tap_ns), sft = p.g.tap_s0 + p.g.tap_step * (c_tap % p.g.tap_ns);
+            const int wtap = r * p.g.S + sft;         // position of this tap in a row of the weight matrix
+            int cw, ch;
+            if (p.g.flip) {   // delta: output pixel of the layer that reaches this input pixel through tap (r, s)
+              cw = tm.pw0 + (p.g.roff_w + p.g.pad - sft) / p.g.stride;
+              ch = tm.ph0 + (p.g.roff_h + p.g.pad - r) / p.g.stride;
+            } else {          // forward: first input pixel of the box (the map steps `stride` pixels per element)
+              cw = tm.pw0 * p.g.stride + sft - p.g.pad;
+              ch = tm.ph0 * p.g.stride + r - p.g.pad;
+            }
+            tma_load_4d_addr(sa, &tmA, fb, c_chunk * 64, cw, ch, tm.pn0);
             if (B_MN) {   // delta: B[k = (tap, co)][n = ci]: rows co, columns tap*pitch + ci
 #pragma unroll
               for (int c = 0; c < BN / 64; ++c)
-                tma_load_2d_addr(sb + c * 8192, &tmB, fb, c_tap * p.g.tap_pitch + tm.n0 + c * 64, c_chunk * 64);
+                tma_load_2d_addr(sb + c * 8192, &tmB, fb, wtap * p.g.tap_pitch + tm.n0 + c * 64, c_chunk * 64);
             } else {      // forward: B[n = co][k = (tap, ci)]
-              tma_load_2d_addr(sb, &tmB, fb, c_tap * p.g.tap_pitch + c_chunk * 64, tm.n0);
+              tma_load_2d_addr(sb, &tmB, fb, wtap * p.g.tap_pitch + c_chunk * 64, tm.n0);
             }
             if (++c_chunk == p.g.chunks_per_tap) { c_chunk = 0; ++c_tap; }
           } else {
@@ -591,7 +608,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_4d_addr(sa + c * 8192, &tmA, fb, tm.m0 + c * 64, bw0, bh0, bn0);
 #pragma unroll
-            for (int c = 0; c < BN / 64; ++c) tma_load_4d_addr(sb + c * 8192, &tmB, fb, tc.col0 + c * 64, bw0 + dw, bh0 + dh, bn0);
+            for (int c = 0; c < BN / 64; ++c)
+              tma_load_4d_addr(sb + c * 8192, &tmB, fb, tc.col0 + c * 64, bw0 * p.g.stride + dw, bh0 * p.g.stride + dh, bn0);
             bw0 += 1 << p.g.lw;
             if (bw0 >= p.g.W) {
               bw0 = 0;

@@ -169,6 +169,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t fb = map_to_cta(full0 + 8u * s, 0);          // the leader's barrier
         if (rank == 0) mbar_arrive_expect_tx_addr(full0 + 8u * s, 2 * STAGE_BYTES);
         if (pix) {
+          // (this kernel serves stride-1 layers: the tap's shift is the whole coordinate arithmetic)
           const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
           const int sh = p.g.flip ? p.g.pad - r : r - p.g.pad;
           const int sw = p.g.flip ? p.g.pad - sft : sft - p.g.pad;

@@ -62,7 +62,11 @@ struct Layer {
   // geometry.  FC: H = W = 1, in_rows = out_rows = B.  Conv (3x3, stride 1, pad 1): in_rows =
   // out_rows = B*H*W; weights are the matrix [Cout][9 * ld_in] (tap-major, padded channels).
   bool conv = false;
-  int imH = 1, imW = 1, taps = 1;
+  int imH = 1, imW = 1, taps = 1;   // conv: INPUT image size; taps = R * S
+  int oH = 1, oW = 1;               // conv: OUTPUT image size (before pooling)
+  int cR = 1, cS = 1, cstride = 1, cpad = 0;
+  bool gen = false;                 // a filter other than 3x3 / stride 1 / pad 1: general implicit-GEMM path only
+  PixBox boxD;                      // delta of a strided layer: boxes of 128 pixels over one residue class of the input grid
   // First convolution layer with few input channels (9 * Cin <= 64): the stash holds 3x3 patches
   // [B*H*W][9 * Cin] and the layer runs as a plain GEMM over pixel rows; n_in = 9 * Cin, taps = 1,
   // c_in = the image's channel count.
@@ -110,7 +114,17 @@ struct Layer {
   // and delta' = columns [split_col, n_in), run on piece_stage[1].  split_col = 0: one piece.
   int split_col = 0;
   int piece_stage[2] = {0, 0};
+  // Activation recomputation (LP_RECOMPUTE): this layer's INPUT a^{l-1} (with the stored z^{l-1} and the
+  // pooling positions that go with it) is not stashed for d_l + 2 minibatches.  The forward pass
+  // keeps it in two short-lived slots (0, 1); when the backward pass of minibatch n reaches the
+  // layer's stage, the forward task of layer l-1 is run again, with the same stashed weight
+  // version, into slots 2 + n % 2, which is what G_l(n) and the f' multiply read.
+  bool recomp = false;
 };
+// slot of layer y's input stash (and of what is stored with it) used by the forward pass / by the
+// backward pass of minibatch n
+static inline int xf_slot(const Layer& y, long long n) { return y.recomp ? int(n & 1) : int(n % y.x_slots); }
+static inline int xb_slot(const Layer& y, long long n) { return y.recomp ? 2 + int(n & 1) : int(n % y.x_slots); }
 
 }  // namespace lp
 
@@ -210,20 +224,27 @@ static int validate(const lp_layer* layers, int n, const lp_config* cfg, std::st
     if (y.act < LP_ACT_NONE || y.act > LP_ACT_GELU) { *why = "unknown activation"; return LP_ERR_INVALID_ARG; }
     if (l == n - 1 && y.act != LP_ACT_NONE) { *why = "last layer must have no activation"; return LP_ERR_INVALID_ARG; }
     if (y.kind == LP_CONV) {
-      if (y.R != 3 || y.S != 3 || y.stride != 1 || y.pad != 1) { *why = "only 3x3 stride-1 pad-1 convolutions are built"; return LP_ERR_UNSUPPORTED; }
+      if (y.R < 1 || y.R > 7 || y.S < 1 || y.S > 7 || y.stride < 1 || y.stride > 2 || y.pad < 0 || y.pad >= y.R || y.pad >= y.S) {
+        *why = "convolutions are built for filters up to 7x7, stride 1 or 2, padding smaller than the filter"; return LP_ERR_UNSUPPORTED;
+      }
       if (y.H < 1 || y.W < 1) { *why = "bad image size"; return LP_ERR_INVALID_ARG; }
+      if (y.H + 2 * y.pad < y.R || y.W + 2 * y.pad < y.S) { *why = "filter larger than the padded image"; return LP_ERR_INVALID_ARG; }
+      if (y.H % y.stride || y.W % y.stride) { *why = "a strided convolution needs an image size divisible by the stride"; return LP_ERR_UNSUPPORTED; }
       if ((long long)cfg->batch * y.H * y.W >= (1ll << 31) / 64) { *why = "batch x image size too large (pixel rows are indexed with 32 bits)"; return LP_ERR_UNSUPPORTED; }
       if (y.act == LP_ACT_GELU) { *why = "GELU after a convolution is not built"; return LP_ERR_UNSUPPORTED; }
       if (y.out % 8 != 0) { *why = "convolution output channels must be a multiple of 8"; return LP_ERR_UNSUPPORTED; }
-      if (y.pool != 0 && (y.pool != 2 || y.H % 2 || y.W % 2 || y.act != LP_ACT_RELU)) { *why = "pooling must be 2x2 on even images after ReLU"; return LP_ERR_UNSUPPORTED; }
+      const int oh = (y.H + 2 * y.pad - y.R) / y.stride + 1, ow = (y.W + 2 * y.pad - y.S) / y.stride + 1;
+      if (y.pool != 0 && (y.pool != 2 || oh % 2 || ow % 2 || y.act != LP_ACT_RELU)) { *why = "pooling must be 2x2 on even images after ReLU"; return LP_ERR_UNSUPPORTED; }
       if (l == n - 1) { *why = "the last layer must be fully connected"; return LP_ERR_UNSUPPORTED; }
-      if (pick_box(y.W, y.H, cfg->batch, 128, nullptr) != LP_OK || pick_box(y.W, y.H, cfg->batch, 64, nullptr) != LP_OK) {
+      if (pick_box(ow, oh, cfg->batch, 128, nullptr) != LP_OK || pick_box(ow, oh, cfg->batch, 64, nullptr) != LP_OK ||
+          pick_box(y.W / y.stride, y.H / y.stride, cfg->batch, 128, nullptr) != LP_OK) {
         *why = "image size / batch cannot be tiled into boxes of 128 and 64 pixels"; return LP_ERR_UNSUPPORTED;
       }
     } else if (y.pool != 0) { *why = "pooling needs a convolution layer"; return LP_ERR_INVALID_ARG; }
     if (l > 0) {
       const lp_layer& pv = layers[l - 1];
-      const int ph = pv.kind == LP_CONV ? pv.H / (pv.pool ? 2 : 1) : 1, pw = pv.kind == LP_CONV ? pv.W / (pv.pool ? 2 : 1) : 1;
+      const int ph = pv.kind == LP_CONV ? ((pv.H + 2 * pv.pad - pv.R) / pv.stride + 1) / (pv.pool ? 2 : 1) : 1;
+      const int pw = pv.kind == LP_CONV ? ((pv.W + 2 * pv.pad - pv.S) / pv.stride + 1) / (pv.pool ? 2 : 1) : 1;
       if (y.kind == LP_CONV) {
         if (pv.kind != LP_CONV || pv.out != y.in || ph != y.H || pw != y.W) { *why = "layer sizes do not chain"; return LP_ERR_INVALID_ARG; }
       } else {
@@ -351,19 +372,30 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     y.ld_in = pad8(y.n_in);
     y.ld_out = pad8(y.n_out);
     y.x_slots = y.delay + 1 + kExtraStashSlots;
+    // recomputation pays where the stash would hold more than the four slots it needs instead, and is
+    // possible where the producing layer sits in the same stage (a stage keeps its own input stashed)
+    y.recomp = (c->cfg.flags & LP_RECOMPUTE) != 0 && l > 0 && st[l] == st[l - 1] && y.x_slots > 4;
+    if (y.recomp) y.x_slots = 4;
     const int B = c->cfg.batch;
     y.conv = layers[l].kind == LP_CONV;
     if (y.conv) {
-      y.imH = layers[l].H; y.imW = layers[l].W; y.taps = 9;
-      y.patch = (l == 0 && 9 * y.n_in <= 64);
+      y.imH = layers[l].H; y.imW = layers[l].W;
+      y.cR = layers[l].R; y.cS = layers[l].S; y.cstride = layers[l].stride; y.cpad = layers[l].pad;
+      y.taps = y.cR * y.cS;
+      y.oH = (y.imH + 2 * y.cpad - y.cR) / y.cstride + 1;
+      y.oW = (y.imW + 2 * y.cpad - y.cS) / y.cstride + 1;
+      y.gen = !(y.cR == 3 && y.cS == 3 && y.cstride == 1 && y.cpad == 1);
+      y.patch = (l == 0 && !y.gen && 9 * y.n_in <= 64);
       if (y.patch) { y.c_in = y.n_in; y.n_in = 9 * y.c_in; y.ld_in = pad8(y.n_in); y.taps = 1; }
-      y.in_rows = y.out_rows = B * y.imH * y.imW;
+      y.in_rows = B * y.imH * y.imW;
+      y.out_rows = B * y.oH * y.oW;
       y.w_rows = y.n_out; y.w_ld = y.taps * y.ld_in;
       y.pool = layers[l].pool;
-      y.Hp = y.pool ? y.imH / 2 : y.imH; y.Wp = y.pool ? y.imW / 2 : y.imW;
+      y.Hp = y.pool ? y.oH / 2 : y.oH; y.Wp = y.pool ? y.oW / 2 : y.oW;
       y.next_rows = (l + 1 < n && layers[l + 1].kind == LP_CONV) ? B * y.Hp * y.Wp : B;
-      pick_box(y.imW, y.imH, B, 128, &y.box128);
-      pick_box(y.imW, y.imH, B, 64, &y.box64);
+      pick_box(y.oW, y.oH, B, 128, &y.box128);      // forward: tile rows = output pixels
+      pick_box(y.oW, y.oH, B, 64, &y.box64);        // G: the contraction runs over output pixels
+      pick_box(y.imW / y.cstride, y.imH / y.cstride, B, 128, &y.boxD);   // delta: tile rows = input pixels of one residue class
       y.bn_f = y.n_out <= 64 ? 64 : 128;
       y.bn_d = y.ld_in <= 64 ? 64 : 128;
       y.bn_g = y.ld_in <= 64 ? 64 : 128;
@@ -373,10 +405,10 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       // 256 -> 256 at 56^2 216 / 240 and 230 / 249 us; 512 -> 512 at 14^2 66 / 79 and 67 / 84 us;
       // 128 -> 256 forward (18 k-blocks) is slower as a pair (149 / 131 us) and stays single.
       const bool even_boxes = ((y.in_rows / GEMM_BM) % 2) == 0;
-      if (even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
-      if (even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
+      if (!y.gen && even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
+      if (!y.gen && even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
       y.split_f = y.split_d = 1;
-      const bool tiles_8x16 = (y.imW % 8 == 0) && (y.imH % 16 == 0);
+      const bool tiles_8x16 = !y.gen && (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
       y.halo_d = l > 0 && tiles_8x16 && y.ld_out <= 64 && y.n_in <= 64;
       y.halo_g = y.halo_f;   // (128 output channels in two passes of the G kernel measured slower than the split-K kernel: 182 / 160 us)
@@ -388,7 +420,7 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       // never more splits than fill two CTAs per SM.  Swept on the small VGG (2 .. 148 splits):
       // the measured optimum of every layer is the power of two next to this value.
       const int tiles = ((y.n_out + GEMM_BM - 1) / GEMM_BM) * y.taps * ((y.ld_in + y.bn_g - 1) / y.bn_g);
-      const int num_kb = y.in_rows / GEMM_BK;
+      const int num_kb = y.out_rows / GEMM_BK;
       const int s_opt = int(std::lround(std::sqrt(double(num_kb) * (y.bn_g <= 64 ? 0.6 : 0.3))));
       y.split_g = std::max(1, std::min(std::min(296 / std::max(tiles, 1), s_opt), y.patch ? 148 : 64));
       const int per = (num_kb + y.split_g - 1) / y.split_g;
@@ -470,15 +502,18 @@ static int build_tensor_maps(lp_ctx* c) {
       // delta:   A = delta^l as NHWC boxes of 128 pixels; B = the same W matrix read MN-major
       // G:       A = delta^l, B = a^{l-1}, both as NHWC boxes of 64 pixels (the contraction index)
       for (int s = 0; s < y.x_slots; ++s) {
+        // (the stash is the layer's INPUT image; a box of output pixels reads every stride-th input pixel)
         if ((rc = make_tmap_bf16_nhwc(&y.tm_f_A[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, y.box128.bw,
-                                      y.box128.bh, y.box128.bn, &err)) != LP_OK) return fail(c, rc, err);
+                                      y.box128.bh, y.box128.bn, &err, y.cstride)) != LP_OK) return fail(c, rc, err);
         if ((rc = make_tmap_bf16_nhwc(&y.tm_g_B[s], y.X + s * y.x_elems, y.ld_in, y.imW, y.imH, B, y.ld_in, y.box64.bw,
-                                      y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
+                                      y.box64.bh, y.box64.bn, &err, y.cstride)) != LP_OK) return fail(c, rc, err);
       }
       for (int s = 0; s < kDeltaSlots; ++s) {
-        if ((rc = make_tmap_bf16_nhwc(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
-                                      y.box128.bw, y.box128.bh, y.box128.bn, &err)) != LP_OK) return fail(c, rc, err);
-        if ((rc = make_tmap_bf16_nhwc(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.ld_out, y.imW, y.imH, B, y.ld_out,
+        // (delta^l lives on the layer's OUTPUT grid; the delta contraction walks it in boxes that match one residue class
+        // of the input grid, the G contraction in boxes of 64 output pixels)
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_d_A[s], y.delta + s * y.delta_elems, y.ld_out, y.oW, y.oH, B, y.ld_out,
+                                      y.boxD.bw, y.boxD.bh, y.boxD.bn, &err)) != LP_OK) return fail(c, rc, err);
+        if ((rc = make_tmap_bf16_nhwc(&y.tm_g_A[s], y.delta + s * y.delta_elems, y.ld_out, y.oW, y.oH, B, y.ld_out,
                                       y.box64.bw, y.box64.bh, y.box64.bn, &err)) != LP_OK) return fail(c, rc, err);
       }
       if (y.halo_f || y.halo_g) {      // the halo box over the stashed input (forward and G)
@@ -608,14 +643,19 @@ struct TimedScope {
 static ConvGeom conv_geom(const Layer& y, int kind, const PixBox& bx, int flip, int chunks_per_tap, int n_per_tap) {
   ConvGeom g{};
   g.kind = kind;
-  g.H = y.imH; g.W = y.imW;
+  // PIX_M forward: rows index the output image; PIX_M delta: the input image (delta^{l-1}); PIX_K: the output grid
+  g.H = (kind == GEOM_PIX_M && flip) ? y.imH : y.oH;
+  g.W = (kind == GEOM_PIX_M && flip) ? y.imW : y.oW;
   g.lw = bx.lw; g.lh = bx.lh;
   g.tiles_w = bx.tiles_w; g.tiles_h = bx.tiles_h;
-  g.S = 3; g.pad = 1;
+  g.S = y.cS; g.pad = y.cpad;
   g.flip = flip;
   g.chunks_per_tap = chunks_per_tap;
   g.tap_pitch = y.ld_in;
   g.n_per_tap = n_per_tap;
+  g.stride = y.cstride;
+  g.rs = 1; g.roff_h = g.roff_w = 0;
+  g.tap_r0 = g.tap_s0 = 0; g.tap_step = 1; g.tap_ns = y.cS;      // all R x S taps
   return g;
 }
 
@@ -630,13 +670,21 @@ static ConvGeom halo_geom(const Layer& y, int flip) {
   g.flip = flip;
   g.chunks_per_tap = 1;
   g.tap_pitch = y.ld_in;
+  g.stride = 1;
+  g.rs = 1;
+  g.tap_step = 1; g.tap_ns = 3;
   return g;
 }
 
-static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st) {
+// again = false: the forward pass of minibatch n.  again = true: the same task re-run by the backward
+// pass (activation recomputation): reads the backward-side slot of its input, writes the backward-side
+// slots of the next layer's input, stored z and pooling positions.
+static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, cudaStream_t st, bool again = false) {
   Layer& y = c->L[l];
   const int nL = int(c->L.size());
   const bool last = (l == nL - 1);
+  const int xin = again ? xb_slot(y, n) : xf_slot(y, n);
+  const int xout = last ? 0 : (again ? xb_slot(c->L[l + 1], n) : xf_slot(c->L[l + 1], n));
   GemmArgs a{};
   a.M = y.out_rows; a.N = y.n_out; a.K = y.n_in;
   if (y.conv && !y.patch) {
@@ -658,10 +706,10 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
     a.ld_out = y.ld_out;
   } else {
     Layer& nx = c->L[l + 1];
-    a.out = nx.X + size_t(n % nx.x_slots) * nx.x_elems;
+    a.out = nx.X + size_t(xout) * nx.x_elems;
     a.ld_out = y.ld_out;              // = nx.ld_in for conv -> conv and FC -> FC; a flattened conv output keeps its channel pitch
-    if (y.Z) {
-      a.out2 = y.Z + size_t(n % y.z_slots) * y.z_elems;
+    if (y.Z && (again || !nx.recomp)) {       // (a layer whose output is recomputed stores z only on the second pass)
+      a.out2 = y.Z + size_t(xout) * y.z_elems;
       a.ld_out2 = y.ld_out;
     }
   }
@@ -669,25 +717,26 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   ++c->launches;
   TimedScope ts(c, LP_TASK_FORWARD, st, l);
   if (y.lean_f) {
-    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
-    return conv_halo_launch(0, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], tmo, a, st);
+    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[xout];
+    return conv_halo_launch(0, y.tm_f_A[xin], y.tm_f_B[ring_slot], tmo, a, st);
   }
   if (y.halo_f) {
     a.g = halo_geom(y, 0);
-    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[n % c->L[l + 1].x_slots];
-    return conv_halo_launch(0, y.tm_hf_A[n % y.x_slots], y.tm_f_B[ring_slot], tmo, a, st);
+    const CUtensorMap& tmo = y.pool ? y.tm_hf_O[0] : y.tm_hf_O[xout];
+    return conv_halo_launch(0, y.tm_hf_A[xin], y.tm_f_B[ring_slot], tmo, a, st);
   }
-  return gemm_launch(0, y.bn_f, y.tm_f_A[n % y.x_slots], y.tm_f_B[ring_slot], a, st);
+  return gemm_launch(0, y.bn_f, y.tm_f_A[xin], y.tm_f_B[ring_slot], a, st);
 }
 
 // 2x2 max pool of layer l's activation into the next layer's stash slot (+ argmax)
-static cudaError_t launch_pool(lp_ctx* c, int l, long long n, cudaStream_t st) {
+static cudaError_t launch_pool(lp_ctx* c, int l, long long n, cudaStream_t st, bool again = false) {
   Layer& y = c->L[l];
   Layer& nx = c->L[l + 1];
+  const int xout = again ? xb_slot(nx, n) : xf_slot(nx, n);
   ++c->launches;
   TimedScope ts(c, LP_TASK_FORWARD, st, l);
-  return launch_maxpool2(y.a_full, nx.X + size_t(n % nx.x_slots) * nx.x_elems, y.pidx + size_t(n % nx.x_slots) * y.pidx_elems,
-                         c->cfg.batch, y.imH, y.imW, y.ld_out, st);
+  return launch_maxpool2(y.a_full, nx.X + size_t(xout) * nx.x_elems, y.pidx + size_t(xout) * y.pidx_elems,
+                         c->cfg.batch, y.oH, y.oW, y.ld_out, st);
 }
 
 // piece: -1 = the whole contraction; 0 = delta'' (columns [0, split_col)); 1 = delta' (the rest)
@@ -701,7 +750,7 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
   if (y.conv) {
     const int cpt = (y.ld_out + 63) / 64;
     a.K = y.taps * cpt * GEMM_BK;
-    a.g = conv_geom(y, GEOM_PIX_M, y.box128, 1, cpt, 0);
+    a.g = conv_geom(y, GEOM_PIX_M, y.boxD, 1, cpt, 0);
   }
   a.act = pv.d.act;
   a.out = pv.delta + size_t(n % kDeltaSlots) * pv.delta_elems;
@@ -710,19 +759,19 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
     // the layer below ended in ReLU + max pool: the product lives on the pooled grid and is
     // routed back through the recorded argmax, gated by the pooled activation
     a.mode = EPI_DGRAD_UNPOOL;
-    a.pool_idx = pv.pidx + size_t(n % y.x_slots) * pv.pidx_elems;
+    a.pool_idx = pv.pidx + size_t(xb_slot(y, n)) * pv.pidx_elems;
     a.pool_C = pv.ld_out;
     a.pool_ppr = y.conv ? 1 : pv.Hp * pv.Wp;
     a.pool_Hp = pv.Hp; a.pool_Wp = pv.Wp;
-    a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;
+    a.aux = y.X + size_t(xb_slot(y, n)) * y.x_elems;
     a.ld_aux = pv.ld_out;
   } else {
     a.mode = EPI_DGRAD;
     if (pv.d.act == LP_ACT_GELU) {
-      a.aux = pv.Z + size_t(n % pv.z_slots) * pv.z_elems;   // stored z^{l-1}
+      a.aux = pv.Z + size_t(xb_slot(y, n)) * pv.z_elems;    // stored z^{l-1}
       a.ld_aux = pv.ld_out;
     } else {
-      a.aux = y.X + size_t(n % y.x_slots) * y.x_elems;      // a^{l-1} > 0  <=>  z^{l-1} > 0
+      a.aux = y.X + size_t(xb_slot(y, n)) * y.x_elems;      // a^{l-1} > 0  <=>  z^{l-1} > 0
       a.ld_aux = y.ld_in;
     }
     if (!y.conv && pv.conv) {
@@ -738,6 +787,27 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
   if (y.halo_d) {
     a.g = halo_geom(y, 1);
     return conv_halo_launch(1, y.tm_hd_A[n % kDeltaSlots], y.tm_d_B[ring_slot], y.tm_hd_A[0], a, st);
+  }
+  if (y.conv && y.cstride > 1) {
+    // Strided layer: input pixel (h, w) is reached through tap (r, s) only when h + pad - r and
+    // w + pad - s are multiples of the stride.  One launch per residue class of (h, w) modulo the
+    // stride: its rows are the pixels of that class, its contraction runs over the taps of that
+    // class only -- together the launches do exactly the R * S * Cout multiply-accumulates per
+    // input pixel that exist, and each element of delta^{l-1} is written once.
+    const int sd = y.cstride, cpt = (y.ld_out + 63) / 64;
+    a.M = y.in_rows / (sd * sd);
+    for (int ph = 0; ph < sd; ++ph)
+      for (int pw = 0; pw < sd; ++pw) {
+        const int r0 = (ph + y.cpad) % sd, s0 = (pw + y.cpad) % sd;
+        const int nr = r0 < y.cR ? (y.cR - r0 + sd - 1) / sd : 0, ns = s0 < y.cS ? (y.cS - s0 + sd - 1) / sd : 0;
+        a.g.rs = sd; a.g.roff_h = ph; a.g.roff_w = pw;
+        a.g.tap_r0 = r0; a.g.tap_s0 = s0; a.g.tap_step = sd; a.g.tap_ns = std::max(ns, 1);
+        a.K = nr * ns * cpt * GEMM_BK;        // (a class without taps stores f'(.) x 0: K = 0 runs the epilogue on zeros)
+        if (ph + pw > 0) ++c->launches;
+        cudaError_t e = gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
+        if (e != cudaSuccess) return e;
+      }
+    return cudaSuccess;
   }
   return gemm_launch(1, y.bn_d, y.tm_d_A[n % kDeltaSlots], y.tm_d_B[ring_slot], a, st);
 }
@@ -764,11 +834,11 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
     }
     c->launches += 2 * ((y.n_out + 63) / 64);
     TimedScope ts(c, LP_TASK_G, st, l);
-    return conv_halo_g_launch(y.tm_hf_A[n % y.x_slots], y.tm_hg_D[n % kDeltaSlots], halo_geom(y, 0), c->cfg.batch, y.part_g,
+    return conv_halo_g_launch(y.tm_hf_A[xb_slot(y, n)], y.tm_hg_D[n % kDeltaSlots], halo_geom(y, 0), c->cfg.batch, y.part_g,
                               u, c->status, st);
   }
   GemmArgs a{};
-  a.M = y.n_out; a.N = y.w_ld; a.K = y.in_rows;
+  a.M = y.n_out; a.N = y.w_ld; a.K = y.out_rows;      // the contraction runs over the samples / output pixels (delta^l's rows)
   if (!y.conv || y.patch) a.N = y.n_in;
   a.ld_out = y.w_ld;
   a.status = c->status;
@@ -800,9 +870,9 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
     um.W = y.tm_u_W;
     um.M = y.mW ? y.tm_u_M : y.tm_u_W;
     um.R = y.tm_u_R[(n + 1) % y.slots];
-    return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st, &um);
+    return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[xb_slot(y, n)], a, st, &um);
   }
-  return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[n % y.x_slots], a, st);
+  return gemm_launch(2, y.bn_g, y.tm_g_A[n % kDeltaSlots], y.tm_g_B[xb_slot(y, n)], a, st);
 }
 
 static cudaError_t launch_update(lp_ctx* c, int l, long long n, cudaStream_t st) {
@@ -1140,11 +1210,12 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   for (int l = 0; l < nL; ++l) {
     Layer& y = c->L[l];
     cudaStream_t st = (serial ? user : c->sF[y.stage % c->n_groups]);
-    Res* rin = &y.rX[n % y.x_slots];
+    Res* rin = &y.rX[xf_slot(y, n)];
     Res* rw = &y.rRing[slot[l]];
-    Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[n % c->L[l + 1].x_slots];
-    Res* rz = y.Z ? &y.rZ[n % y.z_slots] : nullptr;
-    Res* rpool = y.pool ? &y.rPidx[n % c->L[l + 1].x_slots] : nullptr;
+    const int xo = (l == nL - 1) ? 0 : xf_slot(c->L[l + 1], n);
+    Res* rout = (l == nL - 1) ? &c->rZL[ds] : &c->L[l + 1].rX[xo];
+    Res* rz = y.Z ? &y.rZ[xo] : nullptr;
+    Res* rpool = y.pool ? &y.rPidx[xo] : nullptr;
     Res* rfull = y.pool ? &y.rAfull : nullptr;
     LP_CUDA(c, task_begin(c, st, {rin, rw}, {rout, rz, rpool, rfull}));
     LP_CUDA(c, launch_forward(c, l, n, slot[l], st));
@@ -1167,9 +1238,33 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
   // ---- backward: delta and G are independent tasks; update follows G -----------
   for (int l = nL - 1; l >= 0; --l) {
     Layer& y = c->L[l];
+    // Activation recomputation: when the backward pass reaches a stage (at its last layer), the
+    // forward tasks that produce the recomputed inputs of its layers run again, first layer first,
+    // each from the stashed (or just recomputed) input of its own layer and the weight version the
+    // forward pass of this minibatch used -- the same kernels on the same operands, hence the same bits.
+    if (l == nL - 1 || c->L[l + 1].stage != y.stage) {
+      int lo = l;
+      while (lo > 0 && c->L[lo - 1].stage == y.stage) --lo;
+      for (int k = lo + 1; k <= l; ++k) {
+        if (!c->L[k].recomp) continue;
+        Layer& src = c->L[k - 1];
+        cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
+        const int xo = xb_slot(c->L[k], n);
+        Res* rin = &src.rX[xb_slot(src, n)];
+        Res* rwv = &src.rRing[slot[k - 1]];
+        Res* rout = &c->L[k].rX[xo];
+        Res* rz = src.Z ? &src.rZ[xo] : nullptr;
+        Res* rpool = src.pool ? &src.rPidx[xo] : nullptr;
+        Res* rfull = src.pool ? &src.rAfull : nullptr;
+        LP_CUDA(c, task_begin(c, st, {rin, rwv}, {rout, rz, rpool, rfull}));
+        LP_CUDA(c, launch_forward(c, k - 1, n, slot[k - 1], st, true));
+        if (src.pool) LP_CUDA(c, launch_pool(c, k - 1, n, st, true));
+        LP_CUDA(c, task_end(c, st, {rin, rwv}, {rout, rz, rpool, rfull}, nullptr));
+      }
+    }
     Res* rdl = &y.rDelta[ds];
     Res* rw = &y.rRing[slot[l]];
-    Res* rx = &y.rX[n % y.x_slots];
+    Res* rx = &y.rX[xb_slot(y, n)];
     Res* rnew = &y.rRing[(n + 1) % y.slots];
     Res* rdprev = nullptr;
     Res* raux = nullptr;
@@ -1177,8 +1272,8 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     if (l > 0) {
       Layer& pv = c->L[l - 1];
       rdprev = &pv.rDelta[ds];
-      raux = (pv.d.act == LP_ACT_GELU) ? &pv.rZ[n % pv.z_slots] : rx;
-      if (pv.pool) ridx = &pv.rPidx[n % y.x_slots];
+      raux = (pv.d.act == LP_ACT_GELU) ? &pv.rZ[xb_slot(y, n)] : rx;
+      if (pv.pool) ridx = &pv.rPidx[xb_slot(y, n)];
     }
     if (fusedB) {
       cudaStream_t st = (serial ? user : c->sD[y.stage % c->n_groups]);
@@ -1309,15 +1404,15 @@ static int locate(lp_ctx* h, int buffer, int layer, long long index, BufView* v)
   Layer& y = h->L[layer];
   const int wr = y.n_out * y.taps;     // weight-shaped buffers as [Cout * taps][Cin] with pitch ld_in
   switch (buffer) {
-    case LP_BUF_INPUT: *v = {y.X + size_t(index % y.x_slots) * y.x_elems, y.in_rows, y.n_in, y.ld_in, 0}; return LP_OK;
+    case LP_BUF_INPUT: *v = {y.X + size_t(xb_slot(y, index)) * y.x_elems, y.in_rows, y.n_in, y.ld_in, 0}; return LP_OK;
     case LP_BUF_Z:
       if (!y.Z) return fail(h, LP_ERR_NOT_READY, "this layer stores no pre-activation");
-      *v = {y.Z + size_t(index % y.z_slots) * y.z_elems, B, y.n_out, y.ld_out, 0};
+      *v = {y.Z + size_t(xb_slot(h->L[layer + 1], index)) * y.z_elems, B, y.n_out, y.ld_out, 0};
       return LP_OK;
     case LP_BUF_DELTA: *v = {y.delta + size_t(index % kDeltaSlots) * y.delta_elems, y.out_rows, y.n_out, y.ld_out, 0}; return LP_OK;
     case LP_BUF_POOL_IDX:
       if (!y.pidx) return fail(h, LP_ERR_NOT_READY, "this layer does not pool");
-      *v = {y.pidx + size_t(index % h->L[layer + 1].x_slots) * y.pidx_elems, B * y.Hp * y.Wp, y.n_out, y.ld_out, 3};
+      *v = {y.pidx + size_t(xb_slot(h->L[layer + 1], index)) * y.pidx_elems, B * y.Hp * y.Wp, y.n_out, y.ld_out, 3};
       return LP_OK;
     case LP_BUF_RING_W:
       if (index >= y.slots) return fail(h, LP_ERR_INVALID_ARG, "ring slot out of range");

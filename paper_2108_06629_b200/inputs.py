@@ -17,9 +17,27 @@ def fc(n_in, n_out, act="relu", bias=True):
     return dict(kind="fc", n_in=n_in, n_out=n_out, act=act, pool=0, bias=bias)
 
 
-def conv(c_in, c_out, H, W, act="relu", pool=0, bias=True):
-    return dict(kind="conv", n_in=c_in, n_out=c_out, H=H, W=W, R=3, S=3, pad=1,
-                stride=1, act=act, pool=pool, bias=bias)
+def conv(c_in, c_out, H, W, act="relu", pool=0, bias=True, R=3, S=3, pad=1, stride=1):
+    return dict(kind="conv", n_in=c_in, n_out=c_out, H=H, W=W, R=R, S=S, pad=pad,
+                stride=stride, act=act, pool=pool, bias=bias)
+
+
+def conv_out_hw(layer):
+    return ((layer["H"] + 2 * layer["pad"] - layer["R"]) // layer["stride"] + 1,
+            (layer["W"] + 2 * layer["pad"] - layer["S"]) // layer["stride"] + 1)
+
+
+def sample_net(hw=224, classes=10):
+    """The sample network of Table I (four convolution layers: 5x5 stride 2, 5x5 stride 2,
+    3x3 stride 2, 3x3 stride 1; 3 -> 32 -> 64 -> 128 -> 128 channels) followed by one fully
+    connected layer so that it can be trained against a loss."""
+    spec = [(5, 3, 32, 2, 2), (5, 32, 64, 2, 2), (3, 64, 128, 1, 2), (3, 128, 128, 1, 1)]
+    layers, h = [], hw
+    for k, cin, cout, pad, stride in spec:
+        layers.append(conv(cin, cout, h, h, "relu", 0, True, R=k, S=k, pad=pad, stride=stride))
+        h = (h + 2 * pad - k) // stride + 1
+    layers.append(fc(128 * h * h, classes, "none"))
+    return layers
 
 
 def mlp(widths, act):
@@ -63,6 +81,8 @@ WORKLOADS = {
                                        512, 512, 512, "P", 512, 512, 512, "P"],
                                  [4096, 4096, 1000]),
                       batch=64, stages=9, delays=None, lr=0.001, momentum=0.0, steps=10),
+    # the paper's own example (Table I; Section IV-B runs it at 224 x 224 x 3, batch 32, on three processors)
+    "sample4_224": dict(layers=sample_net(224), batch=32, stages=3, delays=None, lr=0.0005, momentum=0.0, steps=10),
     "mlp16_8192": dict(layers=mlp([8192] * 17, "gelu"), batch=2048, stages=9, delays=None,
                        lr=0.01, momentum=0.0, steps=10),
 }
