@@ -34,6 +34,9 @@ int make_tmap_rows32(CUtensorMap* out, const void* base, int elem_bytes, uint64_
 struct GemmArgs;
 struct UpdMaps;
 constexpr int GEMM_BN_PAIR = 512;   // tile code: 256 x 256 tile computed by a pair of CTAs (cta_group::2)
+constexpr int GEMM_BN_PAIR224 = 448;   // tile code: 256 x 224 tile on a pair of CTAs (forward / delta only)
+inline bool gemm_is_pair(int bn) { return bn == GEMM_BN_PAIR || bn == GEMM_BN_PAIR224; }
+inline int gemm_tile_cols(int bn) { return gemm_is_pair(bn) ? bn / 2 : bn; }   // output columns of one tile
 // which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
 // Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
 // (see gemm_box_dims).

@@ -126,6 +126,16 @@ void gemm_set_tuning(int bn, int stages, int splits) {
   if (g_force_persistent > 1) g_force_persistent = -1;
 }
 
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+  }
+  return n;
+}
+
 // Split-K factor.  Measured on B200 (M = 256, N = K = 4096): the split main loop is shorter
 // but writing and re-reading the fp32 partial tiles costs more than it saves (25 us unsplit,
 // 28 / 35 / 52 us at 2 / 4 / 8 splits), and under the stage scheduler other kernels fill the
@@ -146,9 +156,19 @@ int gemm_pick_splits(int M, int N, int K, int bn) {
 
 int gemm_pick_bn(int which, int M, int N, int K) {
   if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256 || g_force_bn == GEMM_BN_PAIR) return g_force_bn;
+  if (g_force_bn == GEMM_BN_PAIR224) return which == 2 ? GEMM_BN_PAIR : GEMM_BN_PAIR224;
   if (N <= 64) return 64;
   // tensor-bound shapes: 256 x 256 tiles on SM pairs (code GEMM_BN_PAIR)
-  if (M >= 1024 && N >= 1024 && K >= 1024) return GEMM_BN_PAIR;
+  if (M >= 1024 && N >= 1024 && K >= 1024) {
+    // forward / delta: a 224-column tile where that fills the last round of SM pairs better (cost =
+    // rounds of tiles over the pairs x tile width); G keeps 256 (its update streams 64-column fills)
+    if (which != 2 && g_force_bn == 0) {
+      const long long pairs = std::max(1, sm_count() / 2), tm = (M + 255) / 256;
+      const long long t256 = tm * ((N + 255) / 256), t224 = tm * ((N + 223) / 224);
+      if (((t224 + pairs - 1) / pairs) * 224 < ((t256 + pairs - 1) / pairs) * 256) return GEMM_BN_PAIR224;
+    }
+    return GEMM_BN_PAIR;
+  }
   (void)which;
   // 128 x 256 tiles need 96 B/clk of operands per SM instead of 128 B/clk and measured 1250 vs
   // 1130 TFLOP/s on 2048 x 8192 x 8192; they only pay off when the contraction is long and
@@ -164,19 +184,9 @@ int gemm_pick_bn(int which, int M, int N, int K) {
 void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
   boxA[0] = 64; boxA[1] = a_mn ? 64 : GEMM_BM;
-  boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(bn == GEMM_BN_PAIR ? 128 : bn);   // a pair CTA stages half of the 256 columns
+  boxB[0] = 64; boxB[1] = b_mn ? 64 : uint32_t(gemm_is_pair(bn) ? gemm_tile_cols(bn) / 2 : bn);   // a pair CTA stages half of the tile's columns
 }
 
-
-static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-  }
-  return n;
-}
 
 template <int BN, bool A_MN, bool B_MN, int MODE>
 static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st,
@@ -265,7 +275,7 @@ static cudaError_t configure_one() {
   X(BN, true, true, EPI_WGRAD_UPDATE)
 
 // ---- two-CTA (SM pair) kernel ---------------------------------------------------------------
-template <bool A_MN, bool B_MN, int MODE>
+template <bool A_MN, bool B_MN, int MODE, int BN2 = GEMM2_BN>
 static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmArgs a, cudaStream_t st, const UpdMaps* um) {
   a.splits = 1;
   if (a.wait_limit <= 0) a.wait_limit = LP_WAIT_LIMIT_CYCLES;
@@ -281,7 +291,7 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   a.num_stages = s;
   cudaLaunchConfig_t cfg = {};
   // (convolution geometry: M is a whole number of 128-pixel boxes, and an even one -- the caller checks)
-  cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N - a.n_begin + GEMM2_BN - 1) / GEMM2_BN, 1);
+  cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N - a.n_begin + BN2 - 1) / BN2, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = size_t(s) * stage_bytes + tail;
   cfg.stream = st;
@@ -292,10 +302,10 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if constexpr (MODE == EPI_WGRAD_UPDATE) {
+  if constexpr (MODE == EPI_WGRAD_UPDATE && BN2 == GEMM2_BN) {
     if (a.upd_tma) return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, tmA, tmB, *um, a);
   }
-  return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false>, tmA, tmB, *um, a);
+  return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false, BN2>, tmA, tmB, *um, a);
 }
 template <bool A_MN, bool B_MN, int MODE>
 static cudaError_t configure_pair() {
@@ -304,6 +314,9 @@ static cudaError_t configure_pair() {
   if constexpr (MODE == EPI_WGRAD_UPDATE) {
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  } else if constexpr (!A_MN) {      // forward / delta also exist with 224-column tiles
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   }
   return e;
 }
@@ -385,6 +398,14 @@ cudaError_t gemm_configure() {
 cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
                         cudaStream_t st, const UpdMaps* um) {
   const bool a_mn = (which == 2), b_mn = (which != 0);
+  if (bn == GEMM_BN_PAIR224) {
+    if (a_mn || args.g.kind != GEOM_PLAIN) return cudaErrorInvalidValue;
+#define LP_TRYP224(A, B, M) \
+  if (!A && b_mn == B && args.mode == M) return launch_pair<A, B, M, 224>(tmA, tmB, args, st, nullptr);
+    LP_FOR_EACH_PAIR_VARIANT(LP_TRYP224)
+#undef LP_TRYP224
+    return cudaErrorInvalidValue;
+  }
   if (bn == GEMM_BN_PAIR) {
     if (args.g.kind == GEOM_PIX_K) return cudaErrorInvalidValue;
 #define LP_TRYP(A, B, M) \

@@ -88,13 +88,21 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 // chunk fill completes on the CTA's own barrier ufull[stage] (the operand fills of both CTAs
 // complete on the leader's full[stage]); both kinds of use release the stage through empty[stage],
 // so the ring position, and with it the phase of empty[], stays uniform in both CTAs.
-template <bool A_MN, bool B_MN, int MODE, bool UTMA = false>
+// BN2: columns of the pair's tile, 256 or a smaller multiple of 32 (each CTA stages BN2 / 2 of them).
+// A narrower tile is chosen where it makes the number of tiles a whole multiple of the SM pairs:
+// 2048 x 8192 outputs are 256 tiles of 256 columns -- 3.46 per SM pair, so some pairs run four and
+// the tensor pipes of the others idle 13 % of the time -- but 296 = 4 x 74 tiles of 224 columns.
+template <bool A_MN, bool B_MN, int MODE, bool UTMA = false, int BN2 = GEMM2_BN>
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ UpdMaps um, const GemmArgs p) {
   static_assert(!UTMA || MODE == EPI_WGRAD_UPDATE, "the streamed update belongs to the G contraction");
   constexpr int STAGE_BYTES = GEMM_A_BYTES + 128 * GEMM_BK * 2;      // A rows + half of the B tile: 32 KiB
-  constexpr int kChunks = GEMM2_BN / 32;
+  static_assert(BN2 % 32 == 0 && BN2 >= 64 && BN2 <= 256 && (!UTMA || BN2 == 256), "pair tile width");
+  constexpr int kChunks = BN2 / 32;
+  // bytes one CTA's loads bring per k-block: its 128 rows of A and its half of the B tile (MN-major B comes in whole
+  // 64-column boxes: the second box may reach past the half)
+  constexpr uint32_t kLoadBytes = GEMM_A_BYTES + (B_MN ? 2 * 8192 : (BN2 / 2) * GEMM_BK * 2);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int S = p.num_stages;
@@ -113,7 +121,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
   TileMap tm;
   tm.m0 = (blockIdx.x >> 1) * 256 + int(rank) * 128;    // this CTA's 128 rows
-  tm.n0 = p.n_begin + blockIdx.y * GEMM2_BN;            // the pair's 256 columns
+  tm.n0 = p.n_begin + blockIdx.y * BN2;                 // the pair's columns
   tm.nlim = p.N;
   tm.pn0 = tm.ph0 = tm.pw0 = 0;
   if (pix) {                                            // this CTA's box of 128 pixels
@@ -123,7 +131,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tm.ph0 = th << p.g.lh;
     tm.pn0 = tn * (GEMM_BM >> (p.g.lw + p.g.lh));
   }
-  const int nb0 = tm.n0 + int(rank) * 128;              // the half of B this CTA stages
+  const int nb0 = tm.n0 + int(rank) * (BN2 / 2);        // the half of B this CTA stages
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmA);
@@ -167,7 +175,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t sa = smem0 + s * uint32_t(STAGE_BYTES);
         const uint32_t sb = sa + GEMM_A_BYTES;
         const uint32_t fb = map_to_cta(full0 + 8u * s, 0);          // the leader's barrier
-        if (rank == 0) mbar_arrive_expect_tx_addr(full0 + 8u * s, 2 * STAGE_BYTES);
+        if (rank == 0) mbar_arrive_expect_tx_addr(full0 + 8u * s, 2u * kLoadBytes);
         if (pix) {
           // (this kernel serves stride-1 layers: the tap's shift is the whole coordinate arithmetic)
           const int r = c_tap / p.g.S, sft = c_tap % p.g.S;
@@ -232,7 +240,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(256, GEMM2_BN, A_MN, B_MN);
+      constexpr uint32_t idesc = make_idesc_bf16(256, BN2, A_MN, B_MN);
       const uint64_t dA = A_MN ? make_smem_desc(smem_u32(smem), 8192, 1024) : make_smem_desc(smem_u32(smem), 16, 1024);
       const uint64_t dB = B_MN ? make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 8192, 1024)
                                : make_smem_desc(smem_u32(smem) + GEMM_A_BYTES, 16, 1024);
@@ -379,7 +387,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tc_fence_after();
     if (ok) {
 #pragma unroll 1
-      for (int c = 0; c < GEMM2_BN / 32; ++c) {
+      for (int c = 0; c < BN2 / 32; ++c) {
         uint32_t r[32];
         __syncwarp();
         tmem_ld_32x32(tmem_base + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
@@ -391,7 +399,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int n = tm.n0 + c * 32 + sub_col;
         if constexpr (upd) {
           WmRegs nxt;
-          if (c + 1 < GEMM2_BN / 32) load_wm(p, row0, n + 32, tm.nlim, sub_row, nxt);
+          if (c + 1 < BN2 / 32) load_wm(p, row0, n + 32, tm.nlim, sub_row, nxt);
           apply_update(p, row0, n, tm.nlim, sub_row, tile, sub_col, cur);
           cur = nxt;
         } else {

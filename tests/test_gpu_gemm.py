@@ -39,7 +39,7 @@ def _reference(which, M, N, K, A, B):
     return a[:K, :M].T @ b[:K, :N]
 
 
-@pytest.mark.parametrize("tile_n", [0, 64, 256, 512])      # 512 = 256 x 256 tile on an SM pair (cta_group::2)
+@pytest.mark.parametrize("tile_n", [0, 64, 256, 512, 448])      # 512 / 448 = 256 x 256 / 256 x 224 tile on an SM pair (cta_group::2)
 @pytest.mark.parametrize("which", [0, 1, 2])
 def test_contraction_matches_definition(which, tile_n):
     import torch

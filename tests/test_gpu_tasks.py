@@ -231,11 +231,12 @@ def test_tasks_sm_pair_tiles():
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
     layers = I.mlp([520, 328, 600, 75], "gelu")
-    lpb.lp_set_tuning(512, 0, 0)
-    try:
-        run_teacher_forced(layers, 300, 3, [2, 1, 0], 0.05, 0.9, 4)
-    finally:
-        lpb.lp_set_tuning(0, 0, 0)
+    for code in (512, 448):          # 256-column tiles; 224-column tiles for forward and delta (G keeps 256)
+        lpb.lp_set_tuning(code, 0, 0)
+        try:
+            run_teacher_forced(layers, 300, 3, [2, 1, 0], 0.05, 0.9, 4)
+        finally:
+            lpb.lp_set_tuning(0, 0, 0)
 
 
 def test_tasks_degenerate_shapes():
