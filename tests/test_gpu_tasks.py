@@ -368,3 +368,19 @@ def test_tasks_sample_network_of_table1_full_size():
     wl = I.WORKLOADS["sample4_224"]
     w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 2)
     print("sample4_224 worst per-task errors", w)
+
+
+def test_tasks_sm_pair_persistent_g_update():
+    """The persistent SM-pair G kernel (one CTA pair per SM pair walks several 256 x 256 tiles, the
+    update of one tile streaming under the main loop of the next): forced onto ragged shapes with
+    fewer tiles than SM pairs and with more (99 tiles: a second tile for 25 pairs), with and without
+    momentum (two or four chunk slots)."""
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    lpb.lp_set_tuning(512, 0, 512)
+    try:
+        run_teacher_forced(I.mlp([520, 328, 600, 75], "gelu"), 300, 3, [2, 1, 0], 0.05, 0.9, 3)
+        run_teacher_forced(I.mlp([2600, 2200, 75], "gelu"), 300, 2, [1, 0], 0.05, 0.9, 2)
+        run_teacher_forced(I.mlp([2600, 2200, 75], "gelu"), 300, 2, [1, 0], 0.05, 0.0, 2)
+    finally:
+        lpb.lp_set_tuning(0, 0, 0)
