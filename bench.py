@@ -197,6 +197,15 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------- our arm
+_T0 = time.perf_counter()
+
+
+def note(msg):
+    """Progress on stderr (the JSON line is the only thing written to stdout)."""
+    sys.stderr.write("[bench %7.1f s] %s\n" % (time.perf_counter() - _T0, msg))
+    sys.stderr.flush()
+
+
 MIN_TIMED_SECONDS = 1.5     # the timed region is repeated until this much device time has been measured
 
 
@@ -438,6 +447,7 @@ def borrowing_report(torch, lpb, w, args, stream):
     steps = args.steps
     for pname, plan in plans.items():
         for split in (False, True):
+            note("  variant %s%s" % (pname, "+split" if split else ""))
             tr = lpb.Trainer(w.layers, w.B, wl["stages"], stage=plan["stage"], delays=wl["delays"] if pname == "mac_model" else None,
                              lr=wl["lr"], momentum=wl["momentum"], schedule=lpb.LP_SCHED_LAYERPIPE, W0=w.W0, b0=w.b0, device=w.dev)
             cols = tr.set_delta_split(plan["piece_stage"], plan["piece_amount"]) if split else None
@@ -479,8 +489,10 @@ def run_ours(args):
     dev = "cuda:%d" % local
     stream = torch.cuda.current_stream()
     sched = lpb.LP_SCHED_FUSED_B if args.schedule == "fused_b" else lpb.LP_SCHED_LAYERPIPE
+    note("workload %s: generating inputs" % args.workload)
     w = Workload(torch, args.workload, dev)
     wl, layers, B = w.wl, w.layers, w.B
+    note("timed loop")
 
     def barrier():
         torch.cuda.synchronize()
@@ -510,6 +522,7 @@ def run_ours(args):
         t = e2e_block(torch, tr, w.hx, w.hy, xd, yd, args.steps, stream, lag, state["first"])
         state["first"] += args.steps
         return t
+    note("end-to-end loop")
     ts_e2e = repeat_blocks(e2e_once, min(args.min_seconds, 1.0))
     barrier()
     e2e_sum = summarize(ts_e2e, args.steps)
@@ -531,6 +544,7 @@ def run_ours(args):
         peaks = load_peaks()
         # ---- same GPU, same kernels, backward as ONE task per layer (PipeDream-style) -------------
         osched = lpb.LP_SCHED_LAYERPIPE if sched == lpb.LP_SCHED_FUSED_B else lpb.LP_SCHED_FUSED_B
+        note("other schedule")
         tro, ts_o, _, _, _ = throughput(torch, lpb, w, osched, args.steps, args.warmup, min(args.min_seconds, 1.0), stream)
         tro.close()
         del tro
@@ -543,19 +557,24 @@ def run_ours(args):
         # duration there is the time it spent sharing, not its own cost.  The roofline uses a second
         # pass of the same steps with every task on one stream (LP_SERIAL_TASKS: the same kernels,
         # launches and operands, none overlapping); the overlapped averages are reported beside it.
+        note("per-kernel times")
         kinds_live = kernel_times(torch, lpb, w, sched, lpb.LP_TIME_TASKS, args.steps, stream)
         kinds = kernel_times(torch, lpb, w, sched, lpb.LP_TIME_TASKS | lpb.LP_SERIAL_TASKS, args.steps, stream)
         for kind in kinds:
             kinds[kind]["avg_us_overlapped"] = kinds_live[kind]["avg_us"]
         roof, wm = roofline(args.workload, wl, kinds, peaks)
+        note("borrowing report")
         borrowing = borrowing_report(torch, lpb, w, args, stream) if world == 1 else None
         del w
         torch.cuda.empty_cache()
         per_workload = {}
         if not args.no_per_workload and world == 1:
             for name in I.WORKLOADS:
+                note("per-workload: %s" % name)
                 per_workload[name] = short_measure(torch, lpb, name, dev, stream, peaks)
+        note("cpu baseline (oracle)")
         cpu = cpu_baseline(wl)
+        note("done")
         value = world * args.steps * B / (ms * 1e-3)
         e2e_value = world * args.steps * B / (ms_e2e * 1e-3)
         in_bytes = xd[0].numel() * xd[0].element_size() + yd[0].numel() * yd[0].element_size()
@@ -615,6 +634,30 @@ def cpu_baseline(wl):
             "sample": "%d whole minibatches of %d, full-size layers, %.1f s" % (n, B, dt)}
 
 
+def supervise(args, limit_s=900.0):
+    env = dict(os.environ, LP_BENCH_CHILD="1")
+    cmd = [sys.executable, "-X", "faulthandler", os.path.abspath(__file__)] + sys.argv[1:]
+    for attempt in (1, 2):
+        p = subprocess.Popen(cmd, env=env, stdout=subprocess.PIPE)
+        try:
+            out, _ = p.communicate(timeout=limit_s)
+        except subprocess.TimeoutExpired:
+            try:
+                p.send_signal(__import__("signal").SIGABRT)     # faulthandler prints the child's Python stack
+                p.wait(timeout=10)
+            except Exception:
+                p.kill()
+                p.wait()
+            note("attempt %d did not finish within %.0f s%s" % (attempt, limit_s, "; trying once more" if attempt == 1 else ""))
+            continue
+        sys.stdout.write(out.decode())
+        sys.stdout.flush()
+        if p.returncode != 0:
+            raise SystemExit(p.returncode)
+        return
+    raise SystemExit("bench.py: the measurement did not finish in two attempts")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -625,6 +668,8 @@ def main():
     ap.add_argument("--schedule", default="layerpipe", choices=["layerpipe", "fused_b"])
     ap.add_argument("--min-seconds", dest="min_seconds", type=float, default=MIN_TIMED_SECONDS)
     ap.add_argument("--no-per-workload", dest="no_per_workload", action="store_true")
+    ap.add_argument("--no-watchdog", dest="no_watchdog", action="store_true",
+                    help="measure in this process instead of a supervised child")
     ap.add_argument("--only-main", dest="only_main", action="store_true",
                     help="time the main loop only and print a reduced line (for profiler launch lists)")
     args = ap.parse_args()
@@ -639,6 +684,10 @@ def main():
         out = replicas.spawn_replicas([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
         sys.stdout.write(out)
         return
+    if os.environ.get("LP_BENCH_CHILD") != "1" and not args.no_watchdog:
+        # Run the measurement in a child process under a time limit and try once more if it neither
+        # finishes nor fails in time: a wedged run must not turn into a benchmark that never ends.
+        return supervise(args)
     run_ours(args)
 
 
