@@ -79,6 +79,10 @@ cudaError_t launch_cast_stash(const void* batch, int input_is_bf16, const int* l
                               int* labels_copy, int rows, int B, int n_in, int ld, cudaStream_t stream);
 cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
                                  int* labels_copy, int B, int H, int W, int C, int ld, cudaStream_t stream);
+// The same for any filter, stride and padding (R*S*C <= 128): one row per OUTPUT pixel, column (r*S + s)*C + ch.
+cudaError_t launch_cast_patch_general(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                                      int* labels_copy, int B, int H, int W, int C, int R, int S, int stride, int pad,
+                                      int Ho, int Wo, int ld, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
                                 int* status, cudaStream_t stream);

@@ -131,6 +131,57 @@ cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int
   return cudaGetLastError();
 }
 
+// General filters / strides: thread t handles 8 consecutive columns of one patch row (one 16-byte
+// store); the column's (tap, channel) and the tap's input pixel are decoded per element.
+__global__ void cast_patch_general_kernel(const void* __restrict__ batch, int input_is_bf16, const int* __restrict__ labels,
+                                          __nv_bfloat16* __restrict__ x0, int* __restrict__ labels_copy, int B, int H, int W,
+                                          int C, int R, int S, int stride, int pad, int Ho, int Wo, int ld) {
+  const int groups = ld / 8;
+  const long long total = (long long)B * Ho * Wo * groups;
+  const int n_cols = R * S * C;
+  for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+    const int g = int(t % groups);
+    const long long pix = t / groups;
+    const int wo = int(pix % Wo), ho = int((pix / Wo) % Ho), b = int(pix / ((long long)Wo * Ho));
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int col = g * 8 + j;
+      v[j] = 0.f;
+      if (col < n_cols) {
+        const int tap = col / C, ch = col % C;
+        const int hh = ho * stride + tap / S - pad, ww = wo * stride + tap % S - pad;
+        if (hh >= 0 && hh < H && ww >= 0 && ww < W) {
+          const long long idx = (((long long)b * H + hh) * W + ww) * C + ch;
+          v[j] = input_is_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(batch)[idx])
+                               : reinterpret_cast<const float*>(batch)[idx];
+        }
+      }
+    }
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&p0); o.y = *reinterpret_cast<uint32_t*>(&p1);
+    o.z = *reinterpret_cast<uint32_t*>(&p2); o.w = *reinterpret_cast<uint32_t*>(&p3);
+    *reinterpret_cast<uint4*>(x0 + pix * ld + g * 8) = o;
+  }
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i < B; i += blockDim.x) labels_copy[i] = labels[i];
+  }
+}
+
+cudaError_t launch_cast_patch_general(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
+                                      int* labels_copy, int B, int H, int W, int C, int R, int S, int stride, int pad,
+                                      int Ho, int Wo, int ld, cudaStream_t stream) {
+  const long long total = (long long)B * Ho * Wo * (ld / 8);
+  if (C < 1 || R * S * C > ld || (ld & 7) || total >= (1ll << 40)) return cudaErrorInvalidValue;
+  int blocks = int(std::min<long long>((total + 255) / 256, 148 * 16));
+  if (blocks < 1) blocks = 1;
+  cast_patch_general_kernel<<<blocks, 256, 0, stream>>>(batch, input_is_bf16, labels, x0, labels_copy, B, H, W, C, R, S, stride,
+                                                        pad, Ho, Wo, ld);
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------
 // One block per row: p = softmax(z^L), delta^L = RN((p - onehot)/B), row loss; the last
 // block to finish adds the row losses in row order (deterministic mean).

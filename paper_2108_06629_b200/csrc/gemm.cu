@@ -308,15 +308,14 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
       // per SM pair, update streamed under the next tile's main loop (8192 x 8192 x 2048: 255 -> 248 us).
       const int tiles_m = (a.M + 255) / 256, tiles_n = (a.N + GEMM2_BN - 1) / GEMM2_BN;
       const int pairs = std::max(1, sm_count() / 2);
-      // (with momentum the 64 KiB of chunk memory hold two slots only and the one-tile form measured faster: 337 / 376 us)
-      const bool persistent = g_force_persistent >= 0 ? g_force_persistent == 1
-                                                      : (tiles_m * tiles_n >= 2 * pairs && num_kb <= 96 && a.mW == nullptr);
+      const bool persistent = g_force_persistent >= 0 ? g_force_persistent == 1 : (tiles_m * tiles_n >= 2 * pairs && num_kb <= 96);
       if (persistent && a.starve_kb == 0) {
         cfg.gridDim = dim3(2 * std::min(tiles_m * tiles_n, pairs), 1, 1);
         cfg.blockDim = dim3(GEMM2P_THREADS, 1, 1);
         cfg.dynamicSmemBytes = GEMM2P_SMEM_BYTES;
         // 192 KiB of shared memory divided between operand stages and update-chunk slots
-        a.num_stages = g_force_stages > 0 ? std::max(2, std::min(g_force_stages, 5)) : 4;
+        // (chunk slots are 16 KiB, 32 KiB with momentum: four operand stages leave four / two of them, three leave six / three)
+        a.num_stages = g_force_stages > 0 ? std::max(2, std::min(g_force_stages, 5)) : (a.mW != nullptr ? 3 : 4);
         return cudaLaunchKernelEx(&cfg, gemm2p_g_update_kernel<0>, tmA, tmB, *um, a, tiles_m, tiles_n);
       }
       return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, tmA, tmB, *um, a);

@@ -10,25 +10,28 @@
 //   warp 6     update-tile producer: streams the fp32 master (and momentum) of the tiles, one 128 x 32
 //              chunk per fill, through chunk slots of its own (64 KiB: four slots, or two with
 //              momentum), independent of the operand ring and as far ahead as the slots allow
-//   warp 7     store issuer: sends every updated chunk (master, momentum, bf16 image) back with TMA
-//              stores and frees its slot as soon as the stores have read it
-// so the update of tile i (an HBM stream) runs under the main loop of tile i + 1.
+// so the update of tile i (an HBM stream) runs under the main loop of tile i + 1.  An epilogue lane
+// owns one row of the chunk: it reads its 128 bytes of master (and momentum) from the slot, applies
+// Eq. 6 to its accumulator row and writes master, momentum and the bf16 image straight to global
+// memory with 32-byte stores -- the results do not pass through shared memory again.  (The SM-pair
+// main loop already uses most of the shared-memory bandwidth: 48 KiB read by the tensor core and
+// 32 KiB written by TMA per k-block; an update staged in shared memory and sent back with TMA stores
+// added 25 % to that traffic and the same 25 % to the kernel's time.)
 //
 // Barriers.  full[s] (leader; both CTAs' operand loads complete on it), empty[s] (each CTA; released by
 // tcgen05.commit multicast), accf[b] (each CTA; accumulator b complete, commit multicast), acce[b]
 // (leader; eight arrivals: the four epilogue warps of each CTA have read accumulator b out of tensor
-// memory), ufull[u] / uempty[u] (each CTA's own chunk slots), staged[k] / sfree[k] (the two bf16 staging
-// tiles between the epilogue warps and the store issuer).  Every wait is bounded.
+// memory), ufull[u] / uempty[u] (each CTA's own chunk slots; 128 arrivals free a slot).  Every wait is bounded.
 #pragma once
 #include "gemm2.cuh"
 
 namespace lp {
 
-constexpr int GEMM2P_THREADS = 256;
+constexpr int GEMM2P_THREADS = 224;
 constexpr int GEMM2P_STAGE = 32 * 1024;
 constexpr int GEMM2P_POOL = 6 * GEMM2P_STAGE;        // operand stages (32 KiB each) + chunk slots (16 KiB, 32 KiB with momentum) share 192 KiB
 constexpr int GEMM2P_MAX_SO = 6, GEMM2P_MAX_SC = 8;
-constexpr int GEMM2P_SMEM_BYTES = GEMM2P_POOL + 2 * UPD_RING_BYTES + 1024 + 1024;
+constexpr int GEMM2P_SMEM_BYTES = GEMM2P_POOL + 1024 + 1024;
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -44,16 +47,13 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* chunk_mem = smem + SO * STAGE;
-  uint8_t* ring_mem = smem + GEMM2P_POOL;                             // two bf16 staging tiles (8 KiB each)
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring_mem + 2 * UPD_RING_BYTES);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + GEMM2P_POOL);
   uint64_t* empty_bar = full_bar + SO_MAX;
   uint64_t* accf_bar = empty_bar + SO_MAX;    // [2]
   uint64_t* acce_bar = accf_bar + 2;          // [2]
   uint64_t* ufull_bar = acce_bar + 2;         // [SC]
   uint64_t* uempty_bar = ufull_bar + SC_MAX;  // [SC]
-  uint64_t* staged_bar = uempty_bar + SC_MAX; // [2] a staging tile (and its chunk slot) is ready to be stored
-  uint64_t* sfree_bar = staged_bar + 2;       // [2] a staging tile may be written again
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sfree_bar + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(uempty_bar + SC_MAX);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -70,7 +70,6 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     tma_prefetch_desc(&tmB);
     tma_prefetch_desc(&um.W);
     if (p.mW != nullptr) tma_prefetch_desc(&um.M);
-    tma_prefetch_desc(&um.R);
     for (int s = 0; s < SO; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
@@ -81,11 +80,7 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     for (int u = 0; u < SC_MAX; ++u) {
       mbar_init(&ufull_bar[u], 1);
-      mbar_init(&uempty_bar[u], 1);
-    }
-    for (int k = 0; k < 2; ++k) {
-      mbar_init(&staged_bar[k], 128);
-      mbar_init(&sfree_bar[k], 1);
+      mbar_init(&uempty_bar[u], 128);     // every epilogue thread has read its row of the slot
     }
     fence_barrier_init();
   }
@@ -205,54 +200,16 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         for (long long i = (issued > SC ? issued - SC : 0); i < issued; ++i) mbar_wait(&ufull_bar[i % SC], uint32_t(i / SC) & 1u, p.wait_limit);
       }
     }
-  } else if (warp == 7) {
-    // ------------------------------------------------------------ store issuer (both CTAs)
-    if (lane == 0) {
-      bool ok = true;
-      const uint32_t chunk0 = smem_u32(chunk_mem), ring0 = smem_u32(ring_mem);
-      const uint32_t staged0 = smem_u32(staged_bar), sfree0 = smem_u32(sfree_bar), uempty0 = smem_u32(uempty_bar);
-      uint32_t u = 0, gc = 0, prev_u = 0;
-      for (int t = pair_id; t < total && ok; t += pairs) {
-        const int m0 = (t % tiles_m) * 256 + int(rank) * 128;
-        const int n0 = (t / tiles_m) * GEMM2_BN;
-        for (int c = 0; c < kChunks; ++c, ++gc) {
-          const uint32_t k = gc & 1u;
-          ok = mbar_wait_addr(staged0 + 8u * k, (gc >> 1) & 1u, p.wait_limit);
-          if (!ok) break;
-          const uint32_t sW = chunk0 + u * slot_bytes;
-          const int n = n0 + c * 32;
-          tma_store_2d_addr(&um.W, sW, n, m0);
-          if (mom) tma_store_2d_addr(&um.M, sW + UPD_CHUNK_BYTES, n, m0);
-          tma_store_2d_addr(&um.R, ring0 + k * uint32_t(UPD_RING_BYTES), n, m0);
-          tma_store_commit();
-          // one group may stay in flight: the stores of the PREVIOUS chunk have read shared memory, so its
-          // chunk slot and its staging tile are free
-          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-          if (gc > 0) {
-            mbar_arrive_addr(uempty0 + 8u * prev_u);
-            mbar_arrive_addr(sfree0 + 8u * (k ^ 1u));
-          }
-          prev_u = u;
-          if (++u == uint32_t(SC)) u = 0;
-        }
-      }
-      tma_store_wait_read0();
-      if (ok && gc > 0) {                                // (the last chunk's slot: nobody waits for it any more, kept for symmetry)
-        mbar_arrive_addr(uempty0 + 8u * prev_u);
-        mbar_arrive_addr(sfree0 + 8u * ((gc - 1) & 1u));
-      }
-      if (!ok) atomicExch(p.status, 20);
-    }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2-5 of both CTAs, own 128 rows)
     const int q = warp & 3;                                     // tensor-memory lane quarter this warp may read
     const int trow = q * 32 + lane;                             // row of this CTA's half tile = tensor-memory lane
-    const uint32_t chunk0 = smem_u32(chunk_mem), ring0 = smem_u32(ring_mem);
-    const uint32_t accf0 = smem_u32(accf_bar), ufull0 = smem_u32(ufull_bar);
-    const uint32_t staged0 = smem_u32(staged_bar), sfree0 = smem_u32(sfree_bar);
+    const uint32_t chunk0 = smem_u32(chunk_mem);
+    const uint32_t accf0 = smem_u32(accf_bar), ufull0 = smem_u32(ufull_bar), uempty0 = smem_u32(uempty_bar);
     const uint32_t acce_leader = map_to_cta(smem_u32(acce_bar), 0);
+    const bool ring32 = (p.ld_out & 15) == 0;                   // rows of the bf16 image start on 32-byte boundaries
     bool good = true;
-    uint32_t it = 0, u = 0, uph = 0, gc = 0;                    // tile count, chunk slot / phase, running chunk count
+    uint32_t it = 0, u = 0, uph = 0;                            // tile count, chunk slot / phase
     for (int t = pair_id; t < total && good; t += pairs, ++it) {
       const int m0 = (t % tiles_m) * 256 + int(rank) * 128;
       const int n0 = (t / tiles_m) * GEMM2_BN;
@@ -265,14 +222,14 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         break;
       }
       tc_fence_after();
+      const int grow = m0 + trow;
+      const bool row_ok = grow < p.M;
+      const size_t rowbase = size_t(row_ok ? grow : 0) * p.ld_out;
 #pragma unroll 1
-      for (int c = 0; c < kChunks; ++c, ++gc) {
-        const uint32_t k = gc & 1u;
+      for (int c = 0; c < kChunks; ++c) {
         const uint32_t sW = chunk0 + u * slot_bytes;
         const uint32_t sM = sW + UPD_CHUNK_BYTES;               // (momentum form only)
-        const uint32_t ringbuf = ring0 + k * uint32_t(UPD_RING_BYTES);
-        // the chunk's master (and momentum) have landed, and the staging tile of two chunks ago has been stored
-        good = mbar_wait_addr(ufull0 + 8u * u, uph, p.wait_limit) && mbar_wait_addr(sfree0 + 8u * k, ((gc >> 1) & 1u) ^ 1u, p.wait_limit);
+        good = mbar_wait_addr(ufull0 + 8u * u, uph, p.wait_limit);
         good = __all_sync(0xffffffffu, good);
         if (!good) {
           if (lane == 0) atomicExch(p.status, 19);
@@ -280,59 +237,82 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
         uint32_t r[32];
         tmem_ld_32x32(tacc + (uint32_t(q * 32) << 16) + uint32_t(c * 32), r);
+        // this lane's row of the chunk: 128 bytes of master (and momentum), 128-byte swizzle
+        const uint32_t rowoff = uint32_t(trow) * 128u;
+        const uint32_t swz = uint32_t(trow & 7);
+        float4 w[8], mm[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t off = rowoff + ((uint32_t(j) ^ swz) << 4);
+          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w[j].x), "=f"(w[j].y), "=f"(w[j].z), "=f"(w[j].w) : "r"(sW + off));
+          if (mom)
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(mm[j].x), "=f"(mm[j].y), "=f"(mm[j].z), "=f"(mm[j].w) : "r"(sM + off));
+        }
         tmem_ld_wait();
+        // the slot has been read (the loads above have returned their values before the arrive is performed)
+        mbar_arrive_addr(uempty0 + 8u * u);
         if (c == kChunks - 1) {
           // last read of this accumulator: hand it back to the MMA issuer (in the leader CTA)
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acce_leader + 8u * buf);
         }
-        const uint32_t rowoff = uint32_t(trow) * 128u;
-        const uint32_t swz = uint32_t(trow & 7);
-        const int grow = m0 + trow;
+        const int nc = n0 + c * 32;
         uint32_t packed[16];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const uint32_t off = rowoff + ((uint32_t(j) ^ swz) << 4);
-          float g[4] = {__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                        __uint_as_float(r[4 * j + 3])};
-          const int n = n0 + c * 32 + 4 * j;
-          if (p.out != nullptr && grow < p.M && n < p.N) {
-            float* dst = reinterpret_cast<float*>(p.out) + size_t(grow) * p.ld_out + n;
-            if (n + 3 < p.N) {
-              __stcs(reinterpret_cast<float4*>(dst), make_float4(g[0], g[1], g[2], g[3]));
-            } else {
-              for (int e = 0; e < 4; ++e) if (n + e < p.N) dst[e] = g[e];
-            }
-          }
+          const float g[4] = {__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                              __uint_as_float(r[4 * j + 3])};
           float m[4] = {g[0], g[1], g[2], g[3]};
           if (mom) {
-            float4 mm;
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(mm.x), "=f"(mm.y), "=f"(mm.z), "=f"(mm.w) : "r"(sM + off));
-            m[0] = p.mu * mm.x + g[0]; m[1] = p.mu * mm.y + g[1];
-            m[2] = p.mu * mm.z + g[2]; m[3] = p.mu * mm.w + g[3];
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sM + off), "f"(m[0]), "f"(m[1]), "f"(m[2]), "f"(m[3]) : "memory");
+            m[0] = p.mu * mm[j].x + g[0]; m[1] = p.mu * mm[j].y + g[1];
+            m[2] = p.mu * mm[j].z + g[2]; m[3] = p.mu * mm[j].w + g[3];
+            mm[j] = make_float4(m[0], m[1], m[2], m[3]);
           }
-          float4 w;
-          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w) : "r"(sW + off));
-          w.x -= p.lr * m[0]; w.y -= p.lr * m[1]; w.z -= p.lr * m[2]; w.w -= p.lr * m[3];
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(sW + off), "f"(w.x), "f"(w.y), "f"(w.z), "f"(w.w) : "memory");
-          packed[2 * j] = pack_bf16x2(w.x, w.y);
-          packed[2 * j + 1] = pack_bf16x2(w.z, w.w);
+          w[j].x -= p.lr * m[0]; w[j].y -= p.lr * m[1]; w[j].z -= p.lr * m[2]; w[j].w -= p.lr * m[3];
+          packed[2 * j] = pack_bf16x2(w[j].x, w[j].y);
+          packed[2 * j + 1] = pack_bf16x2(w[j].z, w[j].w);
         }
-        {
-          const uint32_t roff = ringbuf + uint32_t(trow) * 64u;
-          const uint32_t rs = uint32_t(trow >> 1) & 3u;
+        if (row_ok) {
+          // 32-byte stores: eight fp32 (or sixteen bf16) of this lane's row per instruction, whole sectors
 #pragma unroll
-          for (int v = 0; v < 4; ++v)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(roff + ((uint32_t(v) ^ rs) << 4)), "r"(packed[4 * v]),
-                         "r"(packed[4 * v + 1]), "r"(packed[4 * v + 2]), "r"(packed[4 * v + 3])
+          for (int j = 0; j < 4; ++j) {
+            const int n = nc + 8 * j;
+            if (n >= p.N) continue;                      // (columns up to the padded pitch exist and stay zero)
+            if (p.out != nullptr) {
+              float* dst = reinterpret_cast<float*>(p.out) + rowbase + n;
+              asm volatile("st.global.cs.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "f"(__uint_as_float(r[8 * j])),
+                           "f"(__uint_as_float(r[8 * j + 1])), "f"(__uint_as_float(r[8 * j + 2])), "f"(__uint_as_float(r[8 * j + 3])),
+                           "f"(__uint_as_float(r[8 * j + 4])), "f"(__uint_as_float(r[8 * j + 5])), "f"(__uint_as_float(r[8 * j + 6])),
+                           "f"(__uint_as_float(r[8 * j + 7]))
+                           : "memory");
+            }
+            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.W + rowbase + n), "f"(w[2 * j].x),
+                         "f"(w[2 * j].y), "f"(w[2 * j].z), "f"(w[2 * j].w), "f"(w[2 * j + 1].x), "f"(w[2 * j + 1].y), "f"(w[2 * j + 1].z),
+                         "f"(w[2 * j + 1].w)
                          : "memory");
+            if (mom)
+              asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.mW + rowbase + n), "f"(mm[2 * j].x),
+                           "f"(mm[2 * j].y), "f"(mm[2 * j].z), "f"(mm[2 * j].w), "f"(mm[2 * j + 1].x), "f"(mm[2 * j + 1].y),
+                           "f"(mm[2 * j + 1].z), "f"(mm[2 * j + 1].w)
+                           : "memory");
+          }
+          __nv_bfloat16* rdst = p.ring + rowbase + nc;
+          if (ring32) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              if (nc + 16 * j < p.N)
+                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(rdst + 16 * j), "r"(packed[8 * j]),
+                             "r"(packed[8 * j + 1]), "r"(packed[8 * j + 2]), "r"(packed[8 * j + 3]), "r"(packed[8 * j + 4]),
+                             "r"(packed[8 * j + 5]), "r"(packed[8 * j + 6]), "r"(packed[8 * j + 7])
+                             : "memory");
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (nc + 8 * j < p.N)
+                *reinterpret_cast<uint4*>(rdst + 8 * j) = make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          }
         }
-        // this thread's part of the chunk is in shared memory: make it visible to the copy engine and
-        // tell the store issuer (128 arrivals complete the chunk)
-        fence_proxy_async_smem();
-        mbar_arrive_addr(staged0 + 8u * k);
         if (++u == uint32_t(SC)) { u = 0; uph ^= 1u; }
       }
     }

@@ -385,10 +385,14 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       y.oH = (y.imH + 2 * y.cpad - y.cR) / y.cstride + 1;
       y.oW = (y.imW + 2 * y.cpad - y.cS) / y.cstride + 1;
       y.gen = !(y.cR == 3 && y.cS == 3 && y.cstride == 1 && y.cpad == 1);
-      y.patch = (l == 0 && !y.gen && 9 * y.n_in <= 64);
-      if (y.patch) { y.c_in = y.n_in; y.n_in = 9 * y.c_in; y.ld_in = pad8(y.n_in); y.taps = 1; }
-      y.in_rows = B * y.imH * y.imW;
+      // A first layer with few input channels keeps its input as the matrix of filter patches, one
+      // row per OUTPUT pixel: 3x3 / stride 1 with at most 7 channels (9 Cin <= 64), and general filters
+      // and strides with R S Cin <= 128 (the 5x5, stride-2, 3-channel layer of the paper's sample
+      // network: 75 products per pixel instead of 25 taps x 64 padded channels).
+      y.patch = l == 0 && (y.gen ? (y.taps * y.n_in <= 128 && y.n_in <= 8) : 9 * y.n_in <= 64);
       y.out_rows = B * y.oH * y.oW;
+      y.in_rows = y.patch ? y.out_rows : B * y.imH * y.imW;
+      if (y.patch) { y.c_in = y.n_in; y.n_in = y.taps * y.c_in; y.ld_in = pad8(y.n_in); y.taps = 1; }
       y.w_rows = y.n_out; y.w_ld = y.taps * y.ld_in;
       y.pool = layers[l].pool;
       y.Hp = y.pool ? y.oH / 2 : y.oH; y.Wp = y.pool ? y.oW / 2 : y.oW;
@@ -1200,7 +1204,11 @@ extern "C" int lp_step(lp_handle h, const void* batch_dev, const int* labels_dev
     LP_CUDA(c, task_begin(c, user, {}, {rx, rl}));
     ++c->launches;
     TimedScope ts(c, LP_TASK_CAST, user);
-    if (y0.patch)
+    if (y0.patch && y0.gen)
+      LP_CUDA(c, launch_cast_patch_general(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
+                                           y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.imH,
+                                           y0.imW, y0.c_in, y0.cR, y0.cS, y0.cstride, y0.cpad, y0.oH, y0.oW, y0.ld_in, user));
+    else if (y0.patch)
       LP_CUDA(c, launch_cast_patch3x3(batch_dev, c->cfg.input_dtype == LP_BF16, labels_dev,
                                       y0.X + size_t(n % y0.x_slots) * y0.x_elems, c->labels + size_t(ds) * B, B, y0.imH,
                                       y0.imW, y0.c_in, y0.ld_in, user));
@@ -1452,28 +1460,33 @@ static inline uint16_t f32_to_bf16_rn(float f) {
   return uint16_t(u >> 16);
 }
 // The patch layer's stash seen from the host as the image it was built from, NHWC [B][H][W][Cin]:
-// a write builds every pixel's 3x3 patch row, a read returns the centre tap.
+// a write builds every output pixel's patch row; a read returns the image from the taps that hold
+// each pixel (stride 1 with the centre tap inside the filter only).
 static int patch_io(lp_ctx* h, long long index, const float* in_host, float* out_host) {
   Layer& y = h->L[0];
   const int B = h->cfg.batch, H = y.imH, W = y.imW, C = y.c_in, ld = y.ld_in;
+  const int R = y.cR, S = y.cS, sd = y.cstride, pad = y.cpad, Ho = y.oH, Wo = y.oW;
   __nv_bfloat16* dev = y.X + size_t(index % y.x_slots) * y.x_elems;
   std::vector<uint16_t> tmp(y.x_elems, 0);
   LP_CUDA(h, cudaDeviceSynchronize());
   if (out_host) {
+    if (sd != 1 || pad >= R || pad >= S || Ho != H || Wo != W)
+      return fail(h, LP_ERR_UNSUPPORTED, "the patch matrix of this layer does not hold every input pixel at a fixed tap");
     LP_CUDA(h, cudaMemcpy(tmp.data(), dev, tmp.size() * 2, cudaMemcpyDeviceToHost));
+    const int centre = pad * S + pad;            // tap (pad, pad) of output pixel (h, w) is input pixel (h, w)
     for (size_t pix = 0; pix < size_t(B) * H * W; ++pix)
       for (int ch = 0; ch < C; ++ch) {
-        const uint32_t bits = uint32_t(tmp[pix * ld + 4 * C + ch]) << 16;
+        const uint32_t bits = uint32_t(tmp[pix * ld + centre * C + ch]) << 16;
         memcpy(&out_host[pix * C + ch], &bits, 4);
       }
     return LP_OK;
   }
   for (int b = 0; b < B; ++b)
-    for (int hh = 0; hh < H; ++hh)
-      for (int ww = 0; ww < W; ++ww) {
-        uint16_t* row = &tmp[((size_t(b) * H + hh) * W + ww) * ld];
-        for (int tap = 0; tap < 9; ++tap) {
-          const int sh = hh + tap / 3 - 1, sw = ww + tap % 3 - 1;
+    for (int ho = 0; ho < Ho; ++ho)
+      for (int wo = 0; wo < Wo; ++wo) {
+        uint16_t* row = &tmp[((size_t(b) * Ho + ho) * Wo + wo) * ld];
+        for (int tap = 0; tap < R * S; ++tap) {
+          const int sh = ho * sd + tap / S - pad, sw = wo * sd + tap % S - pad;
           if (sh < 0 || sh >= H || sw < 0 || sw >= W) continue;
           const float* src = in_host + ((size_t(b) * H + sh) * W + sw) * C;
           for (int ch = 0; ch < C; ++ch) row[tap * C + ch] = f32_to_bf16_rn(src[ch]);
