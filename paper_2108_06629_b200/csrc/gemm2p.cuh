@@ -287,12 +287,12 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                            "f"(__uint_as_float(r[8 * j + 7]))
                            : "memory");
             }
-            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.W + rowbase + n), "f"(w[2 * j].x),
+            asm volatile("st.global.cs.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.W + rowbase + n), "f"(w[2 * j].x),
                          "f"(w[2 * j].y), "f"(w[2 * j].z), "f"(w[2 * j].w), "f"(w[2 * j + 1].x), "f"(w[2 * j + 1].y), "f"(w[2 * j + 1].z),
                          "f"(w[2 * j + 1].w)
                          : "memory");
             if (mom)
-              asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.mW + rowbase + n), "f"(mm[2 * j].x),
+              asm volatile("st.global.cs.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.mW + rowbase + n), "f"(mm[2 * j].x),
                            "f"(mm[2 * j].y), "f"(mm[2 * j].z), "f"(mm[2 * j].w), "f"(mm[2 * j + 1].x), "f"(mm[2 * j + 1].y),
                            "f"(mm[2 * j + 1].z), "f"(mm[2 * j + 1].w)
                            : "memory");
@@ -302,7 +302,7 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 #pragma unroll
             for (int j = 0; j < 2; ++j)
               if (nc + 16 * j < p.N)
-                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(rdst + 16 * j), "r"(packed[8 * j]),
+                asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(rdst + 16 * j), "r"(packed[8 * j]),
                              "r"(packed[8 * j + 1]), "r"(packed[8 * j + 2]), "r"(packed[8 * j + 3]), "r"(packed[8 * j + 4]),
                              "r"(packed[8 * j + 5]), "r"(packed[8 * j + 6]), "r"(packed[8 * j + 7])
                              : "memory");
