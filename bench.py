@@ -84,7 +84,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "20"],
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -634,7 +634,7 @@ def cpu_baseline(wl):
             "sample": "%d whole minibatches of %d, full-size layers, %.1f s" % (n, B, dt)}
 
 
-def supervise(args, limit_s=900.0):
+def supervise(args, limit_s=480.0):
     env = dict(os.environ, LP_BENCH_CHILD="1")
     cmd = [sys.executable, "-X", "faulthandler", os.path.abspath(__file__)] + sys.argv[1:]
     for attempt in (1, 2):
@@ -642,6 +642,12 @@ def supervise(args, limit_s=900.0):
         try:
             out, _ = p.communicate(timeout=limit_s)
         except subprocess.TimeoutExpired:
+            try:      # what the GPU is doing while the child makes no progress
+                q = subprocess.run(["nvidia-smi", "--query-gpu=index,utilization.gpu,clocks.sm,power.draw,memory.used",
+                                    "--format=csv,noheader"], capture_output=True, text=True, timeout=20)
+                note("nvidia-smi: " + q.stdout.strip().replace("\n", " | "))
+            except Exception:
+                pass
             try:
                 p.send_signal(__import__("signal").SIGABRT)     # faulthandler prints the child's Python stack
                 p.wait(timeout=10)
