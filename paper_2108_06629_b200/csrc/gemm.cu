@@ -147,7 +147,9 @@ int gemm_pick_splits(int M, int N, int K, int bn) {
   // 392 k-blocks, one CTA streaming 6.4 MB of weights each): 145 us unsplit, 95 / 74 / 89 us at
   // 2 / 4 / 8 splits.
   const long long tiles = (long long)((M + GEMM_BM - 1) / GEMM_BM) * ((N + bn - 1) / bn);
-  const int automatic = (tiles <= 48 && num_kb >= 256) ? 4 : 1;
+  // Fewer tiles with longer contractions take more splits: about one CTA per SM, never fewer than 64 k-blocks per
+  // split (a single 10-column tile over 100352 inputs, the classifier behind an unpooled 28 x 28 x 128 image: 24 splits).
+  const int automatic = (tiles <= 48 && num_kb >= 256) ? int(std::max<long long>(1, std::min<long long>(std::min<long long>(148 / tiles, num_kb / 64), 64))) : 1;
   int s = g_force_splits > 0 ? g_force_splits : automatic;
   s = std::max(1, std::min(s, num_kb));
   const int per = (num_kb + s - 1) / s;
