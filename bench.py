@@ -288,7 +288,7 @@ class Workload:
                            schedule=schedule, flags=flags, W0=self.W0, b0=self.b0, device=self.dev)
 
 
-def throughput(torch, lpb, w, schedule, steps, warmup, min_seconds, stream, flags=0):
+def throughput(torch, lpb, w, schedule, steps, warmup, min_seconds, stream, flags=0, before_timing=None):
     """samples/s of one handle: warm-up (fills every ring), then repeated blocks of `steps` steps."""
     tr = w.trainer(lpb, schedule, flags)
     stage, delays, slots = tr.get_schedule()
@@ -297,6 +297,8 @@ def throughput(torch, lpb, w, schedule, steps, warmup, min_seconds, stream, flag
         tr.step(w.xs[k % w.P], w.ys[k % w.P])
     tr.flush()
     torch.cuda.synchronize()
+    if before_timing is not None:
+        before_timing()
     l0 = tr.kernel_launches()
     ts = repeat_blocks(lambda: timed_block(torch, tr, w.xs, w.ys, steps, stream), min_seconds)
     launches = (tr.kernel_launches() - l0) // len(ts)
@@ -505,10 +507,16 @@ def run_ours(args):
 
     # ---- device-resident throughput: blocks of exactly K steps, repeated for >= 1.5 s ------------
     barrier()
-    clocks = ClockSampler(local)
-    time.sleep(0.25)
+    sampler = {}
+
+    def start_sampler():
+        # clocks and throttle reasons DURING the timed region only: the sampler (an nvidia-smi loop) starts once
+        # the handle exists and the rings are warm, and stops after the end-to-end blocks
+        sampler["clocks"] = ClockSampler(local)
+        time.sleep(0.25)
     tr, ts, launches, prewarm, (stage, delays, slots) = throughput(torch, lpb, w, sched, args.steps, args.warmup,
-                                                                    args.min_seconds, stream)
+                                                                    args.min_seconds, stream, before_timing=start_sampler)
+    clocks = sampler["clocks"]
     barrier()
     dev_sum = summarize(ts, args.steps)
     ms = max_over_ranks(dev_sum["ms_per_step"] * args.steps)
