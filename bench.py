@@ -209,11 +209,25 @@ def note(msg):
 MIN_TIMED_SECONDS = 1.5     # the timed region is repeated until this much device time has been measured
 
 
+TRACE = os.environ.get("LP_BENCH_TRACE") == "1"   # diagnosis of a stalled run: handles mark task progress
+
+
+def _report_progress(tr, stop):
+    """Every 15 s that a block has not finished: which tasks the device still owes (LP_BENCH_TRACE=1)."""
+    while not stop.wait(15.0):
+        note("still waiting for the device:\n" + tr.task_progress())
+
+
 def timed_block(torch, tr, xs, ys, steps, stream):
     """EXACTLY `steps` lp_step calls + lp_flush between two events on the caller's stream."""
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    stop = None
+    if TRACE:
+        import threading
+        stop = threading.Event()
+        threading.Thread(target=_report_progress, args=(tr, stop), daemon=True).start()
     e0.record(stream)
     P = len(xs)
     for k in range(steps):
@@ -221,6 +235,8 @@ def timed_block(torch, tr, xs, ys, steps, stream):
     tr.flush()
     e1.record(stream)
     torch.cuda.synchronize()
+    if stop is not None:
+        stop.set()
     return e0.elapsed_time(e1)
 
 
@@ -284,6 +300,8 @@ class Workload:
 
     def trainer(self, lpb, schedule, flags=0):
         wl = self.wl
+        if TRACE:
+            flags |= lpb.LP_TRACE_TASKS
         return lpb.Trainer(self.layers, self.B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
                            schedule=schedule, flags=flags, W0=self.W0, b0=self.b0, device=self.dev)
 
@@ -302,6 +320,8 @@ def throughput(torch, lpb, w, schedule, steps, warmup, min_seconds, stream, flag
     l0 = tr.kernel_launches()
     ts = repeat_blocks(lambda: timed_block(torch, tr, w.xs, w.ys, steps, stream), min_seconds)
     launches = (tr.kernel_launches() - l0) // len(ts)
+    if TRACE:
+        note(tr.task_progress())
     rc, detail = tr.device_status()
     if rc != 0:
         raise SystemExit("device status %d (%d)" % (rc, detail))

@@ -55,7 +55,10 @@ enum { LP_CAPTURE_GRADS = 1u, /* keep G of the latest step readable by lp_get_gr
                                /* G is only stored when LP_CAPTURE_GRADS is set                    */
        LP_SERIAL_TASKS = 8u,   /* measurement aid: enqueue every task on the caller's stream, so  */
                                /* that no two kernels overlap and LP_TIME_TASKS times each alone  */
-       LP_RECOMPUTE = 16u };   /* activation recomputation instead of stashing, see below         */
+       LP_RECOMPUTE = 16u,     /* activation recomputation instead of stashing, see below         */
+       LP_TRACE_TASKS = 32u }; /* failure detection aid: a one-thread kernel after every task     */
+                               /* writes a progress mark to pinned host memory, which             */
+                               /* lp_task_progress reads while the device is still busy           */
 /* LP_RECOMPUTE (Section III-A names both stashing and recomputation as what the delays between a and
  * the backward pass may stand for): a layer whose input is produced inside its own stage, and whose
  * delay would need a stash of more than four minibatches, keeps that input (with the stored z and
@@ -235,6 +238,15 @@ int lp_get_loss(lp_handle h, long long step, float* loss);
  * the label is never used as an address).  *detail receives the word.  Blocks until the device
  * is idle. */
 int lp_device_status(lp_handle h, int* detail);
+
+/* Which tasks the device has not finished (needs LP_TRACE_TASKS; the paper has no counterpart: it is
+ * how a stalled pipeline is diagnosed without waiting for it).  Writes to text[capacity] (host, NUL
+ * terminated, truncated to fit) one line per scheduler stream with unfinished work -- tasks done of
+ * tasks enqueued and the next up to three unfinished tasks as kind(layer, minibatch) -- and the
+ * status word, copied on a stream of its own.  Does not wait for the scheduler's streams; call it
+ * from any host thread while another is blocked in a synchronisation.  LP_ERR_NOT_READY without
+ * the flag. */
+int lp_task_progress(lp_handle h, char* text, int capacity);
 
 /* Needs LP_TIME_TASKS.  For task kind LP_TASK_* (plus LP_TASK_CAST = 5): number of kernel
  * launches timed since the last lp_reset_task_times and the sum of their durations in

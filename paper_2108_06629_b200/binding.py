@@ -25,6 +25,7 @@ LP_TIME_TASKS = 2
 LP_UNFUSED_UPDATE = 4
 LP_SERIAL_TASKS = 8
 LP_RECOMPUTE = 16
+LP_TRACE_TASKS = 32
 
 
 class lp_layer(C.Structure):
@@ -78,6 +79,7 @@ def lib():
         "lp_reset_task_times": [vp],
         "lp_get_layer_task_time": [vp, C.c_int, C.c_int, llp, _P(C.c_double)],
         "lp_set_delta_split": [vp, ip, llp, ip],
+        "lp_task_progress": [vp, C.c_char_p, C.c_int],
         "lp_get_task_timeline": [vp, C.c_int, C.c_int, _P(C.c_float), _P(C.c_float), _P(C.c_int)],
         "lp_set_tuning": [C.c_int, C.c_int, C.c_int],
         "lp_destroy": [vp],
@@ -100,7 +102,7 @@ def lib():
 
 EXPORTS = ["lp_plan", "lp_plan_costs", "lp_workspace_size", "lp_create", "lp_step", "lp_flush",
            "lp_get_weights", "lp_get_grads", "lp_debug_read", "lp_debug_write", "lp_debug_run_task", "lp_get_schedule", "lp_get_version_log", "lp_get_loss",
-           "lp_device_status", "lp_get_task_time", "lp_reset_task_times", "lp_get_layer_task_time", "lp_set_delta_split", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
+           "lp_device_status", "lp_task_progress", "lp_get_task_time", "lp_reset_task_times", "lp_get_layer_task_time", "lp_set_delta_split", "lp_get_task_timeline", "lp_kernel_launches", "lp_set_tuning", "lp_last_error", "lp_destroy",
            "lp_gemm_bf16", "lp_gemm_status", "lp_debug_gemm_starved", "lp_softmax_xent_static"]
 
 
@@ -318,6 +320,13 @@ class Trainer:
         n, ms = C.c_longlong(), C.c_double()
         _check(lib().lp_get_layer_task_time(self.h, k, layer, C.byref(n), C.byref(ms)), self.h)
         return n.value, ms.value
+
+    def task_progress(self):
+        """Text: unfinished tasks per scheduler stream and the status word (flags=LP_TRACE_TASKS).
+        Does not wait for the device; callable from a second thread."""
+        buf = C.create_string_buffer(4096)
+        _check(lib().lp_task_progress(self.h, buf, 4096), self.h)
+        return buf.value.decode()
 
     def set_delta_split(self, piece_stage, piece_amount):
         """Divide the delta contractions by output columns as a plan's pieces say (before the first

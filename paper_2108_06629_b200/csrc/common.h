@@ -83,6 +83,8 @@ cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int
 cudaError_t launch_cast_patch_general(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
                                       int* labels_copy, int B, int H, int W, int C, int R, int S, int stride, int pad,
                                       int Ho, int Wo, int ld, cudaStream_t stream);
+// one thread writes `value` to *flag (mapped host memory): the progress mark after a task
+cudaError_t launch_trace_mark(unsigned* flag, unsigned value, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,
                                 float* row_loss, unsigned* ticket, float* loss_out, int B, int C,
                                 int* status, cudaStream_t stream);

@@ -305,7 +305,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // memory over ALL tiles of the CTA; at the end each CTA writes its 5 x 128 x 64 partial sums and
 // a second small kernel adds the CTAs' partials in CTA order and applies Eq. 6.  A layer with
 // 128 output channels takes two such passes (64 channels each).
-constexpr int HALOG_STAGES = 4;
+constexpr int HALOG_STAGES = 5;                                 // 201 KiB: this CTA takes all 512 tensor-memory columns, so no other kernel that allocates any may fit beside it
 constexpr int HALOG_D_OFF = 24576;                              // delta box behind the halo box (1 KiB aligned)
 constexpr int HALOG_STAGE_BYTES = HALOG_D_OFF + GEMM_A_BYTES;   // 40 KiB
 constexpr int HALOG_SMEM_BYTES = HALOG_STAGES * HALOG_STAGE_BYTES + 256 + 1024;

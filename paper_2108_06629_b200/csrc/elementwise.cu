@@ -8,6 +8,15 @@
 
 namespace lp {
 
+__global__ void trace_mark_kernel(unsigned* flag, unsigned value) {
+  *reinterpret_cast<volatile unsigned*>(flag) = value;
+  __threadfence_system();
+}
+cudaError_t launch_trace_mark(unsigned* flag, unsigned value, cudaStream_t stream) {
+  trace_mark_kernel<<<1, 1, 0, stream>>>(flag, value);
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------
 // a^0 = RN_bf16(batch) into the first layer's activation-stash slot; labels are copied
 // into the library's label ring so that the caller may reuse its buffers.

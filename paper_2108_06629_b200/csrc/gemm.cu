@@ -225,7 +225,8 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   if (!a.persistent) s = std::max(2, std::min(s, std::max(a.kb_per_split + (a.upd_tma ? BN / 32 : 0), 2)));
   while (s > 2 && size_t(s) * stage_bytes > size_t(227 * 1024 - 1024 - 512 - 1024 - EPI_TILE_BYTES)) --s;
   a.num_stages = s;
-  const size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0, a.upd_tma != 0);
+  size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0, a.upd_tma != 0);
+  if (a.tmem_policy == TMEM_SINGLE_ALONE) smem = std::max<size_t>(smem, 130 * 1024);   // does not fit beside a pair CTA
   const int grid = int(a.persistent ? std::min<long long>(work, slots) : work);
   // single-wave launches stream their weights once: request them into L2 well ahead of the pipeline
   a.l2_ahead = (a.g.kind == GEOM_PLAIN && work <= slots && a.kb_per_split >= 8) ? g_l2_ahead : 0;
@@ -286,7 +287,7 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   if (!a.upd_tma) um = &no_maps;
   const int stage_bytes = 32 * 1024;
   const int num_kb = (a.K + GEMM_BK - 1) / GEMM_BK;
-  int s = g_force_stages > 0 ? g_force_stages : 3;               // 3 x 32 KiB: two CTAs per SM
+  int s = g_force_stages > 0 ? g_force_stages : (a.tmem_policy == TMEM_PAIR_ALONE ? 6 : 3);   // 3 x 32 KiB: two CTAs per SM; 6: alone
   s = std::max(2, std::min(std::min(s, GEMM_MAX_STAGES), std::max(num_kb + (a.upd_tma ? GEMM2_BN / 64 : 0), 2)));
   const size_t tail = 1024 + 256 + (a.upd_tma ? 1024 + UPD_RING_BYTES : 0);   // alignment slack, barriers, bf16 staging tile
   while (s > 2 && size_t(s) * stage_bytes + tail > 227 * 1024) --s;
@@ -296,6 +297,8 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
   cfg.gridDim = dim3(2 * ((a.M + 255) / 256), (a.N - a.n_begin + BN2 - 1) / BN2, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = size_t(s) * stage_bytes + tail;
+  if (a.tmem_policy == TMEM_PAIR_ALONE)      // (also when a short contraction takes fewer stages)
+    cfg.dynamicSmemBytes = std::max<size_t>(cfg.dynamicSmemBytes, size_t(6) * stage_bytes + tail);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -31,6 +31,19 @@ constexpr int GEMM_BK = 64;          // 64 bf16 = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;   // 16 KiB
 constexpr int GEMM_MAX_STAGES = 8;
+// Tensor-memory allocation must never have to wait.  An SM-pair kernel needs the SAME columns on both SMs
+// of its pair; single-CTA kernels resident on those SMs hold columns that differ from SM to SM, the pair's
+// allocation then waits for them, and after such waits a later pair CTA was found waiting for ever on
+// an otherwise idle GPU (VGG-type networks, about once in 10^6 pair CTAs; never in networks of pair
+// kernels only).  So the shared-memory request of every kernel is sized such that the CTAs that can
+// be resident together never ask for more than the 512 columns, and pair CTAs never share an SM with a
+// single-CTA kernel's allocation:
+//   TMEM_PAIR_ALONE  (networks that mix the two kinds): a pair CTA takes six operand stages, 193 KiB,
+//                    and is the only CTA with tensor memory on its SM;
+//   TMEM_SINGLE_ALONE (networks of pair kernels with a small single-CTA layer or two): pair CTAs keep three
+//                    stages and share an SM two by two; the single-CTA kernels ask for 130 KiB, which
+//                    does not fit beside a pair CTA.
+enum { TMEM_DEFAULT = 0, TMEM_PAIR_ALONE = 1, TMEM_SINGLE_ALONE = 2 };
 
 enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2, EPI_WGRAD_UPDATE = 3, EPI_DGRAD_UNPOOL = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
@@ -111,6 +124,8 @@ struct GemmArgs {
   float *bb, *bmb, *bdb, *bbring;   // bias master, momentum (may be null), gradient, destination ring slot
   int* status;              // device status word: set non-zero if a bounded wait expires
   long long wait_limit;     // SM cycles after which a wait on a barrier gives up (0 at the call = the default, about 2 s)
+  int tmem_policy;          // host side only, see TMEM_* below
+  int* phase;               // diagnosis of a stall (LP_TRACE_TASKS): eight counters of CTAs past each phase of the pair kernel, or null
   int starve_kb;            // verification of the bounded waits only: the TMA producer skips the last starve_kb k-blocks of
                             // every tile, so the MMA issuer's wait for them must run out (plain GEMM, one tile per CTA)
 };
@@ -501,7 +516,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     fence_barrier_init();
   }
   if (warp == 1) {
+    const long long t_alloc = p.phase != nullptr ? clock64() : 0;
     tmem_alloc(tmem_slot, PERSIST ? 2 * BN : BN);     // a second accumulator only when tiles follow one another
+    if (p.phase != nullptr && lane == 0) {            // (diagnosis: how many allocations had to wait for columns)
+      atomicAdd(p.phase + 9, 1);
+      if (clock64() - t_alloc > 20000) atomicAdd(p.phase + 8, 1);
+    }
     tmem_relinquish();
   }
   tc_fence_before();

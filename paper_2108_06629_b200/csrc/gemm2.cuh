@@ -81,6 +81,10 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
       : "memory");
 }
 
+__device__ __forceinline__ void phase_mark(const GemmArgs& p, int k) {
+  if (p.phase != nullptr) atomicAdd(p.phase + k, 1);
+}
+
 // UTMA (EPI_WGRAD_UPDATE only): Eq. 6 on the accumulator tile with the fp32 master / momentum tile
 // streamed by TMA through the operand ring once the tile's k-blocks have passed -- each CTA fills
 // "chunks" of its own 128 rows x 32 columns (16 KiB + 16 KiB, one stage), its epilogue updates them in
@@ -134,6 +138,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int nb0 = tm.n0 + int(rank) * (BN2 / 2);        // the half of B this CTA stages
 
   if (threadIdx.x == 0) {
+    phase_mark(p, 0);
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
     if (UTMA) {
@@ -150,7 +155,10 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     fence_barrier_init();
   }
   if (warp == 1) {
+    const long long t_alloc = p.phase != nullptr ? clock64() : 0;
     tmem_alloc2(tmem_slot, GEMM2_BN);
+    if (lane == 0) phase_mark(p, 1);
+    if (p.phase != nullptr && lane == 0 && clock64() - t_alloc > 20000) atomicAdd(p.phase + 10, 1);
     tmem_relinquish2();
   }
   tc_fence_before();
@@ -158,6 +166,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   cluster_sync_all();          // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) phase_mark(p, 2);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -236,6 +245,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int f = max(0, chunks_issued - S); f < chunks_issued; ++f)
           mbar_wait(&ufull_bar[(num_kb + f) % S], uint32_t(f / S) & 1u, p.wait_limit);
       }
+      phase_mark(p, 3);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader only)
@@ -271,6 +281,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
       if (!ok) atomicExch(p.status, 12);
       umma2_commit_both(smem_u32(acc_bar));
+      phase_mark(p, 4);
     }
   } else {
     // ------------------------------------------------------------ epilogue (both CTAs, own rows)
@@ -410,12 +421,15 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
   }
   // neither CTA may release shared or tensor memory while its partner can still touch it
+  if (threadIdx.x == 64) phase_mark(p, 5);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();
+  if (threadIdx.x == 0) phase_mark(p, 6);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc2(tmem_base, GEMM2_BN);
+    if (lane == 0) phase_mark(p, 7);
   }
 }
 

@@ -134,6 +134,7 @@ struct lp_ctx {
   int n_stages = 0;
   int stages_used = 0;
   int n_groups = 1;             // stream triples; stage s runs on triple s % n_groups
+  int tmem_policy = 0;          // TMEM_*: how pair and single-CTA kernels keep out of each other's tensor memory
   int classes = 0, ld_cls = 0;
   // shared buffers
   float* zL = nullptr;          // [kDeltaSlots][B][ld_cls] fp32
@@ -171,6 +172,15 @@ struct lp_ctx {
   size_t tpool_next = 0;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed[6];
   std::vector<int> timed_layer[6];             // layer of each timed launch (-1: none)
+  // task progress marks (LP_TRACE_TASKS): per scheduler stream, how many tasks were enqueued and, in
+  // pinned host memory that a one-thread kernel writes after each task, how many have completed
+  struct TraceRec { int kind, layer; long long n; };
+  static constexpr int kTraceRing = 1024;
+  unsigned* trace_done = nullptr;              // [2][streams.size()] pinned, mapped: tasks finished, tasks started
+  std::vector<unsigned> trace_enq;
+  std::vector<std::vector<TraceRec>> trace_ring;
+  cudaStream_t peek_stream = nullptr;          // reads the status word while the scheduler streams are busy
+  int* peek_host = nullptr;
   std::string err;
   int latched = 0;
   char* ws = nullptr;
@@ -441,6 +451,19 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     }
     y.col_chunks = colsum_chunks(y.out_rows);
   }
+  // SM-pair kernels and single-CTA kernels of one handle run concurrently: keep their tensor-memory
+  // allocations on different SMs (see TMEM_* in gemm.cuh).  A network that is pair kernels except for
+  // a layer or two (the classifier) gives those few the large shared-memory request; every other
+  // mixture gives it to the pair kernels.
+  int n_pair = 0, n_single = 0;
+  for (int l = 0; l < n; ++l) {
+    const Layer& y = c->L[l];
+    const bool any_pair = gemm_is_pair(y.bn_f) || (l > 0 && gemm_is_pair(y.bn_d)) || gemm_is_pair(y.bn_g);
+    const bool all_pair = gemm_is_pair(y.bn_f) && (l == 0 || gemm_is_pair(y.bn_d)) && gemm_is_pair(y.bn_g);
+    n_pair += any_pair ? 1 : 0;
+    n_single += all_pair ? 0 : 1;
+  }
+  c->tmem_policy = n_pair == 0 ? TMEM_DEFAULT : (n_single <= 2 && n_single * 4 <= n ? TMEM_SINGLE_ALONE : TMEM_PAIR_ALONE);
   c->classes = layers[n - 1].out;
   c->ld_cls = pad8(c->classes);
 }
@@ -619,6 +642,9 @@ static void destroy_ctx(lp_ctx* c) {
   for (cudaEvent_t e : c->pool) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->jpool) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->tpool) if (e) cudaEventDestroy(e);
+  if (c->trace_done) cudaFreeHost(c->trace_done);
+  if (c->peek_host) cudaFreeHost(c->peek_host);
+  if (c->peek_stream) cudaStreamDestroy(c->peek_stream);
   delete c;
 }
 
@@ -628,7 +654,7 @@ struct TimedScope {
   cudaStream_t st;
   int kind;
   cudaEvent_t e1 = nullptr;
-  TimedScope(lp_ctx* c_, int kind_, cudaStream_t st_, int layer = -1) : c(c_), st(st_), kind(kind_) {
+  TimedScope(lp_ctx* c_, int kind_, cudaStream_t st_, int layer_ = -1) : c(c_), st(st_), kind(kind_), layer(layer_) {
     if ((c->cfg.flags & LP_TIME_TASKS) && c->tpool_next + 2 <= c->tpool.size()) {
       cudaEvent_t e0 = c->tpool[c->tpool_next++];
       e1 = c->tpool[c->tpool_next++];
@@ -636,10 +662,21 @@ struct TimedScope {
       c->timed[kind].push_back({e0, e1});
       c->timed_layer[kind].push_back(layer);
     }
+    if (c->trace_done) {     // runs once everything the task waits for has completed
+      const int si = c->stream_index(st);
+      launch_trace_mark(c->trace_done + c->streams.size() + si, c->trace_enq[si] + 1, st);
+    }
   }
   ~TimedScope() {
     if (e1) cudaEventRecord(e1, st);
+    if (c->trace_done) {
+      const int si = c->stream_index(st);
+      const unsigned seq = ++c->trace_enq[si];
+      c->trace_ring[si][seq % lp_ctx::kTraceRing] = {kind, layer, c->n_steps};
+      launch_trace_mark(c->trace_done + si, seq, st);
+    }
   }
+  int layer = -1;
 };
 
 // ---------------------------------------------------------------------------
@@ -700,6 +737,8 @@ static cudaError_t launch_forward(lp_ctx* c, int l, long long n, int ring_slot, 
   a.act = y.d.act;
   a.bias = y.d.has_bias ? y.bring + size_t(ring_slot) * y.ld_out : nullptr;
   a.status = c->status;
+  a.tmem_policy = c->tmem_policy;
+  a.phase = c->trace_done ? c->status + 8 : nullptr;
   if (last) {
     a.out = nullptr;
     a.out2 = c->zL + size_t(n % kDeltaSlots) * c->cfg.batch * c->ld_cls;
@@ -785,6 +824,8 @@ static cudaError_t launch_delta(lp_ctx* c, int l, long long n, int ring_slot, cu
     }
   }
   a.status = c->status;
+  a.tmem_policy = c->tmem_policy;
+  a.phase = c->trace_done ? c->status + 8 : nullptr;
   a.splits = y.split_d; a.partial = y.part_d; a.tile_counter = y.cnt_d;
   ++c->launches;
   TimedScope ts(c, LP_TASK_DELTA, st, l);
@@ -846,6 +887,8 @@ static cudaError_t launch_G(lp_ctx* c, int l, long long n, cudaStream_t st) {
   if (!y.conv || y.patch) a.N = y.n_in;
   a.ld_out = y.w_ld;
   a.status = c->status;
+  a.tmem_policy = c->tmem_policy;
+  a.phase = c->trace_done ? c->status + 8 : nullptr;
   if (y.conv && !y.patch) a.g = conv_geom(y, GEOM_PIX_K, y.box64, 0, 0, (y.ld_in + y.bn_g - 1) / y.bn_g);
   if (y.split_g > 1) { a.splits = y.split_g; a.partial = y.part_g; a.tile_counter = y.cnt_g; }
   if (fused_update(c)) {
@@ -1023,6 +1066,15 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   c->streams.assign(1, nullptr);
   for (int s = 0; s < c->n_groups; ++s) { c->streams.push_back(c->sF[s]); c->streams.push_back(c->sD[s]); c->streams.push_back(c->sG[s]); }
   c->waited.assign(c->streams.size(), std::vector<long long>(c->streams.size(), 0));
+  if (c->cfg.flags & LP_TRACE_TASKS) {
+    const size_t ns = c->streams.size();
+    LP_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&c->trace_done), 2 * ns * sizeof(unsigned), cudaHostAllocMapped));
+    LP_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&c->peek_host), 128, cudaHostAllocDefault));
+    LP_CUDA(nullptr, cudaStreamCreateWithFlags(&c->peek_stream, cudaStreamNonBlocking));
+    for (size_t i = 0; i < 2 * ns; ++i) c->trace_done[i] = 0;
+    c->trace_enq.assign(ns, 0u);
+    c->trace_ring.assign(ns, std::vector<lp_ctx::TraceRec>(lp_ctx::kTraceRing));
+  }
   if (cfg->flags & LP_TIME_TASKS) {
     c->tpool.assign(2 * 32768, nullptr);
     for (auto& e : c->tpool) LP_CUDA(nullptr, cudaEventCreate(&e));
@@ -1640,6 +1692,46 @@ extern "C" int lp_get_loss(lp_handle h, long long step, float* loss) {
   const Ev& e = h->loss_ev[step % kLossRing];
   if (e.e) LP_CUDA(h, cudaEventSynchronize(e.e));
   LP_CUDA(h, cudaMemcpy(loss, h->loss + (step % kLossRing), 4, cudaMemcpyDeviceToHost));
+  return LP_OK;
+}
+
+extern "C" int lp_task_progress(lp_handle h, char* text, int capacity) {
+  if (!h || !text || capacity < 1) return LP_ERR_INVALID_ARG;
+  if (!h->trace_done) return fail(h, LP_ERR_NOT_READY, "the handle was created without LP_TRACE_TASKS");
+  static const char* kinds[6] = {"forward", "loss", "delta", "G", "update", "cast"};
+  std::string out;
+  char line[400];
+  for (size_t si = 0; si < h->streams.size(); ++si) {
+    const unsigned done = *reinterpret_cast<volatile unsigned*>(h->trace_done + si), enq = h->trace_enq[si];
+    if (done == enq) continue;
+    const char* role = si == 0 ? "caller" : ((si - 1) % 3 == 0 ? "F" : (si - 1) % 3 == 1 ? "delta" : "G");
+    const unsigned started = *reinterpret_cast<volatile unsigned*>(h->trace_done + h->streams.size() + si);
+    snprintf(line, sizeof line, "stream %d (%s, triple %d): %u of %u tasks done, %s; unfinished:", int(si), role,
+             si == 0 ? -1 : int((si - 1) / 3), done, enq, started > done ? "the next one has STARTED" : "the next one has not started");
+    out += line;
+    for (unsigned q = done + 1; q <= enq && q <= done + 3; ++q) {
+      if (enq - q >= unsigned(lp_ctx::kTraceRing)) continue;
+      const lp_ctx::TraceRec& r = h->trace_ring[si][q % lp_ctx::kTraceRing];
+      snprintf(line, sizeof line, " %s(layer %d, minibatch %lld)", r.kind >= 0 && r.kind < 6 ? kinds[r.kind] : "?", r.layer, r.n);
+      out += line;
+    }
+    out += "\n";
+  }
+  // the status word, read on a stream of its own: works while the scheduler's streams are stuck
+  if (cudaMemcpyAsync(h->peek_host, h->status, 128, cudaMemcpyDeviceToHost, h->peek_stream) == cudaSuccess &&
+      cudaStreamSynchronize(h->peek_stream) == cudaSuccess) {
+    snprintf(line, sizeof line, "status word %d\n", h->peek_host[0]);
+    out += line;
+    const int* ph = h->peek_host + 8;
+    snprintf(line, sizeof line, "pair-kernel CTAs past: entry %d, allocation %d, first cluster barrier %d, loads %d, MMAs (leaders) %d, "
+             "epilogue %d, last cluster barrier %d, release %d\n", ph[0], ph[1], ph[2], ph[3], ph[4], ph[5], ph[6], ph[7]);
+    out += line;
+    snprintf(line, sizeof line, "tensor-memory allocations that waited more than 20000 cycles: %d of %d single-CTA, %d of %d pair CTAs\n",
+             ph[8], ph[9], ph[10], ph[1]);
+    out += line;
+  }
+  if (out.empty()) out = "idle\n";
+  snprintf(text, size_t(capacity), "%s", out.c_str());
   return LP_OK;
 }
 

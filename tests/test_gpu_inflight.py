@@ -173,3 +173,36 @@ def test_inflight_unfused_update_and_captured_gradients():
             for sched in (lpb.LP_SCHED_LAYERPIPE, lpb.LP_SCHED_FUSED_B):
                 got, _, _ = run(*args, sched, mode, flags=flags)
                 same_bits(got, ref, ("flags", flags, mode, sched))
+
+
+def test_task_progress_names_the_unfinished_tasks_without_waiting():
+    """LP_TRACE_TASKS: while a bounded gate holds the caller's stream, lp_task_progress (which does
+    not wait for the device) lists the tasks that have not run; after the flush it reports none,
+    and the traced run is bit-identical to the untraced one."""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([264, 192, 320, 40], "gelu")
+    args = (layers, 56, 3, [2, 1, 0], 0.02, 0.9, 6)
+    ref, _, _ = run(*args, lpb.LP_SCHED_LAYERPIPE, "natural")
+    got, _, _ = run(*args, lpb.LP_SCHED_LAYERPIPE, "gated", flags=lpb.LP_TRACE_TASKS)
+    same_bits(got, ref, "traced")
+    W0, b0 = I.initial_weights(layers, 0)
+    tr = lpb.Trainer(layers, 56, 3, delays=[2, 1, 0], lr=0.02, momentum=0.9, flags=lpb.LP_TRACE_TASKS, W0=W0, b0=b0)
+    x, y = I.minibatch(layers, 56, 0)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    torch.cuda.synchronize()
+    torch.cuda._sleep(GATE_CYCLES)
+    tr.step(xd, yd)
+    text = tr.task_progress()            # returns while the gate still holds every task back
+    assert "cast(layer -1, minibatch 0)" in text and "has not started" in text, text
+    assert "status word 0" in text
+    tr.flush()
+    torch.cuda.synchronize()
+    assert tr.task_progress().startswith("status word 0")
+    plain = lpb.Trainer(layers, 56, 3, delays=[2, 1, 0], W0=W0, b0=b0)
+    with pytest.raises(lpb.LayerPipeError) as e:
+        plain.task_progress()
+    assert e.value.code == lpb.LP_ERR_NOT_READY
+    plain.close()
+    tr.close()
