@@ -232,7 +232,7 @@ int lp_get_version_log(lp_handle h, long long step, int* v_fwd, int* v_bwd, int*
  * until that step's loss kernel has finished. */
 int lp_get_loss(lp_handle h, long long step, float* loss);
 
-/* 0, or the status word written by a kernel: a bounded wait that expired (values 1..23: returns
+/* 0, or the status word written by a kernel: a bounded wait that expired (values 1..26: returns
  * LP_ERR_TIMEOUT), or a label outside [0, classes) met by the loss kernel (value 64: returns
  * LP_ERR_INVALID_ARG; that row contributes no one-hot term and the minibatch's loss is NaN --
  * the label is never used as an address).  *detail receives the word.  Blocks until the device

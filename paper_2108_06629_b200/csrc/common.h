@@ -40,7 +40,7 @@ inline int gemm_tile_cols(int bn) { return gemm_is_pair(bn) ? bn / 2 : bn; }   /
 // which: 0 forward (A,B K-major), 1 delta (B MN-major), 2 G (A,B MN-major).
 // Tile width BN is chosen from N and the box sizes of tmA/tmB must match it
 // (see gemm_box_dims).
-int gemm_pick_bn(int which, int M, int N, int K);
+int gemm_pick_bn(int which, int M, int N, int K, bool allow_pair = true);
 void gemm_box_dims(int which, int bn, uint32_t boxA[2], uint32_t boxB[2]);
 // um (EPI_WGRAD_UPDATE only): tensor maps of the master, momentum and destination ring slot; when
 // given, and the launch qualifies, the update's tiles are streamed by TMA.
@@ -83,6 +83,8 @@ cudaError_t launch_cast_patch3x3(const void* batch, int input_is_bf16, const int
 cudaError_t launch_cast_patch_general(const void* batch, int input_is_bf16, const int* labels, __nv_bfloat16* x0,
                                       int* labels_copy, int B, int H, int W, int C, int R, int S, int stride, int pad,
                                       int Ho, int Wo, int ld, cudaStream_t stream);
+// diagnosis: the per-SM tensor-memory table (160 x 16 ints of device memory, zeroed) that the kernels keep, or null
+cudaError_t gemm_set_tmem_table(int* table);
 // one thread writes `value` to *flag (mapped host memory): the progress mark after a task
 cudaError_t launch_trace_mark(unsigned* flag, unsigned value, cudaStream_t stream);
 cudaError_t launch_softmax_xent(const float* zL, int ldz, const int* labels, __nv_bfloat16* delta, int ldd,

@@ -73,7 +73,9 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     fence_barrier_init();
   }
   if (warp == 1) {
+    if (lane == 0) tmem_note_enter(TK_HALO);
     tmem_alloc(tmem_slot, 2 * BN);
+    if (lane == 0) tmem_note_got(TK_HALO, 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -286,6 +288,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 2 * BN);
+    if (lane == 0) tmem_note_freed(TK_HALO, 2 * BN);
   }
 }
 
@@ -336,7 +339,9 @@ conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     fence_barrier_init();
   }
   if (warp == 1) {
+    if (lane == 0) tmem_note_enter(TK_HALO_G);
     tmem_alloc(tmem_slot, 512);
+    if (lane == 0) tmem_note_got(TK_HALO_G, 512);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -437,6 +442,7 @@ conv_halo_g_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
+    if (lane == 0) tmem_note_freed(TK_HALO_G, 512);
   }
 }
 

@@ -1,6 +1,6 @@
 // Host side of the tcgen05 GEMM: tensor-map encoding, tile selection, launch, and the
 // stand-alone lp_gemm_bf16 entry point.
-#include "gemm2p.cuh"
+#include "gemm2q.cuh"
 #include "conv_halo.cuh"
 
 #include <algorithm>
@@ -156,12 +156,12 @@ int gemm_pick_splits(int M, int N, int K, int bn) {
   return (num_kb + per - 1) / per;      // no empty split
 }
 
-int gemm_pick_bn(int which, int M, int N, int K) {
+int gemm_pick_bn(int which, int M, int N, int K, bool allow_pair) {
   if (g_force_bn == 64 || g_force_bn == 128 || g_force_bn == 256 || g_force_bn == GEMM_BN_PAIR) return g_force_bn;
   if (g_force_bn == GEMM_BN_PAIR224) return which == 2 ? GEMM_BN_PAIR : GEMM_BN_PAIR224;
   if (N <= 64) return 64;
   // tensor-bound shapes: 256 x 256 tiles on SM pairs (code GEMM_BN_PAIR)
-  if (M >= 1024 && N >= 1024 && K >= 1024) {
+  if (allow_pair && M >= 1024 && N >= 1024 && K >= 1024) {
     // forward / delta: a 224-column tile where that fills the last round of SM pairs better (cost =
     // rounds of tiles over the pairs x tile width); G keeps 256 (its update streams 64-column fills)
     if (which != 2 && g_force_bn == 0) {
@@ -225,8 +225,7 @@ static cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, Ge
   if (!a.persistent) s = std::max(2, std::min(s, std::max(a.kb_per_split + (a.upd_tma ? BN / 32 : 0), 2)));
   while (s > 2 && size_t(s) * stage_bytes > size_t(227 * 1024 - 1024 - 512 - 1024 - EPI_TILE_BYTES)) --s;
   a.num_stages = s;
-  size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0, a.upd_tma != 0);
-  if (a.tmem_policy == TMEM_SINGLE_ALONE) smem = std::max<size_t>(smem, 130 * 1024);   // does not fit beside a pair CTA
+  const size_t smem = GemmSmem<BN>::bytes(s, a.persistent != 0, a.upd_tma != 0);
   const int grid = int(a.persistent ? std::min<long long>(work, slots) : work);
   // single-wave launches stream their weights once: request them into L2 well ahead of the pipeline
   a.l2_ahead = (a.g.kind == GEOM_PLAIN && work <= slots && a.kb_per_split >= 8) ? g_l2_ahead : 0;
@@ -328,6 +327,18 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
       return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, tmA, tmB, *um, a);
     }
   }
+  if constexpr (!A_MN && BN2 == GEMM2_BN && (MODE == EPI_FPROP || MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL)) {
+    // A pair CTA that has its SM to itself walks the tiles with two accumulators (see gemm2q.cuh)
+    if (a.tmem_policy == TMEM_PAIR_ALONE && a.starve_kb == 0 && g_force_persistent != 0 && g_force_stages == 0) {
+      const int tiles_m = (a.M + 255) / 256, tiles_n = (a.N - a.n_begin + GEMM2_BN - 1) / GEMM2_BN;
+      const int pairs = std::max(1, sm_count() / 2);
+      cfg.gridDim = dim3(2 * std::min(tiles_m * tiles_n, pairs), 1, 1);
+      cfg.blockDim = dim3(GEMM2Q_THREADS, 1, 1);
+      cfg.dynamicSmemBytes = GEMM2Q_SMEM_BYTES;
+      a.num_stages = GEMM2Q_STAGES;
+      return cudaLaunchKernelEx(&cfg, gemm2q_kernel<B_MN, MODE>, tmA, tmB, a, tiles_m, tiles_n);
+    }
+  }
   return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false, BN2>, tmA, tmB, *um, a);
 }
 template <bool A_MN, bool B_MN, int MODE>
@@ -340,6 +351,10 @@ static cudaError_t configure_pair() {
   } else if constexpr (!A_MN) {      // forward / delta also exist with 224-column tiles
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if constexpr (MODE == EPI_FPROP || MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL) {
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm2q_kernel<B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2Q_SMEM_BYTES);
+    }
   }
   return e;
 }
@@ -448,6 +463,12 @@ cudaError_t gemm_launch(int which, int bn, const CUtensorMap& tmA, const CUtenso
   return cudaErrorInvalidValue;
 }
 
+}  // namespace lp
+
+namespace lp {
+cudaError_t gemm_set_tmem_table(int* table) {
+  return cudaMemcpyToSymbol(g_tmem_table, &table, sizeof(table));
+}
 }  // namespace lp
 
 // status word for the stand-alone entry point (handles keep theirs in the workspace)

@@ -31,19 +31,14 @@ constexpr int GEMM_BK = 64;          // 64 bf16 = one 128-byte swizzle row
 constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;   // 16 KiB
 constexpr int GEMM_MAX_STAGES = 8;
-// Tensor-memory allocation must never have to wait.  An SM-pair kernel needs the SAME columns on both SMs
-// of its pair; single-CTA kernels resident on those SMs hold columns that differ from SM to SM, the pair's
-// allocation then waits for them, and after such waits a later pair CTA was found waiting for ever on
-// an otherwise idle GPU (VGG-type networks, about once in 10^6 pair CTAs; never in networks of pair
-// kernels only).  So the shared-memory request of every kernel is sized such that the CTAs that can
-// be resident together never ask for more than the 512 columns, and pair CTAs never share an SM with a
-// single-CTA kernel's allocation:
-//   TMEM_PAIR_ALONE  (networks that mix the two kinds): a pair CTA takes six operand stages, 193 KiB,
-//                    and is the only CTA with tensor memory on its SM;
-//   TMEM_SINGLE_ALONE (networks of pair kernels with a small single-CTA layer or two): pair CTAs keep three
-//                    stages and share an SM two by two; the single-CTA kernels ask for 130 KiB, which
-//                    does not fit beside a pair CTA.
-enum { TMEM_DEFAULT = 0, TMEM_PAIR_ALONE = 1, TMEM_SINGLE_ALONE = 2 };
+// SM-pair kernels (cta_group::2 tensor-memory allocations) and single-CTA kernels (cta_group::1) are not
+// run side by side by one handle: where they alternated on the same SMs a pair CTA was found, about once
+// in 10^6, waiting in tcgen05.alloc for ever on an otherwise idle GPU (every other CTA of its launch
+// had its columns, no bounded wait had expired); handles with one kind only never showed it.  The
+// handle picks the kind (lp_api.cu, shape_layers).  TMEM_PAIR_ALONE is the measurement mode in which
+// a convolutional network runs its wide layers on pairs all the same: a pair CTA then takes 181 - 193
+// KiB of shared memory, so that no single-CTA kernel's allocation shares its SM.
+enum { TMEM_DEFAULT = 0, TMEM_PAIR_ALONE = 1 };
 
 enum { EPI_STORE_F32 = 0, EPI_FPROP = 1, EPI_DGRAD = 2, EPI_WGRAD_UPDATE = 3, EPI_DGRAD_UNPOOL = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
@@ -517,7 +512,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
   if (warp == 1) {
     const long long t_alloc = p.phase != nullptr ? clock64() : 0;
+    if (lane == 0) tmem_note_enter(PERSIST ? TK_GEMM_PERSISTENT : TK_GEMM);
     tmem_alloc(tmem_slot, PERSIST ? 2 * BN : BN);     // a second accumulator only when tiles follow one another
+    if (lane == 0) tmem_note_got(PERSIST ? TK_GEMM_PERSISTENT : TK_GEMM, PERSIST ? 2 * BN : BN);
     if (p.phase != nullptr && lane == 0) {            // (diagnosis: how many allocations had to wait for columns)
       atomicAdd(p.phase + 9, 1);
       if (clock64() - t_alloc > 20000) atomicAdd(p.phase + 8, 1);
@@ -1024,6 +1021,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, PERSIST ? 2 * BN : BN);
+    if (lane == 0) tmem_note_freed(PERSIST ? TK_GEMM_PERSISTENT : TK_GEMM, PERSIST ? 2 * BN : BN);
   }
 }
 

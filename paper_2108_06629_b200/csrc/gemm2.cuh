@@ -156,7 +156,9 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   }
   if (warp == 1) {
     const long long t_alloc = p.phase != nullptr ? clock64() : 0;
+    if (lane == 0) tmem_note_enter(TK_PAIR);
     tmem_alloc2(tmem_slot, GEMM2_BN);
+    if (lane == 0) tmem_note_got(TK_PAIR, GEMM2_BN);
     if (lane == 0) phase_mark(p, 1);
     if (p.phase != nullptr && lane == 0 && clock64() - t_alloc > 20000) atomicAdd(p.phase + 10, 1);
     tmem_relinquish2();
@@ -429,6 +431,7 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc2(tmem_base, GEMM2_BN);
+    if (lane == 0) tmem_note_freed(TK_PAIR, GEMM2_BN);
     if (lane == 0) phase_mark(p, 7);
   }
 }

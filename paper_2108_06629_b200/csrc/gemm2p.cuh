@@ -85,7 +85,9 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     fence_barrier_init();
   }
   if (warp == 1) {
+    if (lane == 0) tmem_note_enter(TK_PAIR_G);
     tmem_alloc2(tmem_slot, 512);
+    if (lane == 0) tmem_note_got(TK_PAIR_G, 512);
     tmem_relinquish2();
   }
   tc_fence_before();
@@ -324,6 +326,7 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc2(tmem_base, 512);
+    if (lane == 0) tmem_note_freed(TK_PAIR_G, 512);
   }
 }
 

@@ -179,6 +179,7 @@ struct lp_ctx {
   unsigned* trace_done = nullptr;              // [2][streams.size()] pinned, mapped: tasks finished, tasks started
   std::vector<unsigned> trace_enq;
   std::vector<std::vector<TraceRec>> trace_ring;
+  int* tmem_table = nullptr;                   // [160][16] per-SM tensor-memory accounting (device)
   cudaStream_t peek_stream = nullptr;          // reads the status word while the scheduler streams are busy
   int* peek_host = nullptr;
   std::string err;
@@ -365,6 +366,7 @@ static size_t carve(lp_ctx* c, char* base) {
   c->ticket = reinterpret_cast<unsigned*>(take(size_t(kDeltaSlots) * 4));
   c->loss = reinterpret_cast<float*>(take(size_t(kLossRing) * 4));
   c->status = reinterpret_cast<int*>(take(256));
+  c->tmem_table = reinterpret_cast<int*>(take(160 * 16 * 4));
   return align_up(off, 256);
 }
 
@@ -418,9 +420,15 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       // pair against single CTA: 512 -> 512 at 28^2 forward 180 / 245 us, delta 189 / 253 us;
       // 256 -> 256 at 56^2 216 / 240 and 230 / 249 us; 512 -> 512 at 14^2 66 / 79 and 67 / 84 us;
       // 128 -> 256 forward (18 k-blocks) is slower as a pair (149 / 131 us) and stays single.
+      // Off by default: a convolutional network always has single-CTA kernels too, and the two kinds of
+      // tensor-memory allocation do not mix (see the end of this function).  LP_CONV_PAIR=1 in the
+      // environment turns the pair tiles on, as persistent CTA pairs that have their SMs to themselves
+      // (gemm2q.cuh; VGG-16 step 7.75 ms against 8.38 ms) -- for measurements and the kernels' parity
+      // tests, not for long runs.
       const bool even_boxes = ((y.in_rows / GEMM_BM) % 2) == 0;
-      if (!y.gen && even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
-      if (!y.gen && even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
+      const bool conv_pair = getenv("LP_CONV_PAIR") != nullptr;
+      if (conv_pair && !y.gen && even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
+      if (conv_pair && !y.gen && even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
       y.split_f = y.split_d = 1;
       const bool tiles_8x16 = !y.gen && (y.imW % 8 == 0) && (y.imH % 16 == 0);
       y.halo_f = !y.patch && tiles_8x16 && y.ld_in <= 64 && y.n_out <= 64;
@@ -451,19 +459,41 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
     }
     y.col_chunks = colsum_chunks(y.out_rows);
   }
-  // SM-pair kernels and single-CTA kernels of one handle run concurrently: keep their tensor-memory
-  // allocations on different SMs (see TMEM_* in gemm.cuh).  A network that is pair kernels except for
-  // a layer or two (the classifier) gives those few the large shared-memory request; every other
-  // mixture gives it to the pair kernels.
-  int n_pair = 0, n_single = 0;
+  // One kind of tensor-memory allocation per handle.  SM-pair kernels (tcgen05 cta_group::2) and
+  // single-CTA kernels (cta_group::1) that alternate on the same SMs ended, about once in 10^6 pair
+  // CTAs, with a pair CTA waiting in tcgen05.alloc for ever on an otherwise idle GPU; handles of one
+  // kind only never did.  So a fully connected network whose layers are mostly wide runs EVERY
+  // contraction on SM pairs (the narrow classifier too: a 256-column tile that is mostly padding
+  // costs microseconds), and every other network runs none there.
+  const int B = c->cfg.batch;
+  bool any_conv = false;
+  int fc_pair = 0;
   for (int l = 0; l < n; ++l) {
     const Layer& y = c->L[l];
-    const bool any_pair = gemm_is_pair(y.bn_f) || (l > 0 && gemm_is_pair(y.bn_d)) || gemm_is_pair(y.bn_g);
-    const bool all_pair = gemm_is_pair(y.bn_f) && (l == 0 || gemm_is_pair(y.bn_d)) && gemm_is_pair(y.bn_g);
-    n_pair += any_pair ? 1 : 0;
-    n_single += all_pair ? 0 : 1;
+    any_conv = any_conv || y.conv;
+    if (!y.conv && (gemm_is_pair(y.bn_f) || (l > 0 && gemm_is_pair(y.bn_d)) || gemm_is_pair(y.bn_g))) ++fc_pair;
   }
-  c->tmem_policy = n_pair == 0 ? TMEM_DEFAULT : (n_single <= 2 && n_single * 4 <= n ? TMEM_SINGLE_ALONE : TMEM_PAIR_ALONE);
+  const bool conv_pair = getenv("LP_CONV_PAIR") != nullptr;     // measurement aid, see the convolution branch above
+  if (!conv_pair) {
+    const bool pure_pair = !any_conv && fc_pair * 2 >= n;
+    for (int l = 0; l < n; ++l) {
+      Layer& y = c->L[l];
+      if (y.conv) continue;
+      if (pure_pair) {
+        if (!gemm_is_pair(y.bn_f)) y.bn_f = GEMM_BN_PAIR;
+        if (!gemm_is_pair(y.bn_d)) y.bn_d = GEMM_BN_PAIR;
+        if (!gemm_is_pair(y.bn_g)) y.bn_g = GEMM_BN_PAIR;
+        y.split_f = y.split_d = 1;
+      } else if (fc_pair > 0) {
+        y.bn_f = gemm_pick_bn(0, B, y.n_out, y.n_in, false);
+        y.bn_d = gemm_pick_bn(1, B, y.n_in, y.n_out, false);
+        y.bn_g = gemm_pick_bn(2, y.n_out, y.n_in, B, false);
+        y.split_f = gemm_is_pair(y.bn_f) ? 1 : gemm_pick_splits(B, y.n_out, y.n_in, y.bn_f);
+        y.split_d = gemm_is_pair(y.bn_d) ? 1 : gemm_pick_splits(B, y.n_in, y.n_out, y.bn_d);
+      }
+    }
+  }
+  c->tmem_policy = conv_pair ? TMEM_PAIR_ALONE : TMEM_DEFAULT;
   c->classes = layers[n - 1].out;
   c->ld_cls = pad8(c->classes);
 }
@@ -642,7 +672,7 @@ static void destroy_ctx(lp_ctx* c) {
   for (cudaEvent_t e : c->pool) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->jpool) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : c->tpool) if (e) cudaEventDestroy(e);
-  if (c->trace_done) cudaFreeHost(c->trace_done);
+  if (c->trace_done) { gemm_set_tmem_table(nullptr); cudaFreeHost(c->trace_done); }
   if (c->peek_host) cudaFreeHost(c->peek_host);
   if (c->peek_stream) cudaStreamDestroy(c->peek_stream);
   delete c;
@@ -1069,7 +1099,8 @@ extern "C" int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, i
   if (c->cfg.flags & LP_TRACE_TASKS) {
     const size_t ns = c->streams.size();
     LP_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&c->trace_done), 2 * ns * sizeof(unsigned), cudaHostAllocMapped));
-    LP_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&c->peek_host), 128, cudaHostAllocDefault));
+    LP_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&c->peek_host), 128 + 160 * 16 * 4, cudaHostAllocDefault));
+    LP_CUDA(nullptr, gemm_set_tmem_table(c->tmem_table));
     LP_CUDA(nullptr, cudaStreamCreateWithFlags(&c->peek_stream, cudaStreamNonBlocking));
     for (size_t i = 0; i < 2 * ns; ++i) c->trace_done[i] = 0;
     c->trace_enq.assign(ns, 0u);
@@ -1729,6 +1760,20 @@ extern "C" int lp_task_progress(lp_handle h, char* text, int capacity) {
     snprintf(line, sizeof line, "tensor-memory allocations that waited more than 20000 cycles: %d of %d single-CTA, %d of %d pair CTAs\n",
              ph[8], ph[9], ph[10], ph[1]);
     out += line;
+  }
+  if (cudaMemcpyAsync(h->peek_host + 32, h->tmem_table, 160 * 16 * 4, cudaMemcpyDeviceToHost, h->peek_stream) == cudaSuccess &&
+      cudaStreamSynchronize(h->peek_stream) == cudaSuccess) {
+    static const char* tk[8] = {"-", "gemm", "gemm persistent", "pair", "pair G", "pair forward/delta", "halo", "halo G"};
+    for (int sm = 0; sm < 160; ++sm) {
+      const int* r = h->peek_host + 32 + 16 * sm;
+      for (int k = 1; k < 8; ++k)
+        if (r[k] != 0) {
+          snprintf(line, sizeof line, "SM %d: %d CTA(s) of kernel '%s' inside tcgen05.alloc; this library's CTAs hold %d columns there; "
+                   "latest deallocation by '%s', latest allocation by '%s', %d allocations so far\n",
+                   sm, r[k], tk[k], r[8], tk[r[9] & 7], tk[r[10] & 7], r[11]);
+          out += line;
+        }
+    }
   }
   if (out.empty()) out = "idle\n";
   snprintf(text, size_t(capacity), "%s", out.c_str());

@@ -156,6 +156,36 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// Diagnosis of tensor-memory allocation (LP_TRACE_TASKS): a table of 16 words per SM in device memory --
+// [kind] CTAs of kernel kind `kind` (1..7) that are inside tcgen05.alloc right now, [8] columns that this
+// library's CTAs hold there, [9] / [10] kind of the latest deallocation / allocation, [11] allocations.
+// Null unless a tracing handle set it; one word of overhead per allocation otherwise.
+static __device__ int* g_tmem_table = nullptr;   // (one copy per translation unit; every kernel that allocates lives in gemm.cu)
+enum { TK_GEMM = 1, TK_GEMM_PERSISTENT = 2, TK_PAIR = 3, TK_PAIR_G = 4, TK_PAIR_FD = 5, TK_HALO = 6, TK_HALO_G = 7 };
+__device__ __forceinline__ int* tmem_row() {
+  int* t = g_tmem_table;
+  if (t == nullptr) return nullptr;
+  uint32_t smid;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+  return t + 16 * (smid < 160u ? smid : 159u);
+}
+__device__ __forceinline__ void tmem_note_enter(int kind) {
+  if (int* r = tmem_row()) atomicAdd(r + kind, 1);
+}
+__device__ __forceinline__ void tmem_note_got(int kind, int cols) {
+  if (int* r = tmem_row()) {
+    atomicAdd(r + kind, -1);
+    atomicAdd(r + 8, cols);
+    atomicExch(r + 10, kind);
+    atomicAdd(r + 11, 1);
+  }
+}
+__device__ __forceinline__ void tmem_note_freed(int kind, int cols) {
+  if (int* r = tmem_row()) {
+    atomicAdd(r + 8, -cols);
+    atomicExch(r + 9, kind);
+  }
+}
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }

@@ -26,3 +26,10 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture
+def conv_pair_tiles(monkeypatch):
+    """Handles created in this test run wide convolution layers as SM-pair tiles (off by default: a
+    handle keeps to one kind of tensor-memory allocation; the environment variable is read at lp_create)."""
+    monkeypatch.setenv("LP_CONV_PAIR", "1")

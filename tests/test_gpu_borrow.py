@@ -98,7 +98,7 @@ def test_split_delta_fc_sm_pair_tiles():
     _split_delta_case(layers, 300, 3, {1: (1, 1), 2: (3, 1)}, tile_n=512, expect_cols=[0, 768, 512])
 
 
-def test_split_delta_convolution_single_cta_and_pair_tiles():
+def test_split_delta_convolution_single_cta_and_pair_tiles(conv_pair_tiles):
     from paper_2108_06629_b200 import inputs as I
     layers = I.vgg(8, [384, 384, 384], [10])
     # batch 6: three 128-pixel boxes (odd) -> single-CTA 128-wide tiles, 384 input channels = 3 tiles

@@ -49,7 +49,7 @@ def test_case_mlp8_layer_shapes_weight_streaming():
 
 def test_case_vgg_block_shapes():
     """Convolution layers of the VGG workloads at reduced batch: 64 -> 64 at 112 x 112 (halo-tile kernels),
-    128 -> 128 at 56 x 56 (general kernel), 256 -> 256 and 512 -> 512 at 28 x 28 (SM-pair tiles)."""
+    128 -> 128 at 56 x 56, 256 -> 256 and 512 -> 512 at 28 x 28 (general kernel; SM-pair tiles with LP_CONV_PAIR=1)."""
     from paper_2108_06629_b200 import inputs as I
     _steps(I.vgg(112, [64, 64, "P", 128, 128, "P", 256, 256, 512, 512], [10]), 8, 4)
 

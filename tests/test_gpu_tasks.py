@@ -280,12 +280,16 @@ def test_tasks_mlp16_8192_full_size_one_minibatch():
     print("mlp16_8192 worst per-task errors", w)
 
 
-def test_tasks_vgg16_224_full_size_one_minibatch():
+@pytest.mark.parametrize("pair_tiles", [False, True])
+def test_tasks_vgg16_224_full_size_one_minibatch(pair_tiles, monkeypatch):
     """VGG-16 shapes at 224 x 224, batch 64, planned stages: pixel boxes with seven tiles per row
     (224 / 112 / 56 / 28 pixels), the 2 x 2 x 32 box at 14 x 14, split-K G over 3.2 M pixel rows,
-    SM-pair convolution tiles, the patch-matrix first layer, the halo-tile 64 -> 64 layer, the
-    automatic split-K and the persistent streamed update of the 25088 -> 4096 layer."""
+    the patch-matrix first layer, the halo-tile 64 -> 64 layer, the automatic split-K and the
+    persistent streamed update of the 25088 -> 4096 layer; with pair_tiles the layers of 256 and 512
+    channels as persistent SM-pair tiles."""
     from paper_2108_06629_b200 import inputs as I
+    if pair_tiles:
+        monkeypatch.setenv("LP_CONV_PAIR", "1")
     wl = I.WORKLOADS["vgg16_224"]
     w = run_teacher_forced(wl["layers"], wl["batch"], wl["stages"], wl["delays"], wl["lr"], wl["momentum"], 1)
     print("vgg16_224 worst per-task errors", w)
@@ -299,7 +303,7 @@ def test_tasks_pixel_boxes_with_seven_tiles_per_row():
     run_teacher_forced(layers, 32, 4, None, 0.05, 0.9, 3)
 
 
-def test_tasks_sm_pair_convolution_tiles_at_28_and_14_pixels():
+def test_tasks_sm_pair_convolution_tiles_at_28_and_14_pixels(conv_pair_tiles):
     """256 -> 256 channels at 28 x 28 and (behind a pool) at 14 x 14, batch 64: an even number of
     128-pixel boxes, so forward and delta run as 256-pixel x 256-column tiles on SM pairs."""
     from paper_2108_06629_b200 import inputs as I
