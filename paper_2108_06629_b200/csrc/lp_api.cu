@@ -426,6 +426,13 @@ static void shape_layers(lp_ctx* c, const lp_layer* layers, int n, const std::ve
       // (gemm2q.cuh; VGG-16 step 7.75 ms against 8.38 ms) -- for measurements and the kernels' parity
       // tests, not for long runs.
       const bool even_boxes = ((y.in_rows / GEMM_BM) % 2) == 0;
+      // 128 x 256 single-CTA tiles where gemm_pick_bn's rule for them holds (a long contraction, enough tiles for
+      // one persistent CTA on every SM): a third less operand traffic per multiply-accumulate than 128 x 128
+      const long long row_tiles = y.in_rows / GEMM_BM;
+      if (!y.gen) {      // (VGG-16 step 8.40 -> 8.17 ms)
+        if (y.n_out >= 256 && y.taps * y.ld_in >= 1024 && row_tiles * ((y.n_out + 255) / 256) >= 2 * 148) y.bn_f = 256;
+        if (l > 0 && y.ld_in >= 256 && y.taps * y.n_out >= 1024 && row_tiles * ((y.ld_in + 255) / 256) >= 2 * 148) y.bn_d = 256;
+      }
       const bool conv_pair = getenv("LP_CONV_PAIR") != nullptr;
       if (conv_pair && !y.gen && even_boxes && y.n_out >= 256 && y.ld_in >= 256) y.bn_f = GEMM_BN_PAIR;
       if (conv_pair && !y.gen && even_boxes && l > 0 && y.ld_in >= 256 && y.n_out >= 256) y.bn_d = GEMM_BN_PAIR;
