@@ -239,6 +239,17 @@ def test_tasks_sm_pair_tiles():
             lpb.lp_set_tuning(0, 0, 0)
 
 
+def test_tasks_wide_network_runs_its_narrow_classifier_on_sm_pairs():
+    """A fully connected network whose layers are mostly wide keeps to one kind of tensor-memory
+    allocation: the 10-unit classifier runs on SM-pair tiles too -- forward with N = 10, delta with
+    K = 10 (one zero-filled k-block), G with M = 10 and the streamed update clipped to ten rows.
+    With and without momentum (the persistent and the one-tile G kernel)."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([1024, 1280, 1024, 10], "gelu")
+    run_teacher_forced(layers, 1024, 3, [2, 1, 0], 0.02, 0.9, 3)
+    run_teacher_forced(layers, 1024, 3, [2, 1, 0], 0.02, 0.0, 2)
+
+
 def test_tasks_degenerate_shapes():
     """The paper's bias-free Eq. 1; a single layer (no delta task at all); batch 1; one stage with
     all delays zero (plain backpropagation); a delay larger than the number of steps run."""
