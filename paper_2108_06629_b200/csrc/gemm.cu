@@ -327,16 +327,21 @@ static cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, G
       return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, true>, tmA, tmB, *um, a);
     }
   }
-  if constexpr (!A_MN && BN2 == GEMM2_BN && (MODE == EPI_FPROP || MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL)) {
+  if constexpr (!A_MN && (MODE == EPI_FPROP || MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL)) {
     // A pair CTA that has its SM to itself walks the tiles with two accumulators (see gemm2q.cuh)
-    if (a.tmem_policy == TMEM_PAIR_ALONE && a.starve_kb == 0 && g_force_persistent != 0 && g_force_stages == 0) {
-      const int tiles_m = (a.M + 255) / 256, tiles_n = (a.N - a.n_begin + GEMM2_BN - 1) / GEMM2_BN;
-      const int pairs = std::max(1, sm_count() / 2);
+    const int tiles_m = (a.M + 255) / 256, tiles_n = (a.N - a.n_begin + BN2 - 1) / BN2;
+    const int pairs = std::max(1, sm_count() / 2);
+    // also for the delta contraction of wide fully connected layers (MN-major B: 211 -> 206 us on 2048 x 8192 x 8192
+    // in a burst, 252 -> 246 us in a 300-step run; the forward contraction measures the same either way)
+    const bool long_delta = (MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL) && a.g.kind == GEOM_PLAIN &&
+                            tiles_m * tiles_n >= 2 * pairs && num_kb >= 32;
+    if ((a.tmem_policy == TMEM_PAIR_ALONE || g_force_persistent == 1 || long_delta) && a.starve_kb == 0 && g_force_persistent != 0 &&
+        g_force_stages == 0) {
       cfg.gridDim = dim3(2 * std::min(tiles_m * tiles_n, pairs), 1, 1);
       cfg.blockDim = dim3(GEMM2Q_THREADS, 1, 1);
       cfg.dynamicSmemBytes = GEMM2Q_SMEM_BYTES;
       a.num_stages = GEMM2Q_STAGES;
-      return cudaLaunchKernelEx(&cfg, gemm2q_kernel<B_MN, MODE>, tmA, tmB, a, tiles_m, tiles_n);
+      return cudaLaunchKernelEx(&cfg, gemm2q_kernel<B_MN, MODE, BN2>, tmA, tmB, a, tiles_m, tiles_n);
     }
   }
   return cudaLaunchKernelEx(&cfg, gemm2_tcgen05_kernel<A_MN, B_MN, MODE, false, BN2>, tmA, tmB, *um, a);
@@ -354,6 +359,8 @@ static cudaError_t configure_pair() {
     if constexpr (MODE == EPI_FPROP || MODE == EPI_DGRAD || MODE == EPI_DGRAD_UNPOOL) {
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(gemm2q_kernel<B_MN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2Q_SMEM_BYTES);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm2q_kernel<B_MN, MODE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2Q_SMEM_BYTES);
     }
   }
   return e;

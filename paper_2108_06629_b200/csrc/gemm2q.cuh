@@ -23,12 +23,12 @@ constexpr int GEMM2Q_STAGES = 5;
 constexpr int GEMM2Q_STAGE = 32 * 1024;
 constexpr int GEMM2Q_SMEM_BYTES = GEMM2Q_STAGES * GEMM2Q_STAGE + EPI_TILE_BYTES + 1024 + 1024;   // 181 KiB: no other allocating kernel fits beside it
 
-template <bool B_MN, int MODE>
+template <bool B_MN, int MODE, int BN2 = GEMM2_BN>
 __global__ void __launch_bounds__(GEMM2Q_THREADS, 1)
 gemm2q_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs p,
               const int tiles_m, const int tiles_n) {
   constexpr int STAGE = GEMM2Q_STAGE, S = GEMM2Q_STAGES;
-  constexpr int BN2 = GEMM2_BN;
+  static_assert(BN2 % 32 == 0 && BN2 >= 64 && BN2 <= 256, "pair tile width");
   constexpr uint32_t kLoadBytes = GEMM_A_BYTES + (B_MN ? 2 * 8192 : (BN2 / 2) * GEMM_BK * 2);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -162,7 +162,7 @@ gemm2q_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         ok = mbar_wait_addr(acce0 + 8u * buf, ((it >> 1) & 1u) ^ 1u, p.wait_limit);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tacc = tmem_base + buf * uint32_t(BN2);
+        const uint32_t tacc = tmem_base + buf * 256u;
         uint32_t acc = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait_addr(full0 + 8u * s, ph, p.wait_limit);
@@ -200,7 +200,7 @@ gemm2q_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     for (int t = pair_id; t < total && good; t += pairs, ++it) {
       const TileMap tm = tile_map(t);
       const uint32_t buf = it & 1u;
-      const uint32_t tacc = tmem_base + buf * uint32_t(BN2);
+      const uint32_t tacc = tmem_base + buf * 256u;
       good = mbar_wait_addr(accf0 + 8u * buf, (it >> 1) & 1u, p.wait_limit);
       good = __all_sync(0xffffffffu, good);
       if (!good) {

@@ -397,5 +397,9 @@ def test_tasks_sm_pair_persistent_g_update():
         run_teacher_forced(I.mlp([520, 328, 600, 75], "gelu"), 300, 3, [2, 1, 0], 0.05, 0.9, 3)
         run_teacher_forced(I.mlp([2600, 2200, 75], "gelu"), 300, 2, [1, 0], 0.05, 0.9, 2)
         run_teacher_forced(I.mlp([2600, 2200, 75], "gelu"), 300, 2, [1, 0], 0.05, 0.0, 2)
+        # (the forced persistent mode also sends forward and delta through the persistent pair kernel with two
+        # accumulators; here with 224-column tiles: 2600 columns = 12 tiles, the last one 136 wide)
+        lpb.lp_set_tuning(448, 0, 512)
+        run_teacher_forced(I.mlp([2600, 2200, 75], "gelu"), 300, 2, [1, 0], 0.05, 0.0, 2)
     finally:
         lpb.lp_set_tuning(0, 0, 0)
