@@ -98,6 +98,14 @@ def test_split_delta_fc_sm_pair_tiles():
     _split_delta_case(layers, 300, 3, {1: (1, 1), 2: (3, 1)}, tile_n=512, expect_cols=[0, 768, 512])
 
 
+def test_split_delta_fc_persistent_pair_kernel():
+    """Batch 2048, 4864 -> 2048: the delta contraction takes 224-column pair tiles (176 of them, 32 k-blocks) and runs
+    as the persistent pair kernel with two accumulators; its two pieces start at column 0 and at a tile boundary."""
+    from paper_2108_06629_b200 import inputs as I
+    layers = I.mlp([1024, 4864, 2048, 75], "gelu")
+    _split_delta_case(layers, 2048, 3, {1: (1, 1), 2: (1, 2)})
+
+
 def test_split_delta_convolution_single_cta_and_pair_tiles(conv_pair_tiles):
     from paper_2108_06629_b200 import inputs as I
     layers = I.vgg(8, [384, 384, 384], [10])
