@@ -251,8 +251,6 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(mm[j].x), "=f"(mm[j].y), "=f"(mm[j].z), "=f"(mm[j].w) : "r"(sM + off));
         }
         tmem_ld_wait();
-        // the slot has been read (the loads above have returned their values before the arrive is performed)
-        mbar_arrive_addr(uempty0 + 8u * u);
         if (c == kChunks - 1) {
           // last read of this accumulator: hand it back to the MMA issuer (in the leader CTA)
           tc_fence_before();
@@ -275,6 +273,11 @@ gemm2p_g_update_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           packed[2 * j] = pack_bf16x2(w[j].x, w[j].y);
           packed[2 * j + 1] = pack_bf16x2(w[j].z, w[j].w);
         }
+        // The slot is handed back only here, after the arithmetic above has consumed every value read from it:
+        // an arrive issued right behind the ld.shared instructions let the refill overwrite, now and then,
+        // the last 16-byte units before those loads had read them (free-running runs differed from
+        // serialised ones in a few float4 per million).
+        mbar_arrive_addr(uempty0 + 8u * u);
         if (row_ok) {
           // 32-byte stores: eight fp32 (or sixteen bf16) of this lane's row per instruction, whole sectors
 #pragma unroll

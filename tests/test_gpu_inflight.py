@@ -206,3 +206,50 @@ def test_task_progress_names_the_unfinished_tasks_without_waiting():
     assert e.value.code == lpb.LP_ERR_NOT_READY
     plain.close()
     tr.close()
+
+
+def test_inflight_mlp16_8192_full_size_bitwise_against_synchronised_run():
+    """The benchmark's own configuration (sixteen 8192 x 8192 layers, batch 2048, planned delays 8 .. 0,
+    SM-pair kernels only, persistent delta and G kernels): twelve minibatches enqueued without any host
+    call in between, under both schedules, give bit for bit the losses and weights of the run that
+    waits for the device after every step.  (The oracle comparison of this configuration is the
+    teacher-forced test of test_gpu_tasks.py; twelve free-running oracle minibatches would take
+    six minutes of host time.)"""
+    import torch
+    from paper_2108_06629_b200 import binding as lpb
+    from paper_2108_06629_b200 import inputs as I
+    wl = I.WORKLOADS["mlp16_8192"]
+    layers, B, steps = wl["layers"], wl["batch"], 12
+    W0, b0 = I.initial_weights(layers, 0)
+    xs, ys = [], []
+    for n in range(3):
+        x, y = I.minibatch(layers, B, n)
+        xs.append(torch.from_numpy(x).cuda())
+        ys.append(torch.from_numpy(y).cuda())
+
+    def go(schedule, mode):
+        tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+                         schedule=schedule, W0=W0, b0=b0)
+        torch.cuda.synchronize()
+        if mode == "gated":
+            torch.cuda._sleep(GATE_CYCLES)
+        for n in range(steps):
+            tr.step(xs[n % 3], ys[n % 3])
+            if mode == "sync":
+                torch.cuda.synchronize()
+        tr.flush()
+        torch.cuda.synchronize()
+        loss = [tr.get_loss(n) for n in range(steps)]
+        assert tr.device_status() == (0, 0)
+        return tr, loss
+
+    ref, ref_loss = go(lpb.LP_SCHED_LAYERPIPE, "sync")
+    assert all(np.isfinite(ref_loss))
+    for sched, mode in ((lpb.LP_SCHED_LAYERPIPE, "natural"), (lpb.LP_SCHED_LAYERPIPE, "gated"), (lpb.LP_SCHED_FUSED_B, "natural")):
+        got, loss = go(sched, mode)
+        assert loss == ref_loss, (sched, mode)
+        for l in range(len(layers)):
+            a, b = got.get_weights(l), ref.get_weights(l)
+            assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and a[2] == b[2] == steps, (sched, mode, l)
+        got.close()
+    ref.close()
