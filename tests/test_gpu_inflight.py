@@ -208,18 +208,23 @@ def test_task_progress_names_the_unfinished_tasks_without_waiting():
     tr.close()
 
 
-def test_inflight_mlp16_8192_full_size_bitwise_against_synchronised_run():
-    """The benchmark's own configuration (sixteen 8192 x 8192 layers, batch 2048, planned delays 8 .. 0,
-    SM-pair kernels only, persistent delta and G kernels): twelve minibatches enqueued without any host
-    call in between, under both schedules, give bit for bit the losses and weights of the run that
-    waits for the device after every step.  (The oracle comparison of this configuration is the
-    teacher-forced test of test_gpu_tasks.py; twelve free-running oracle minibatches would take
-    six minutes of host time.)"""
+@pytest.mark.parametrize("workload, steps, momentum", [("mlp16_8192", 12, None), ("mlp16_8192", 6, 0.9), ("vgg16_224", 10, None),
+                                                       ("sample4_224", 12, None)])
+def test_inflight_full_size_bitwise_against_synchronised_run(workload, steps, momentum):
+    """The large configurations at full size -- mlp16_8192 is the benchmark's own (sixteen 8192 x 8192 layers, batch
+    2048, planned delays 8 .. 0, SM-pair kernels only, persistent delta and G kernels); VGG-16 at 224 x 224 and the
+    paper's sample network are the convolutional ones: the minibatches are enqueued without any host
+    call in between, under both schedules, and give bit for bit the losses and weights of the run that
+    waits for the device after every step; mlp16_8192 also with momentum (the one-tile G kernel with the
+    streamed update instead of the persistent one).  (The oracle comparison of these configurations is the
+    teacher-forced test of test_gpu_tasks.py; free-running oracle minibatches at these sizes would take
+    minutes of host time each.)"""
     import torch
     from paper_2108_06629_b200 import binding as lpb
     from paper_2108_06629_b200 import inputs as I
-    wl = I.WORKLOADS["mlp16_8192"]
-    layers, B, steps = wl["layers"], wl["batch"], 12
+    wl = I.WORKLOADS[workload]
+    layers, B = wl["layers"], wl["batch"]
+    mu = wl["momentum"] if momentum is None else momentum
     W0, b0 = I.initial_weights(layers, 0)
     xs, ys = [], []
     for n in range(3):
@@ -228,7 +233,7 @@ def test_inflight_mlp16_8192_full_size_bitwise_against_synchronised_run():
         ys.append(torch.from_numpy(y).cuda())
 
     def go(schedule, mode):
-        tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=wl["momentum"],
+        tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=mu,
                          schedule=schedule, W0=W0, b0=b0)
         torch.cuda.synchronize()
         if mode == "gated":
