@@ -242,8 +242,11 @@ int lp_device_status(lp_handle h, int* detail);
 /* Which tasks the device has not finished (needs LP_TRACE_TASKS; the paper has no counterpart: it is
  * how a stalled pipeline is diagnosed without waiting for it).  Writes to text[capacity] (host, NUL
  * terminated, truncated to fit) one line per scheduler stream with unfinished work -- tasks done of
- * tasks enqueued and the next up to three unfinished tasks as kind(layer, minibatch) -- and the
- * status word, copied on a stream of its own.  Does not wait for the scheduler's streams; call it
+ * tasks enqueued, whether the next one has started, and the next up to three unfinished tasks as
+ * kind(layer, minibatch) -- then, copied on a stream of its own: the status word, how many CTAs of the
+ * SM-pair kernel have passed each of its phases, how many tensor-memory allocations took more than
+ * 20000 cycles, and every SM on which a CTA sits inside tcgen05.alloc (with the kernel it belongs to
+ * and the columns this library's CTAs hold there).  Does not wait for the scheduler's streams; call it
  * from any host thread while another is blocked in a synchronisation.  LP_ERR_NOT_READY without
  * the flag. */
 int lp_task_progress(lp_handle h, char* text, int capacity);
