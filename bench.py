@@ -433,6 +433,7 @@ def short_measure(torch, lpb, name, dev, stream, peaks, seconds=0.6):
         out["delays"] = delays
         out["launches_per_step"] = launches // steps
     out["speedup_vs_fused_b"] = out["layerpipe"]["samples_per_s"] / out["fused_b"]["samples_per_s"]
+    out["selfcheck"] = free_running_selfcheck(torch, lpb, w, lpb.LP_SCHED_LAYERPIPE)
     wm = work_model(w.layers, w.B, w.wl["momentum"])
     out["step"] = step_figures(wm, out["layerpipe"]["ms_per_step"], peaks)
     del w
@@ -591,6 +592,8 @@ def run_ours(args):
         for kind in kinds:
             kinds[kind]["avg_us_overlapped"] = kinds_live[kind]["avg_us"]
         roof, wm = roofline(args.workload, wl, kinds, peaks)
+        note("self-check: free-running against serialised")
+        selfcheck = free_running_selfcheck(torch, lpb, w, sched)
         note("borrowing report")
         borrowing = borrowing_report(torch, lpb, w, args, stream) if world == 1 else None
         del w
@@ -628,6 +631,7 @@ def run_ours(args):
             "speedup_vs_fused_b": ((value / world) / other["value"] if other["schedule"] == "fused_b"
                                    else other["value"] / (value / world)),
             "borrowing": borrowing,
+            "selfcheck": selfcheck,
             "per_workload": per_workload,
             "cpu_baseline": cpu,
         }
@@ -636,6 +640,32 @@ def run_ours(args):
         dist.destroy_process_group()
     if line is not None:
         print(json.dumps(line))
+
+
+def free_running_selfcheck(torch, lpb, w, sched, steps=6):
+    """The timed mode against the mode in which nothing overlaps: `steps` minibatches enqueued back to back on
+    the scheduler's streams, and the same minibatches with every task on one stream (LP_SERIAL_TASKS).  The
+    kernels are deterministic, so the losses must agree bit for bit; a difference is a hazard the scheduler
+    missed or a race inside a kernel that only other kernels' traffic brings out (from the second step
+    on every loss depends on every earlier update)."""
+    losses = []
+    for flags in (0, lpb.LP_SERIAL_TASKS):
+        tr = w.trainer(lpb, sched, flags)
+        for k in range(steps):
+            tr.step(w.xs[k % w.P], w.ys[k % w.P])
+        tr.flush()
+        torch.cuda.synchronize()
+        losses.append([tr.get_loss(k) for k in range(steps)])
+        rc, detail = tr.device_status()
+        tr.close()
+        del tr
+        torch.cuda.empty_cache()
+        if rc != 0:
+            raise SystemExit("device status %d (%d)" % (rc, detail))
+    same = losses[0] == losses[1]
+    if not same:
+        raise SystemExit("bench.py: free-running losses %s differ from serialised losses %s" % (losses[0], losses[1]))
+    return {"steps": steps, "free_running_losses_equal_serialised": same, "last_loss": losses[0][-1]}
 
 
 def cpu_baseline(wl):
