@@ -216,7 +216,7 @@ def test_inflight_full_size_bitwise_against_synchronised_run(workload, steps, mo
     paper's sample network are the convolutional ones: the minibatches are enqueued without any host
     call in between, under both schedules, and give bit for bit the losses and weights of the run that
     waits for the device after every step, also with the planner's delta'' / delta' pieces executed as two
-    concurrent launches; mlp16_8192 also with momentum (the one-tile G kernel with the
+    concurrent launches, and with recomputation instead of the deep stashes (LP_RECOMPUTE); mlp16_8192 also with momentum (the one-tile G kernel with the
     streamed update instead of the persistent one).  (The oracle comparison of these configurations is the
     teacher-forced test of test_gpu_tasks.py; free-running oracle minibatches at these sizes would take
     minutes of host time each.)"""
@@ -235,9 +235,9 @@ def test_inflight_full_size_bitwise_against_synchronised_run(workload, steps, mo
 
     plan = lpb.lp_plan(layers, B, wl["stages"])
 
-    def go(schedule, mode, split=False):
+    def go(schedule, mode, split=False, flags=0):
         tr = lpb.Trainer(layers, B, wl["stages"], delays=wl["delays"], lr=wl["lr"], momentum=mu,
-                         schedule=schedule, W0=W0, b0=b0)
+                         schedule=schedule, flags=flags, W0=W0, b0=b0)
         if split:        # Algorithm 1's delta'' / delta' pieces as two concurrent launches (Section III-B)
             cols = tr.set_delta_split(plan["piece_stage"], plan["piece_amount"])
             assert workload != "mlp16_8192" or any(c > 0 for c in cols)
@@ -256,10 +256,11 @@ def test_inflight_full_size_bitwise_against_synchronised_run(workload, steps, mo
 
     ref, ref_loss = go(lpb.LP_SCHED_LAYERPIPE, "sync")
     assert all(np.isfinite(ref_loss))
-    for sched, mode, split in ((lpb.LP_SCHED_LAYERPIPE, "natural", False), (lpb.LP_SCHED_LAYERPIPE, "gated", False),
-                               (lpb.LP_SCHED_FUSED_B, "natural", False), (lpb.LP_SCHED_LAYERPIPE, "natural", True)):
-        got, loss = go(sched, mode, split)
-        assert loss == ref_loss, (sched, mode, split)
+    for sched, mode, split, flags in ((lpb.LP_SCHED_LAYERPIPE, "natural", False, 0), (lpb.LP_SCHED_LAYERPIPE, "gated", False, 0),
+                                      (lpb.LP_SCHED_FUSED_B, "natural", False, 0), (lpb.LP_SCHED_LAYERPIPE, "natural", True, 0),
+                                      (lpb.LP_SCHED_LAYERPIPE, "natural", False, lpb.LP_RECOMPUTE)):
+        got, loss = go(sched, mode, split, flags)
+        assert loss == ref_loss, (sched, mode, split, flags)
         for l in range(len(layers)):
             a, b = got.get_weights(l), ref.get_weights(l)
             assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and a[2] == b[2] == steps, (sched, mode, split, l)
