@@ -266,9 +266,3 @@ def test_inflight_full_size_bitwise_against_synchronised_run(workload, steps, mo
             assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and a[2] == b[2] == steps, (sched, mode, split, l)
         got.close()
     ref.close()
-
-
-def test_inflight_vgg16_224_with_sm_pair_convolution_tiles(conv_pair_tiles):
-    """The same comparison with the wide convolution layers on persistent SM-pair tiles (the measurement
-    mode LP_CONV_PAIR=1; a short run)."""
-    test_inflight_full_size_bitwise_against_synchronised_run("vgg16_224", 6, None)
