@@ -132,7 +132,13 @@ int lp_workspace_size(const lp_layer* layers, int n_layers, int n_stages, const 
  * work queue, and a process has CUDA_DEVICE_MAX_CONNECTIONS of those (8 if unset, at most 32),
  * fixed when its CUDA context is created: set the variable to 32 before the first CUDA call.
  * lp_create reads the variable and folds the stages onto (value - 2) / 3 stream triples so that
- * no two of its streams share a queue.
+ * no two of its streams share a queue (LP_STREAM_TRIPLES in the environment overrides the count).
+ * Kernel selection: a handle uses one kind of tensor-memory allocation -- a fully connected network
+ * whose layers are mostly wide (batch, inputs and outputs all >= 1024) runs every contraction on SM
+ * pairs (tcgen05 cta_group::2), every other network runs single-CTA kernels only.  LP_CONV_PAIR=1
+ * in the environment also puts wide convolution layers on SM pairs: a measurement mode, not for
+ * long runs (networks that alternate the two kinds on the same SMs have stalled in tcgen05.alloc
+ * after some 10^6 pair CTAs).  Two handles of different kinds should not run concurrently on one GPU.
  */
 int lp_create(lp_handle* out, const lp_layer* layers, int n_layers, int n_stages,
               const int* stage, const int* delays, const lp_config* cfg,
